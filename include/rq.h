@@ -1,0 +1,198 @@
+/*
+ * rq.h — C ABI of the sparse-decode library: query-aware (Quest-style) sparse
+ * decode attention over exponentially decaying key/value memory, for NVIDIA
+ * B200 (sm_100a).
+ *
+ * The method (paper sections in brackets):
+ *   [Eq. 1]   k~_t = g_t*k~_{t-1} + (1-g_t)*k_t and the same for v with the
+ *             same gate; zero initial state; state kept in fp32.
+ *   [App. A.1, "Sparse inference settings"]  the cache of k~, v~ is split into
+ *             pages (blocks) and every page keeps the per-channel minimum and
+ *             maximum of its stored keys.
+ *   [Eq. 3]   each decode query scores every page by the upper bound
+ *             U_p = sum_i max(q_i*min_p[i], q_i*max_p[i]) and keeps the top
+ *             `budget_pages` pages per head; the first page(s) and the newest
+ *             page(s) are always kept and count inside the budget; equal
+ *             scores go to the lower page index.
+ *   [Eq. 4]   softmax attention over the valid tokens of the kept pages only,
+ *             on the decayed keys and decayed values.
+ *
+ * Conventions
+ *   - Every function returns an int status (RQ_OK = 0, otherwise RQ_ERR_*).
+ *     Argument errors are found on the host before anything is enqueued; no
+ *     function aborts, throws or traps the device.
+ *   - Pointers are DEVICE pointers unless the name of the function ends in
+ *     `_host` or the parameter is documented as host memory.
+ *   - The caller owns every byte of device memory.  The library allocates no
+ *     device memory and keeps no global state; `rq_sizes` tells the caller how
+ *     much to allocate and `rq_cache_init` adopts the buffers.  Buffers must be
+ *     256-byte aligned and must outlive the `rq_cache`.
+ *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = default stream).
+ *     Work is enqueued on it and the call returns without synchronising,
+ *     except where stated.  Calls on one cache must be stream-ordered; two
+ *     calls on the same cache running concurrently race on its workspace.
+ *   - Shapes: B = batch, H = heads (q heads = kv heads), D = head_dim,
+ *     S = page_size.  All sequences of a batch have the same length.
+ *   - Layouts in device memory (row-major, last index contiguous):
+ *       kv        [B][H][page_capacity][2][S][D]  storage dtype; [..][0] keys, [..][1] values
+ *       meta      [B][H][page_capacity][2][D]     storage dtype; [..][0] min,  [..][1] max
+ *       state     [B][H][2][D]                    fp32; [..][0] k~ state, [..][1] v~ state
+ *       workspace opaque
+ *     page_capacity = ceil(capacity_tokens / S).
+ */
+#ifndef RQ_H_
+#define RQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* exported-symbol marker (the library is built with hidden default visibility) */
+#if defined(__GNUC__)
+#define RQ_API __attribute__((visibility("default")))
+#else
+#define RQ_API
+#endif
+
+#define RQ_VERSION_MAJOR 0
+#define RQ_VERSION_MINOR 1
+
+/* status codes */
+#define RQ_OK 0
+#define RQ_ERR_INVALID_ARG 1 /* NULL / misaligned pointer, non-positive size, bad enum    */
+#define RQ_ERR_UNSUPPORTED 2 /* a shape or dtype outside the compiled set (see rq_sizes) */
+#define RQ_ERR_CAPACITY 3    /* the call would exceed capacity_tokens / max_budget_pages  */
+#define RQ_ERR_CUDA 4        /* a CUDA runtime call or launch failed                      */
+#define RQ_ERR_TIMEOUT 5     /* a bounded device-side wait ran out (device status only)   */
+
+/* element types */
+#define RQ_F32 0
+#define RQ_BF16 1
+
+/* Description of a cache.  Supported: head_dim in {64, 128}; page_size in
+ * {16, 64}; dtype and gate_dtype each RQ_F32 or RQ_BF16; capacity such that
+ * page_capacity <= 32768. */
+typedef struct rq_config {
+    int32_t batch;            /* B >= 1                                                     */
+    int32_t heads;            /* H >= 1                                                     */
+    int32_t head_dim;         /* D                                                          */
+    int32_t page_size;        /* S, tokens per page                                         */
+    int64_t capacity_tokens;  /* most tokens a sequence may ever hold                       */
+    int32_t dtype;            /* type of q, k, v, o, the cache and the page bounds          */
+    int32_t gate_dtype;       /* type of g                                                  */
+    int32_t n_sink_pages;     /* first pages always kept (paper: "the first block"); >= 0   */
+    int32_t n_local_pages;    /* newest pages always kept (paper: "local blocks"); >= 0     */
+    int32_t max_budget_pages; /* largest budget_pages any later call will pass              */
+    int32_t reserved;         /* must be 0                                                  */
+} rq_config;
+
+/* Host-side handle: plain data, copyable, holds no resources. */
+typedef struct rq_cache {
+    rq_config cfg;
+    void *kv;
+    void *meta;
+    void *state;
+    void *workspace;
+    int64_t len;           /* tokens currently in every sequence                           */
+    int64_t page_capacity; /* ceil(capacity_tokens / page_size)                            */
+    int64_t reserved[4];
+} rq_cache;
+
+/* Bytes the caller must allocate for a configuration.  Host only, no CUDA
+ * call.  Any output pointer may be NULL.
+ * Errors: INVALID_ARG (NULL cfg, non-positive sizes, bad enums, reserved != 0),
+ * UNSUPPORTED (shape outside the supported set). */
+RQ_API int rq_sizes(const rq_config *cfg, size_t *kv_bytes, size_t *meta_bytes,
+             size_t *state_bytes, size_t *workspace_bytes);
+
+/* Adopt caller-allocated device buffers of at least rq_sizes() bytes each and
+ * start an empty cache: enqueues the clearing of the running state and of the
+ * workspace's status word; kv and meta are not cleared (every page is
+ * initialised when its first token is written).  `out` is host memory.
+ * Errors: as rq_sizes; INVALID_ARG for a NULL or not 256-byte-aligned buffer. */
+RQ_API int rq_cache_init(rq_cache *out, const rq_config *cfg, void *kv, void *meta,
+                  void *state, void *workspace, void *stream);
+
+/* Forget all tokens: len = 0 and zero running state (enqueued on stream). */
+RQ_API int rq_cache_reset(rq_cache *cache, void *stream);
+
+/* Prefill [Eq. 1 + App. A.1]: run the gated decay recurrence over T new tokens,
+ * continuing from the cache's running state (zero for an empty cache), round
+ * every state to the storage dtype, write it to the paged cache at positions
+ * len .. len+T-1, bring the min/max of every touched page up to date, leave
+ * the fp32 state after the last token in `state`, and set len += T.
+ *   k, v : [B][T][H][D] of cfg.dtype, element (b,t,h,d) at
+ *          b*stride_b + t*stride_t + h*stride_h + d  (strides in elements, all
+ *          multiples of 16 bytes; d contiguous; base 16-byte aligned)
+ *   g    : same indexing, of cfg.gate_dtype, values in [0, 1]; the same gate
+ *          drives k and v.
+ * Errors: INVALID_ARG (NULL, T < 0, misaligned), CAPACITY (len + T exceeds
+ * capacity_tokens; nothing is enqueued), CUDA.  T == 0 is a no-op. */
+RQ_API int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
+                   int64_t T, int64_t stride_b, int64_t stride_t, int64_t stride_h,
+                   void *stream);
+
+/* One decode step [Eq. 1, Eq. 3, Eq. 4], in this order: (1) one step of the
+ * recurrence with (k_t, v_t, g_t), append the rounded state to the cache,
+ * update the newest page's min/max, len += 1; (2) score all pages with q;
+ * (3) keep min(budget_pages, #pages) pages per (b,h); (4) attend over their
+ * valid tokens — the query sees its own token.
+ *   q, k_t, v_t, o : [B][H][D] contiguous, cfg.dtype;  g_t : [B][H][D], cfg.gate_dtype
+ *   budget_pages   : 1 .. cfg.max_budget_pages (>= #pages means dense attention)
+ *   scale          : softmax scale; <= 0 selects 1/sqrt(D)
+ *   sel_idx_out    : NULL, or int32 [B][H][budget_pages]; receives the kept
+ *                    page indices in ascending order, unused tail = -1
+ * Errors: INVALID_ARG, CAPACITY (len == capacity_tokens, or budget_pages >
+ * max_budget_pages; nothing is enqueued), CUDA. */
+RQ_API int rq_decode_step(rq_cache *cache, const void *q, const void *k_t, const void *v_t,
+                   const void *g_t, int32_t budget_pages, float scale, void *o,
+                   int32_t *sel_idx_out, void *stream);
+
+/* The same step for callers whose tensors live in HOST memory (pinned memory
+ * makes the copies asynchronous): q, k_t, v_t, g_t are copied to the device,
+ * the step runs, o (and sel_idx_out if not NULL) are copied back to host
+ * memory, all on `stream`.  The outputs are valid after the stream is
+ * synchronised.  Bytes moved per call: 4 inputs + 1 output of B*H*D elements
+ * (+ the index list). */
+RQ_API int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_host,
+                        const void *v_t_host, const void *g_t_host,
+                        int32_t budget_pages, float scale, void *o_host,
+                        int32_t *sel_idx_out_host, void *stream);
+
+/* Stage export [Eq. 3 only]: score and select against the current cache without
+ * changing it.  scores_out: NULL or fp32 [B][H][P] with P = ceil(len / S);
+ * idx_out: int32 [B][H][budget_pages] as in rq_decode_step (must not be NULL).
+ * Errors: INVALID_ARG (also for an empty cache), CAPACITY, CUDA. */
+RQ_API int rq_select_pages(rq_cache *cache, const void *q, int32_t budget_pages,
+                    float *scores_out, int32_t *idx_out, void *stream);
+
+/* Stage export [Eq. 4 only]: attention over caller-chosen pages.
+ *   idx : int32 [B][H][n_idx], page indices in [0, P); duplicates are attended
+ *         twice; an entry < 0 is skipped; an entry >= P is skipped and sets
+ *         the device status to RQ_ERR_INVALID_ARG.
+ * At least one valid page per (b,h) is required for a defined result.
+ * Errors: INVALID_ARG, CAPACITY (n_idx > max_budget_pages), CUDA. */
+RQ_API int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t n_idx,
+                    float scale, void *o, void *stream);
+
+/* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
+RQ_API int64_t rq_cache_len(const rq_cache *cache);
+
+/* Synchronises `stream`, reads the device status word into *status_out (host
+ * memory; RQ_OK if no kernel reported anything) and clears it.
+ * Returns RQ_OK, INVALID_ARG or CUDA. */
+RQ_API int rq_device_status(rq_cache *cache, int32_t *status_out, void *stream);
+
+/* Static text for a status code; never NULL. */
+RQ_API const char *rq_status_string(int status);
+
+/* RQ_VERSION_MAJOR * 1000 + RQ_VERSION_MINOR of the loaded library. */
+RQ_API int rq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RQ_H_ */

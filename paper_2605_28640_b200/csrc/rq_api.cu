@@ -1,0 +1,313 @@
+// Host side of the C ABI declared in rq.h: argument checks, workspace carving
+// and kernel sequencing.  No device memory is allocated here.
+#include <math.h>
+#include <string.h>
+
+#include "rq_internal.h"
+
+namespace rq {
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static int check_config(const rq_config *c)
+{
+    if (!c) return RQ_ERR_INVALID_ARG;
+    if (c->batch < 1 || c->heads < 1 || c->head_dim < 1 || c->page_size < 1 || c->capacity_tokens < 1)
+        return RQ_ERR_INVALID_ARG;
+    if ((c->dtype != RQ_F32 && c->dtype != RQ_BF16) || (c->gate_dtype != RQ_F32 && c->gate_dtype != RQ_BF16))
+        return RQ_ERR_INVALID_ARG;
+    if (c->n_sink_pages < 0 || c->n_local_pages < 0 || c->max_budget_pages < 1 || c->reserved != 0)
+        return RQ_ERR_INVALID_ARG;
+    if (c->head_dim != 64 && c->head_dim != 128) return RQ_ERR_UNSUPPORTED;
+    if (c->page_size != 16 && c->page_size != 64) return RQ_ERR_UNSUPPORTED;
+    const int64_t pc = (c->capacity_tokens + c->page_size - 1) / c->page_size;
+    if (pc > (int64_t)kTopkThreads * kTopkMaxPerThread) return RQ_ERR_UNSUPPORTED;
+    if ((int64_t)c->batch * c->heads > 65535) return RQ_ERR_UNSUPPORTED;
+    return RQ_OK;
+}
+
+static size_t elem_size(int dtype) { return dtype == RQ_BF16 ? 2 : 4; }
+
+WorkspaceLayout workspace_layout(const rq_config &c)
+{
+    WorkspaceLayout w;
+    const size_t BH = (size_t)c.batch * c.heads;
+    const size_t pc = (size_t)((c.capacity_tokens + c.page_size - 1) / c.page_size);
+    const int ct = scan_chunk_tokens(c.head_dim, c.dtype);
+    w.scan_chunks_cap = (c.capacity_tokens + ct - 1) / ct + 1;
+    size_t off = 0;
+    w.status = off;  off += align256(64 * sizeof(int32_t));
+    w.scores = off;  off += align256(BH * pc * sizeof(float));
+    w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
+    w.partial = off; off += align256(BH * kMaxSplits * (size_t)(c.head_dim + 2) * sizeof(float));
+    w.agg = off;     off += align256(BH * (size_t)w.scan_chunks_cap * 3 * c.head_dim * sizeof(float));
+    w.staging = off; off += align256(5 * BH * (size_t)c.head_dim * 4);
+    w.total = off;
+    return w;
+}
+
+static int sm_count()
+{
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            cached = kTargetSMs;
+    }
+    return cached;
+}
+
+static DecodeArgs decode_args(const rq_cache *c, int64_t len)
+{
+    DecodeArgs a;
+    a.kv = c->kv; a.meta = c->meta; a.state = (float *)c->state;
+    a.B = c->cfg.batch; a.H = c->cfg.heads; a.D = c->cfg.head_dim; a.S = c->cfg.page_size;
+    a.dtype = c->cfg.dtype; a.gate_dtype = c->cfg.gate_dtype;
+    a.len = len; a.page_cap = c->page_capacity;
+    a.n_sink = c->cfg.n_sink_pages; a.n_local = c->cfg.n_local_pages;
+    a.status = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).status);
+    return a;
+}
+
+static bool aligned(const void *p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+
+static int check_cache(const rq_cache *c)
+{
+    if (!c || !c->kv || !c->meta || !c->state || !c->workspace) return RQ_ERR_INVALID_ARG;
+    return check_config(&c->cfg);
+}
+
+// score + select into `idx` (device, stride idx_stride), for a cache of length len
+static int select_into(const rq_cache *c, int64_t len, const void *q, int budget, float *scores,
+                       int32_t *idx, int idx_stride, cudaStream_t s)
+{
+    DecodeArgs a = decode_args(c, len);
+    if (launch_score(a, q, scores, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (launch_topk(a, scores, budget, idx, idx_stride, s) != cudaSuccess) return RQ_ERR_CUDA;
+    return RQ_OK;
+}
+
+static int attend_from(const rq_cache *c, int64_t len, const void *q, const int32_t *idx, int n_idx,
+                       int idx_stride, float scale, void *o, cudaStream_t s)
+{
+    DecodeArgs a = decode_args(c, len);
+    const WorkspaceLayout w = workspace_layout(c->cfg);
+    float *partial = (float *)((char *)c->workspace + w.partial);
+    if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
+    const int nsplit = choose_splits(a.B * a.H, n_idx, sm_count());
+    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, o, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    return RQ_OK;
+}
+
+}  // namespace rq
+
+using namespace rq;
+
+extern "C" {
+
+int rq_sizes(const rq_config *cfg, size_t *kv_bytes, size_t *meta_bytes, size_t *state_bytes,
+             size_t *workspace_bytes)
+{
+    const int rc = check_config(cfg);
+    if (rc != RQ_OK) return rc;
+    const size_t BH = (size_t)cfg->batch * cfg->heads;
+    const size_t pc = (size_t)((cfg->capacity_tokens + cfg->page_size - 1) / cfg->page_size);
+    const size_t es = elem_size(cfg->dtype);
+    if (kv_bytes) *kv_bytes = BH * pc * 2 * cfg->page_size * cfg->head_dim * es;
+    if (meta_bytes) *meta_bytes = BH * pc * 2 * cfg->head_dim * es;
+    if (state_bytes) *state_bytes = BH * 2 * cfg->head_dim * sizeof(float);
+    if (workspace_bytes) *workspace_bytes = workspace_layout(*cfg).total;
+    return RQ_OK;
+}
+
+int rq_cache_init(rq_cache *out, const rq_config *cfg, void *kv, void *meta, void *state,
+                  void *workspace, void *stream)
+{
+    if (!out) return RQ_ERR_INVALID_ARG;
+    const int rc = check_config(cfg);
+    if (rc != RQ_OK) return rc;
+    if (!kv || !meta || !state || !workspace) return RQ_ERR_INVALID_ARG;
+    if (!aligned(kv, 256) || !aligned(meta, 256) || !aligned(state, 256) || !aligned(workspace, 256))
+        return RQ_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    out->cfg = *cfg;
+    out->kv = kv; out->meta = meta; out->state = state; out->workspace = workspace;
+    out->page_capacity = (cfg->capacity_tokens + cfg->page_size - 1) / cfg->page_size;
+    return rq_cache_reset(out, stream);
+}
+
+int rq_cache_reset(rq_cache *cache, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t BH = (size_t)cache->cfg.batch * cache->cfg.heads;
+    const WorkspaceLayout w = workspace_layout(cache->cfg);
+    if (cudaMemsetAsync(cache->state, 0, BH * 2 * cache->cfg.head_dim * sizeof(float), s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    if (cudaMemsetAsync((char *)cache->workspace + w.status, 0, 64 * sizeof(int32_t), s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    cache->len = 0;
+    return RQ_OK;
+}
+
+int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g, int64_t T,
+                   int64_t stride_b, int64_t stride_t, int64_t stride_h, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (T < 0) return RQ_ERR_INVALID_ARG;
+    if (T == 0) return RQ_OK;
+    if (!k || !v || !g) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    // 16-byte vectors of the narrower of the two element types must stay aligned
+    const size_t es = elem_size(c.dtype), gs = elem_size(c.gate_dtype);
+    const size_t emin = es < gs ? es : gs;
+    if (!aligned(k, 16) || !aligned(v, 16) || !aligned(g, 16)) return RQ_ERR_INVALID_ARG;
+    if (stride_b < 0 || stride_t < 0 || stride_h < 0) return RQ_ERR_INVALID_ARG;
+    if ((stride_b * emin) % 16 || (stride_t * emin) % 16 || (stride_h * emin) % 16) return RQ_ERR_INVALID_ARG;
+    if (cache->len + T > c.capacity_tokens) return RQ_ERR_CAPACITY;
+    const WorkspaceLayout w = workspace_layout(c);
+    ScanArgs a;
+    a.k = k; a.v = v; a.g = g;
+    a.sb = stride_b; a.st = stride_t; a.sh = stride_h;
+    a.kv = cache->kv; a.meta = cache->meta; a.state = (float *)cache->state;
+    a.agg = (float *)((char *)cache->workspace + w.agg);
+    a.B = c.batch; a.H = c.heads; a.D = c.head_dim; a.S = c.page_size;
+    a.dtype = c.dtype; a.gate_dtype = c.gate_dtype;
+    a.len0 = cache->len; a.T = T; a.page_cap = cache->page_capacity; a.chunks_cap = w.scan_chunks_cap;
+    if (launch_scan(a, (cudaStream_t)stream) != cudaSuccess) return RQ_ERR_CUDA;
+    cache->len += T;
+    return RQ_OK;
+}
+
+int rq_decode_step(rq_cache *cache, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                   int32_t budget_pages, float scale, void *o, int32_t *sel_idx_out, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q || !k_t || !v_t || !g_t || !o || budget_pages < 1) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    if (budget_pages > c.max_budget_pages) return RQ_ERR_CAPACITY;
+    if (cache->len >= c.capacity_tokens) return RQ_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    const WorkspaceLayout w = workspace_layout(c);
+    float *scores = (float *)((char *)cache->workspace + w.scores);
+    int32_t *sel = sel_idx_out ? sel_idx_out : (int32_t *)((char *)cache->workspace + w.sel);
+
+    DecodeArgs a = decode_args(cache, cache->len);
+    if (launch_update(a, k_t, v_t, g_t, s) != cudaSuccess) return RQ_ERR_CUDA;
+    cache->len += 1;
+    const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
+    int st = select_into(cache, cache->len, q, budget_pages, scores, sel, budget_pages, s);
+    if (st != RQ_OK) return st;
+    const int n_idx = (int)(budget_pages < P ? budget_pages : P);
+    return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s);
+}
+
+int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_host,
+                        const void *v_t_host, const void *g_t_host, int32_t budget_pages, float scale,
+                        void *o_host, int32_t *sel_idx_out_host, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q_host || !k_t_host || !v_t_host || !g_t_host || !o_host || budget_pages < 1)
+        return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    if (budget_pages > c.max_budget_pages) return RQ_ERR_CAPACITY;
+    if (cache->len >= c.capacity_tokens) return RQ_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    const WorkspaceLayout w = workspace_layout(c);
+    const size_t n = (size_t)c.batch * c.heads * c.head_dim;
+    const size_t slot = n * 4;
+    char *stg = (char *)cache->workspace + w.staging;
+    void *dq = stg, *dk = stg + slot, *dv = stg + 2 * slot, *dg = stg + 3 * slot, *dout = stg + 4 * slot;
+    const size_t eb = n * elem_size(c.dtype), gb = n * elem_size(c.gate_dtype);
+    if (cudaMemcpyAsync(dq, q_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk, k_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dg, g_t_host, gb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    int32_t *sel = (int32_t *)((char *)cache->workspace + w.sel);
+    const int st = rq_decode_step(cache, dq, dk, dv, dg, budget_pages, scale, dout,
+                                  sel_idx_out_host ? sel : nullptr, stream);
+    if (st != RQ_OK) return st;
+    if (cudaMemcpyAsync(o_host, dout, eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (sel_idx_out_host) {
+        const size_t ib = (size_t)c.batch * c.heads * budget_pages * sizeof(int32_t);
+        if (cudaMemcpyAsync(sel_idx_out_host, sel, ib, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return RQ_ERR_CUDA;
+    }
+    return RQ_OK;
+}
+
+int rq_select_pages(rq_cache *cache, const void *q, int32_t budget_pages, float *scores_out,
+                    int32_t *idx_out, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q || !idx_out || budget_pages < 1 || cache->len < 1) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    if (budget_pages > c.max_budget_pages) return RQ_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    const WorkspaceLayout w = workspace_layout(c);
+    float *scores = (float *)((char *)cache->workspace + w.scores);
+    const int st = select_into(cache, cache->len, q, budget_pages, scores, idx_out, budget_pages, s);
+    if (st != RQ_OK) return st;
+    if (scores_out) {
+        const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
+        // workspace rows are page_capacity apart; the caller's are P apart
+        if (cudaMemcpy2DAsync(scores_out, (size_t)P * sizeof(float), scores,
+                              (size_t)cache->page_capacity * sizeof(float), (size_t)P * sizeof(float),
+                              (size_t)c.batch * c.heads, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return RQ_ERR_CUDA;
+    }
+    return RQ_OK;
+}
+
+int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t n_idx, float scale,
+                    void *o, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q || !idx || !o || n_idx < 1 || cache->len < 1) return RQ_ERR_INVALID_ARG;
+    if (n_idx > cache->cfg.max_budget_pages) return RQ_ERR_CAPACITY;
+    return attend_from(cache, cache->len, q, idx, n_idx, n_idx, scale, o, (cudaStream_t)stream);
+}
+
+int64_t rq_cache_len(const rq_cache *cache) { return cache ? cache->len : -1; }
+
+int rq_device_status(rq_cache *cache, int32_t *status_out, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!status_out) return RQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    int32_t *dev = (int32_t *)((char *)cache->workspace + workspace_layout(cache->cfg).status);
+    if (cudaMemcpyAsync(status_out, dev, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    if (cudaMemsetAsync(dev, 0, sizeof(int32_t), s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return RQ_ERR_CUDA;
+    return RQ_OK;
+}
+
+const char *rq_status_string(int status)
+{
+    switch (status) {
+    case RQ_OK: return "ok";
+    case RQ_ERR_INVALID_ARG: return "invalid argument";
+    case RQ_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case RQ_ERR_CAPACITY: return "capacity exceeded";
+    case RQ_ERR_CUDA: return "CUDA error";
+    case RQ_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+    }
+}
+
+int rq_version(void) { return RQ_VERSION_MAJOR * 1000 + RQ_VERSION_MINOR; }
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Internal declarations shared by the library's translation units (host side).
+// Not part of the public ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rq.h"
+
+namespace rq {
+
+// ---- geometry of the prefill scan (must agree between sizing and launch) ----
+constexpr int kScanThreads = 256;  // threads per CTA
+
+// tokens a scan thread keeps in registers; chosen so that a chunk
+// (threads / channel-groups * tokens) is a whole number of 64-token pages too
+__host__ __device__ constexpr int scan_ts(int head_dim, int elem_bytes)
+{
+    return (kScanThreads / (head_dim / (16 / elem_bytes))) * 4 >= 64 ? 4 : 8;
+}
+
+// tokens covered by one scan CTA for a (head_dim, dtype) pair
+inline int scan_chunk_tokens(int head_dim, int dtype)
+{
+    int eb = dtype == RQ_BF16 ? 2 : 4;
+    int ncg = head_dim / (16 / eb);        // channel groups of one 16-byte vector
+    return (kScanThreads / ncg) * scan_ts(head_dim, eb);
+}
+
+// ---- decode-side geometry ----
+constexpr int kMaxSplits = 64;         // most split-K partials per (b,h)
+constexpr int kAttendWarps = 4;        // warps per flash-decode CTA
+constexpr int kTopkThreads = 1024;     // threads of the selection CTA
+constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
+constexpr int kTargetSMs = 148;        // B200
+
+// ---- workspace carving (byte offsets, every region 256-byte aligned) ----
+struct WorkspaceLayout {
+    size_t status;    // int32[64]
+    size_t scores;    // float [BH][page_capacity]
+    size_t sel;       // int32 [BH][max_budget]
+    size_t partial;   // float [BH][kMaxSplits][D + 2]
+    size_t agg;       // float [BH][scan chunks][3][D]
+    size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
+    size_t total;
+    int64_t scan_chunks_cap;
+};
+
+WorkspaceLayout workspace_layout(const rq_config &c);
+
+// ---- kernel launchers (defined in rq_scan.cu / rq_decode.cu) ----
+struct ScanArgs {
+    const void *k, *v, *g;
+    int64_t sb, st, sh;     // element strides of k, v, g
+    void *kv, *meta;
+    float *state, *agg;
+    int B, H, D, S, dtype, gate_dtype;
+    int64_t len0, T, page_cap, chunks_cap;
+};
+cudaError_t launch_scan(const ScanArgs &a, cudaStream_t s);
+
+struct DecodeArgs {
+    void *kv, *meta;
+    float *state;
+    int B, H, D, S, dtype, gate_dtype;
+    int64_t len;        // tokens in the cache the kernel should see
+    int64_t page_cap;
+    int n_sink, n_local;
+    int32_t *status;
+};
+cudaError_t launch_update(const DecodeArgs &a, const void *k_t, const void *v_t, const void *g_t,
+                          cudaStream_t s);
+cudaError_t launch_score(const DecodeArgs &a, const void *q, float *scores, cudaStream_t s);
+cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
+                        int idx_stride, cudaStream_t s);
+cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
+                          int idx_stride, float scale, float *partial, int nsplit, void *o,
+                          cudaStream_t s);
+int choose_splits(int BH, int n_idx, int sm_count);
+
+}  // namespace rq

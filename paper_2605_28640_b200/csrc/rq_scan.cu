@@ -1,0 +1,330 @@
+// Prefill: chunked parallel scan of the gated decay recurrence (Eq. 1) fused
+// with the paged cache write and the per-page min/max of the stored keys
+// (Appendix A.1, "Sparse inference settings").
+//
+// The recurrence x~_t = g_t x~_{t-1} + (1-g_t) x_t is a first-order linear
+// recurrence, so a run of tokens acts on the incoming state as the affine map
+// s -> A s + B with A = prod g and B = the run's own state from zero.  Maps
+// compose as (A2,B2)o(A1,B1) = (A2 A1, A2 B1 + B2), which is associative, so
+// time can be cut into pieces that are reduced independently.
+//
+// Work decomposition.  One CTA owns one (batch, head) pair and one chunk of
+// CT consecutive cache positions.  A thread owns CH channels (one 16-byte
+// vector of the storage type) and TS consecutive tokens whose k, v and g stay
+// in registers from the first to the last use.  Threads with the same
+// channels and consecutive token slices sit NCG lanes apart, so the carry
+// between the slices of a warp moves with warp shuffles; warps exchange their
+// totals through shared memory.
+//
+// Three launches: (0) every chunk's (A, Bk, Bv) -> workspace; (carry) a
+// sequential pass over the chunk maps per channel turns them into the state
+// entering each chunk; (1) every chunk re-reads its inputs and applies the
+// recurrence from the true incoming state, rounds to the storage type, writes
+// the pages and the page bounds, and the last token's owner leaves the fp32
+// state behind.
+#include "rq_device.cuh"
+#include "rq_internal.h"
+
+namespace rq {
+
+namespace {
+
+constexpr int NT = kScanThreads;
+
+template <typename T, typename G, int D, int S, int MODE>
+__global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
+{
+    constexpr int CH = VecOf<T>::N;
+    constexpr int NCG = D / CH;
+    constexpr int NSL = NT / NCG;
+    constexpr int TS = scan_ts(D, (int)sizeof(T));
+    constexpr int CT = NSL * TS;
+    constexpr int NW = NT / 32;
+    static_assert(CT % S == 0 && S % TS == 0, "chunk must hold whole pages of whole slices");
+    static_assert(NCG <= 32 && 32 % NCG == 0, "a warp must hold whole slices");
+
+    __shared__ float wtot[NW][3][D];
+    __shared__ float mm[MODE == 1 ? NSL : 1][2][D];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cg = tid % NCG, sl = tid / NCG;
+    const int bh = blockIdx.y, b = bh / a.H, h = bh % a.H;
+    const int64_t chunk = chunk0 + blockIdx.x;
+    const int64_t pos0 = chunk * CT + (int64_t)sl * TS;
+    const int64_t end = a.len0 + a.T;
+
+    const T *kp = static_cast<const T *>(a.k);
+    const T *vp = static_cast<const T *>(a.v);
+    const G *gp = static_cast<const G *>(a.g);
+
+    // ---- load this thread's TS tokens (identity map for positions outside the new range)
+    uint4 rk[TS], rv[TS];
+    float g[TS][CH];
+#pragma unroll
+    for (int i = 0; i < TS; ++i) {
+        const int64_t pos = pos0 + i;
+        if (pos >= a.len0 && pos < end) {
+            const int64_t src = (int64_t)b * a.sb + (pos - a.len0) * a.st + (int64_t)h * a.sh + cg * CH;
+            rk[i] = ldg16(kp + src);
+            rv[i] = ldg16(vp + src);
+            load_n<G, CH>(gp + src, g[i]);
+        } else {
+            rk[i] = make_uint4(0, 0, 0, 0);
+            rv[i] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) g[i][c] = 1.0f;
+        }
+    }
+
+    // ---- the slice's own map (A, Bk, Bv) from a zero state
+    float A[CH], Bk[CH], Bv[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) { A[c] = 1.0f; Bk[c] = 0.0f; Bv[c] = 0.0f; }
+#pragma unroll
+    for (int i = 0; i < TS; ++i) {
+        float kf[CH], vf[CH];
+        unpack16<T>(rk[i], kf);
+        unpack16<T>(rv[i], vf);
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const float om = 1.0f - g[i][c];
+            Bk[c] = fmaf(g[i][c], Bk[c], om * kf[c]);
+            Bv[c] = fmaf(g[i][c], Bv[c], om * vf[c]);
+            A[c] *= g[i][c];
+        }
+    }
+
+    // ---- inclusive scan over the slices of this warp: carry by warp shuffle
+#pragma unroll
+    for (int off = NCG; off < 32; off <<= 1) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const float pa = __shfl_up_sync(0xffffffffu, A[c], off);
+            const float pk = __shfl_up_sync(0xffffffffu, Bk[c], off);
+            const float pv = __shfl_up_sync(0xffffffffu, Bv[c], off);
+            if (lane >= off) {
+                Bk[c] = fmaf(A[c], pk, Bk[c]);
+                Bv[c] = fmaf(A[c], pv, Bv[c]);
+                A[c] *= pa;
+            }
+        }
+    }
+    if (lane >= 32 - NCG) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            wtot[warp][0][cg * CH + c] = A[c];
+            wtot[warp][1][cg * CH + c] = Bk[c];
+            wtot[warp][2][cg * CH + c] = Bv[c];
+        }
+    }
+    __syncthreads();
+
+    // ---- map of everything in the chunk before this warp
+    float Ap[CH], Pk[CH], Pv[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) { Ap[c] = 1.0f; Pk[c] = 0.0f; Pv[c] = 0.0f; }
+    for (int w = 0; w < warp; ++w) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            const float wa = wtot[w][0][cg * CH + c];
+            Pk[c] = fmaf(wa, Pk[c], wtot[w][1][cg * CH + c]);
+            Pv[c] = fmaf(wa, Pv[c], wtot[w][2][cg * CH + c]);
+            Ap[c] *= wa;
+        }
+    }
+
+    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + blockIdx.x) * 3 * D;
+
+    if constexpr (MODE == 0) {
+        // the chunk's map = (last warp's total) o (everything before the last warp)
+        if (warp == NW - 1 && lane >= 32 - NCG) {
+            float oa[CH], ok[CH], ov[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                ok[c] = fmaf(A[c], Pk[c], Bk[c]);
+                ov[c] = fmaf(A[c], Pv[c], Bv[c]);
+                oa[c] = A[c] * Ap[c];
+            }
+#pragma unroll
+            for (int c = 0; c < CH; c += 4) {
+                *reinterpret_cast<float4 *>(agg + 0 * D + cg * CH + c) = make_float4(oa[c], oa[c + 1], oa[c + 2], oa[c + 3]);
+                *reinterpret_cast<float4 *>(agg + 1 * D + cg * CH + c) = make_float4(ok[c], ok[c + 1], ok[c + 2], ok[c + 3]);
+                *reinterpret_cast<float4 *>(agg + 2 * D + cg * CH + c) = make_float4(ov[c], ov[c + 1], ov[c + 2], ov[c + 3]);
+            }
+        }
+        return;
+    } else {
+        // ---- exclusive map inside the warp = inclusive map of the previous slice
+        float sk[CH], sv[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            float ea = __shfl_up_sync(0xffffffffu, A[c], NCG % 32);
+            float ek = __shfl_up_sync(0xffffffffu, Bk[c], NCG % 32);
+            float ev = __shfl_up_sync(0xffffffffu, Bv[c], NCG % 32);
+            if (NCG == 32 || lane < NCG) { ea = 1.0f; ek = 0.0f; ev = 0.0f; }
+            // state entering the chunk (left by the carry pass in slots 1 and 2)
+            const float ck = agg[1 * D + cg * CH + c];
+            const float cv = agg[2 * D + cg * CH + c];
+            // entering this warp, then entering this slice
+            const float wk = fmaf(Ap[c], ck, Pk[c]);
+            const float wv = fmaf(Ap[c], cv, Pv[c]);
+            sk[c] = fmaf(ea, wk, ek);
+            sv[c] = fmaf(ea, wv, ev);
+        }
+
+        // ---- apply the recurrence token by token, round, store, track bounds
+        T *kv = static_cast<T *>(a.kv);
+        float mn[CH], mx[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) { mn[c] = INFINITY; mx[c] = -INFINITY; }
+        const int64_t tail_end = (end + S - 1) / S * S;   // end of the last touched page
+#pragma unroll
+        for (int i = 0; i < TS; ++i) {
+            const int64_t pos = pos0 + i;
+            float kf[CH], vf[CH];
+            unpack16<T>(rk[i], kf);
+            unpack16<T>(rv[i], vf);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const float om = 1.0f - g[i][c];
+                sk[c] = fmaf(g[i][c], sk[c], om * kf[c]);
+                sv[c] = fmaf(g[i][c], sv[c], om * vf[c]);
+            }
+            const bool valid = pos >= a.len0 && pos < end;
+            const bool fill = pos >= end && pos < tail_end;   // unused slots of the last page
+            if (valid || fill) {
+                const int64_t page = pos / S;
+                const int slot = (int)(pos % S);
+                T *dst = kv + ((((int64_t)bh * a.page_cap + page) * 2) * S + slot) * D + cg * CH;
+                uint4 wk, wv;
+                if (valid) {
+                    wk = pack16<T>(sk);
+                    wv = pack16<T>(sv);
+                    float rk_[CH];
+                    unpack16<T>(wk, rk_);
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        mn[c] = fminf(mn[c], rk_[c]);
+                        mx[c] = fmaxf(mx[c], rk_[c]);
+                    }
+                } else {
+                    wk = make_uint4(0, 0, 0, 0);
+                    wv = wk;
+                }
+                *reinterpret_cast<uint4 *>(dst) = wk;
+                *reinterpret_cast<uint4 *>(dst + (int64_t)S * D) = wv;
+            }
+        }
+        // the owner of the last new token leaves the fp32 state behind
+        if (end - 1 >= pos0 && end - 1 < pos0 + TS) {
+            float *st = a.state + (int64_t)bh * 2 * D;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                st[cg * CH + c] = sk[c];
+                st[D + cg * CH + c] = sv[c];
+            }
+        }
+
+        // ---- page bounds: reduce the slices of each page through shared memory
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            mm[sl][0][cg * CH + c] = mn[c];
+            mm[sl][1][cg * CH + c] = mx[c];
+        }
+        __syncthreads();
+        constexpr int SPP = S / TS;      // slices per page
+        constexpr int PPC = CT / S;      // pages per chunk
+        T *meta = static_cast<T *>(a.meta);
+        for (int idx = tid; idx < PPC * D; idx += NT) {
+            const int pg = idx / D, d = idx % D;
+            const int64_t page = chunk * PPC + pg;
+            const int64_t pstart = page * S;
+            if (pstart >= end || pstart + S <= a.len0) continue;   // no new token in this page
+            float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+            for (int s2 = 0; s2 < SPP; ++s2) {
+                lo = fminf(lo, mm[pg * SPP + s2][0][d]);
+                hi = fmaxf(hi, mm[pg * SPP + s2][1][d]);
+            }
+            T *m = meta + (((int64_t)bh * a.page_cap + page) * 2) * D + d;
+            if (pstart < a.len0) {                                  // page already held tokens
+                lo = fminf(lo, load1<T>(m));
+                hi = fmaxf(hi, load1<T>(m + D));
+            }
+            store1<T>(m, lo);
+            store1<T>(m + D, hi);
+        }
+    }
+}
+
+// Sequential composition of the chunk maps, one thread per (b, h, channel):
+// slot 1/2 of every chunk's record is overwritten with the state entering it.
+template <int BATCH>
+__global__ void scan_carry_kernel(float *agg, const float *state, int D, int64_t nchunks,
+                                  int64_t chunks_cap)
+{
+    const int bh = blockIdx.x, d = threadIdx.x;
+    if (d >= D) return;
+    float sk = state[(int64_t)bh * 2 * D + d];
+    float sv = state[(int64_t)bh * 2 * D + D + d];
+    float *base = agg + (int64_t)bh * chunks_cap * 3 * D + d;
+    for (int64_t c0 = 0; c0 < nchunks; c0 += BATCH) {
+        float A[BATCH], Bk[BATCH], Bv[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+            if (c0 + j < nchunks) {
+                const float *r = base + (c0 + j) * 3 * D;
+                A[j] = r[0]; Bk[j] = r[D]; Bv[j] = r[2 * D];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < BATCH; ++j) {
+            if (c0 + j < nchunks) {
+                float *r = base + (c0 + j) * 3 * D;
+                r[D] = sk; r[2 * D] = sv;
+                sk = fmaf(A[j], sk, Bk[j]);
+                sv = fmaf(A[j], sv, Bv[j]);
+            }
+        }
+    }
+}
+
+template <typename T, typename G, int D, int S>
+cudaError_t run(const ScanArgs &a, cudaStream_t s)
+{
+    constexpr int CH = VecOf<T>::N;
+    constexpr int CT = (NT / (D / CH)) * scan_ts(D, (int)sizeof(T));
+    const int64_t end = a.len0 + a.T;
+    const int64_t c0 = a.len0 / CT;
+    const int64_t c1 = (end + CT - 1) / CT;
+    const int64_t nchunks = c1 - c0;
+    if (nchunks <= 0) return cudaSuccess;
+    if (nchunks > a.chunks_cap) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)nchunks, (unsigned)(a.B * a.H));
+    scan_kernel<T, G, D, S, 0><<<grid, NT, 0, s>>>(a, c0);
+    scan_carry_kernel<16><<<a.B * a.H, D, 0, s>>>(a.agg, a.state, D, nchunks, a.chunks_cap);
+    scan_kernel<T, G, D, S, 1><<<grid, NT, 0, s>>>(a, c0);
+    return cudaGetLastError();
+}
+
+template <typename T, typename G>
+cudaError_t dispatch_shape(const ScanArgs &a, cudaStream_t s)
+{
+    if (a.D == 128 && a.S == 16) return run<T, G, 128, 16>(a, s);
+    if (a.D == 128 && a.S == 64) return run<T, G, 128, 64>(a, s);
+    if (a.D == 64 && a.S == 16) return run<T, G, 64, 16>(a, s);
+    if (a.D == 64 && a.S == 64) return run<T, G, 64, 64>(a, s);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+cudaError_t launch_scan(const ScanArgs &a, cudaStream_t s)
+{
+    if (a.dtype == RQ_BF16) {
+        return a.gate_dtype == RQ_BF16 ? dispatch_shape<bf16, bf16>(a, s) : dispatch_shape<bf16, float>(a, s);
+    }
+    return a.gate_dtype == RQ_BF16 ? dispatch_shape<float, bf16>(a, s) : dispatch_shape<float, float>(a, s);
+}
+
+}  // namespace rq

@@ -1,0 +1,139 @@
+"""Staged comparison of the CUDA path with the fp64 oracle for one (batch, head).
+
+Levels (tolerances are the ones the benchmark definition states):
+  1. state     : fp32 running state vs the oracle's fp64 state, 1e-4 relative
+                 (with an absolute floor of 1e-5 of the state's rms for channels
+                 that are near zero by cancellation)
+  2. cache     : stored k~, v~ equal to the oracle's stored values or one
+                 storage-ulp apart, at least 99.9 % exactly equal;
+                 page bounds bit-exact against min/max of the device's own cache
+  3. selection : the oracle's scoring + top-k run on the DEVICE's bounds and q
+                 bits must give the same pages, except where the oracle flags a
+                 near-tie (1e-5 relative) at the cut — those are counted
+  4. attention : the oracle's attention over the device's pages and stored
+                 cache vs the device output: 2e-2 max-abs / 5e-3 mean-abs for
+                 bf16, 1e-4 / 1e-5 for fp32; and the oracle's own end-to-end
+                 chain wherever its page set equals the device's
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+
+ODT = {torch.float32: oracle.F32, torch.bfloat16: oracle.BF16}
+ATT_TOL = {torch.bfloat16: (2e-2, 5e-3), torch.float32: (1e-4, 1e-5)}
+
+
+def f64(t):
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def storage_ulp(x, dtype):
+    """Spacing of the storage format at |x| (normal range)."""
+    ax = np.maximum(np.abs(x), 1e-30)
+    e = np.floor(np.log2(ax))
+    return 2.0 ** (e - (7 if dtype == torch.bfloat16 else 23))
+
+
+def assert_state_close(gpu, ref, what):
+    rms = float(np.sqrt(np.mean(ref ** 2))) or 1.0
+    err = np.abs(gpu - ref)
+    tol = 1e-4 * np.abs(ref) + 1e-5 * rms
+    assert (err <= tol).all(), f"{what}: max excess {(err - tol).max():.3e} (rms {rms:.3e})"
+
+
+def oracle_head(w, k, v, g, b, h, capacity, n_sink=1, n_local=1):
+    """Oracle cache of head (b, h) prefilled with the same input bits."""
+    hd = oracle.Head(w.D, w.S, capacity, ODT[w.dtype], n_sink, n_local)
+    if k is not None and k.shape[1] > 0:
+        hd.append(f64(k[b, :, h, :]), f64(v[b, :, h, :]), f64(g[b, :, h, :]))
+    return hd
+
+
+def device_head_arrays(cache, b, h):
+    """The device's stored cache, bounds and state for head (b, h) as float64."""
+    T = len(cache)
+    S, D = cache.cfg.page_size, cache.cfg.head_dim
+    P = (T + S - 1) // S
+    kv = cache.kv_view()[b, h, :P]                     # [P, 2, S, D]
+    k = f64(kv[:, 0]).reshape(P * S, D)[:T]
+    v = f64(kv[:, 1]).reshape(P * S, D)[:T]
+    meta = f64(cache.meta_view()[b, h, :P])            # [P, 2, D]
+    st = f64(cache.state_view()[b, h])
+    return {"k": k, "v": v, "min": meta[:, 0], "max": meta[:, 1], "state_k": st[0], "state_v": st[1],
+            "k_tail": f64(kv[:, 0]).reshape(P * S, D)[T:], "v_tail": f64(kv[:, 1]).reshape(P * S, D)[T:]}
+
+
+def check_cache_level(cache, hd, b, h, dtype):
+    """Levels 1 and 2.  Returns the device arrays for later levels."""
+    dev = device_head_arrays(cache, b, h)
+    ex = hd.export()
+    assert dev["k"].shape == ex["k"].shape
+    assert_state_close(dev["state_k"], ex["state_k"], f"state_k[{b},{h}]")
+    assert_state_close(dev["state_v"], ex["state_v"], f"state_v[{b},{h}]")
+    for name in ("k", "v"):
+        a, r = dev[name], ex[name]
+        ne = a != r
+        frac = ne.mean() if a.size else 0.0
+        assert frac <= 1e-3, f"{name}[{b},{h}]: {frac:.2e} of stored values differ"
+        if ne.any():
+            gap = np.abs(a - r)[ne]
+            ulp = storage_ulp(np.maximum(np.abs(a), np.abs(r)), dtype)[ne]
+            assert (gap <= ulp * 1.0000001).all(), f"{name}[{b},{h}]: a stored value is more than 1 ulp off"
+    # unused slots of the last page are defined (zero)
+    assert not dev["k_tail"].any() and not dev["v_tail"].any()
+    mn, mx = oracle.page_bounds(dev["k"], cache.cfg.page_size)
+    assert np.array_equal(mn, dev["min"]), f"min bounds [{b},{h}] differ from min of the device cache"
+    assert np.array_equal(mx, dev["max"]), f"max bounds [{b},{h}] differ from max of the device cache"
+    return dev
+
+
+def check_query_level(dev, hd, cache, b, h, q, K, scale, o, idx, scores, dtype, stats):
+    """Levels 3 and 4 for one head.  idx: device [B,H,K] int32; scores: device [B,H,P] or None."""
+    S = cache.cfg.page_size
+    n_sink, n_local = cache.cfg.n_sink_pages, cache.cfg.n_local_pages
+    q64 = f64(q[b, h])
+    U = oracle.page_scores(q64, dev["min"], dev["max"])
+    if scores is not None:
+        gU = f64(scores[b, h])
+        assert gU.shape == U.shape
+        denom = np.maximum(np.abs(U), 1e-3 * np.sqrt(np.mean(U ** 2)) + 1e-30)
+        assert (np.abs(gU - U) / denom).max() <= 1e-5, f"scores[{b},{h}] off by {(np.abs(gU - U) / denom).max():.2e}"
+    want, near = oracle.select_pages(U, K, n_sink, n_local)
+    got = idx[b, h].cpu().numpy().astype(np.int64)
+    n = len(want)
+    assert (got[n:] == -1).all(), "unused tail of the index list must be -1"
+    got = got[:n]
+    assert (np.diff(got) > 0).all(), "page list must be strictly ascending"
+    stats["heads"] = stats.get("heads", 0) + 1
+    if not np.array_equal(got, want):
+        assert near, f"pages [{b},{h}] differ from the oracle's with no near-tie at the cut"
+        # whatever was swapped must sit within 1e-5 relative of the cut
+        sel_o = set(want.tolist())
+        sel_g = set(got.tolist())
+        forced = set(range(min(n_sink, len(U)))) | set(range(max(len(U) - n_local, 0), len(U)))
+        cut = min(U[p] for p in sel_o - forced)
+        for p in sel_o ^ sel_g:
+            assert abs(U[p] - cut) <= 2e-5 * abs(cut), f"page {p} swapped far from the cut"
+        stats["near_tie_mismatch"] = stats.get("near_tie_mismatch", 0) + 1
+    if near:
+        stats["near_tie"] = stats.get("near_tie", 0) + 1
+    # level 4: attention over the device's own pages and stored cache
+    y = oracle.sparse_attention(q64, scale, dev["k"], dev["v"], got, S)
+    go = f64(o[b, h])
+    mx_tol, mean_tol = ATT_TOL[dtype]
+    err = np.abs(go - y)
+    assert err.max() <= mx_tol and err.mean() <= mean_tol, \
+        f"attention[{b},{h}]: max {err.max():.3e} mean {err.mean():.3e}"
+    stats["att_max"] = max(stats.get("att_max", 0.0), float(err.max()))
+    # end to end: the oracle's own chain from the raw inputs
+    e2e = hd.query(q64, K, scale)
+    if np.array_equal(e2e["idx"], got):
+        err2 = np.abs(go - e2e["y"])
+        assert err2.max() <= mx_tol and err2.mean() <= mean_tol, \
+            f"end-to-end attention[{b},{h}]: max {err2.max():.3e} mean {err2.mean():.3e}"
+        stats["e2e_same_pages"] = stats.get("e2e_same_pages", 0) + 1
+    stats["e2e_overlap"] = stats.get("e2e_overlap", 0.0) + len(set(e2e["idx"].tolist()) & set(got.tolist())) / max(n, 1)
+    return stats
