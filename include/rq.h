@@ -162,6 +162,22 @@ RQ_API int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *
                         int32_t budget_pages, float scale, void *o_host,
                         int32_t *sel_idx_out_host, void *stream);
 
+/* rq_decode_step with per-kernel device timing, for benchmarks: CUDA events are
+ * recorded on `stream` between the kernels of the step, the stream is
+ * SYNCHRONISED, and the elapsed microseconds of every kernel go to
+ * kernel_us[0 .. RQ_PROFILE_SLOTS-1] (host memory), in launch order;
+ * rq_profile_slot_name(i) names slot i.  The computation and its results are
+ * those of rq_decode_step [Eq. 1, Eq. 3, Eq. 4].
+ * Errors: as rq_decode_step; INVALID_ARG for NULL kernel_us. */
+#define RQ_PROFILE_SLOTS 5
+RQ_API int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t,
+                                   const void *v_t, const void *g_t, int32_t budget_pages,
+                                   float scale, void *o, int32_t *sel_idx_out,
+                                   float *kernel_us, void *stream);
+
+/* Name of the kernel timed in slot i ("" if out of range). */
+RQ_API const char *rq_profile_slot_name(int slot);
+
 /* Stage export [Eq. 3 only]: score and select against the current cache without
  * changing it.  scores_out: NULL or fp32 [B][H][P] with P = ceil(len / S);
  * idx_out: int32 [B][H][budget_pages] as in rq_decode_step (must not be NULL).

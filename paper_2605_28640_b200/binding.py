@@ -42,6 +42,9 @@ SIGNATURES = {
     "rq_build_cache": (C.c_int, [_cachep, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _vp]),
     "rq_decode_step": (C.c_int, [_cachep, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp]),
     "rq_decode_step_host": (C.c_int, [_cachep, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp, _vp]),
+    "rq_decode_step_profiled": (C.c_int, [_cachep, _vp, _vp, _vp, _vp, _i32, _f, _vp, _vp,
+                                          C.POINTER(C.c_float), _vp]),
+    "rq_profile_slot_name": (C.c_char_p, [C.c_int]),
     "rq_select_pages": (C.c_int, [_cachep, _vp, _i32, _vp, _vp, _vp]),
     "rq_attend_pages": (C.c_int, [_cachep, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
@@ -127,6 +130,19 @@ def rq_decode_step_host(cache: rq_cache, q, k_t, v_t, g_t, budget_pages, scale, 
     _check(lib().rq_decode_step_host(C.byref(cache), _ptr(q), _ptr(k_t), _ptr(v_t), _ptr(g_t), budget_pages,
                                      scale, _ptr(o), _ptr(sel_idx_out), _stream(stream)),
            "rq_decode_step_host")
+
+
+RQ_PROFILE_SLOTS = 5
+
+
+def rq_decode_step_profiled(cache: rq_cache, q, k_t, v_t, g_t, budget_pages, scale, o, sel_idx_out=None,
+                            stream=None):
+    """rq_decode_step with per-kernel timing; synchronises; returns {kernel name: microseconds}."""
+    us = (C.c_float * RQ_PROFILE_SLOTS)()
+    _check(lib().rq_decode_step_profiled(C.byref(cache), _ptr(q), _ptr(k_t), _ptr(v_t), _ptr(g_t),
+                                         budget_pages, scale, _ptr(o), _ptr(sel_idx_out), us,
+                                         _stream(stream)), "rq_decode_step_profiled")
+    return {lib().rq_profile_slot_name(i).decode(): us[i] for i in range(RQ_PROFILE_SLOTS)}
 
 
 def rq_select_pages(cache: rq_cache, q, budget_pages, scores_out, idx_out, stream=None):

@@ -80,27 +80,65 @@ static int check_cache(const rq_cache *c)
     return check_config(&c->cfg);
 }
 
+// Optional per-kernel timing: when `ev` is not NULL an event is recorded after
+// every kernel of a decode step (ev[0] before the first one).
+static void mark(cudaEvent_t *ev, int i, cudaStream_t s)
+{
+    if (ev) cudaEventRecord(ev[i], s);
+}
+
 // score + select into `idx` (device, stride idx_stride), for a cache of length len
 static int select_into(const rq_cache *c, int64_t len, const void *q, int budget, float *scores,
-                       int32_t *idx, int idx_stride, cudaStream_t s)
+                       int32_t *idx, int idx_stride, cudaStream_t s, cudaEvent_t *ev = nullptr)
 {
     DecodeArgs a = decode_args(c, len);
     if (launch_score(a, q, scores, s) != cudaSuccess) return RQ_ERR_CUDA;
+    mark(ev, 2, s);
     if (launch_topk(a, scores, budget, idx, idx_stride, s) != cudaSuccess) return RQ_ERR_CUDA;
+    mark(ev, 3, s);
     return RQ_OK;
 }
 
 static int attend_from(const rq_cache *c, int64_t len, const void *q, const int32_t *idx, int n_idx,
-                       int idx_stride, float scale, void *o, cudaStream_t s)
+                       int idx_stride, float scale, void *o, cudaStream_t s, cudaEvent_t *ev = nullptr)
 {
     DecodeArgs a = decode_args(c, len);
     const WorkspaceLayout w = workspace_layout(c->cfg);
     float *partial = (float *)((char *)c->workspace + w.partial);
     if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
     const int nsplit = choose_splits(a.B * a.H, n_idx, sm_count());
-    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, o, s) != cudaSuccess)
+    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, s) != cudaSuccess)
         return RQ_ERR_CUDA;
+    mark(ev, 4, s);
+    if (launch_combine(a, partial, nsplit, o, s) != cudaSuccess) return RQ_ERR_CUDA;
+    mark(ev, 5, s);
     return RQ_OK;
+}
+
+static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, const void *v_t,
+                            const void *g_t, int32_t budget_pages, float scale, void *o,
+                            int32_t *sel_idx_out, cudaStream_t s, cudaEvent_t *ev)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q || !k_t || !v_t || !g_t || !o || budget_pages < 1) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    if (budget_pages > c.max_budget_pages) return RQ_ERR_CAPACITY;
+    if (cache->len >= c.capacity_tokens) return RQ_ERR_CAPACITY;
+    const WorkspaceLayout w = workspace_layout(c);
+    float *scores = (float *)((char *)cache->workspace + w.scores);
+    int32_t *sel = sel_idx_out ? sel_idx_out : (int32_t *)((char *)cache->workspace + w.sel);
+
+    DecodeArgs a = decode_args(cache, cache->len);
+    mark(ev, 0, s);
+    if (launch_update(a, k_t, v_t, g_t, s) != cudaSuccess) return RQ_ERR_CUDA;
+    mark(ev, 1, s);
+    cache->len += 1;
+    const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
+    int st = select_into(cache, cache->len, q, budget_pages, scores, sel, budget_pages, s, ev);
+    if (st != RQ_OK) return st;
+    const int n_idx = (int)(budget_pages < P ? budget_pages : P);
+    return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s, ev);
 }
 
 }  // namespace rq
@@ -188,25 +226,39 @@ int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
 int rq_decode_step(rq_cache *cache, const void *q, const void *k_t, const void *v_t, const void *g_t,
                    int32_t budget_pages, float scale, void *o, int32_t *sel_idx_out, void *stream)
 {
-    const int rc = check_cache(cache);
-    if (rc != RQ_OK) return rc;
-    if (!q || !k_t || !v_t || !g_t || !o || budget_pages < 1) return RQ_ERR_INVALID_ARG;
-    const rq_config &c = cache->cfg;
-    if (budget_pages > c.max_budget_pages) return RQ_ERR_CAPACITY;
-    if (cache->len >= c.capacity_tokens) return RQ_ERR_CAPACITY;
-    cudaStream_t s = (cudaStream_t)stream;
-    const WorkspaceLayout w = workspace_layout(c);
-    float *scores = (float *)((char *)cache->workspace + w.scores);
-    int32_t *sel = sel_idx_out ? sel_idx_out : (int32_t *)((char *)cache->workspace + w.sel);
+    return decode_step_impl(cache, q, k_t, v_t, g_t, budget_pages, scale, o, sel_idx_out,
+                            (cudaStream_t)stream, nullptr);
+}
 
-    DecodeArgs a = decode_args(cache, cache->len);
-    if (launch_update(a, k_t, v_t, g_t, s) != cudaSuccess) return RQ_ERR_CUDA;
-    cache->len += 1;
-    const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
-    int st = select_into(cache, cache->len, q, budget_pages, scores, sel, budget_pages, s);
-    if (st != RQ_OK) return st;
-    const int n_idx = (int)(budget_pages < P ? budget_pages : P);
-    return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s);
+int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t, const void *v_t,
+                            const void *g_t, int32_t budget_pages, float scale, void *o,
+                            int32_t *sel_idx_out, float *kernel_us, void *stream)
+{
+    if (!kernel_us) return RQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaEvent_t ev[RQ_PROFILE_SLOTS + 1];
+    int made = 0;
+    for (; made <= RQ_PROFILE_SLOTS; ++made)
+        if (cudaEventCreate(&ev[made]) != cudaSuccess) break;
+    int st = made == RQ_PROFILE_SLOTS + 1 ? RQ_OK : RQ_ERR_CUDA;
+    if (st == RQ_OK)
+        st = decode_step_impl(cache, q, k_t, v_t, g_t, budget_pages, scale, o, sel_idx_out, s, ev);
+    if (st == RQ_OK && cudaStreamSynchronize(s) != cudaSuccess) st = RQ_ERR_CUDA;
+    if (st == RQ_OK) {
+        for (int i = 0; i < RQ_PROFILE_SLOTS; ++i) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, ev[i], ev[i + 1]) != cudaSuccess) st = RQ_ERR_CUDA;
+            kernel_us[i] = ms * 1000.0f;
+        }
+    }
+    for (int i = 0; i < made; ++i) cudaEventDestroy(ev[i]);
+    return st;
+}
+
+const char *rq_profile_slot_name(int slot)
+{
+    static const char *names[RQ_PROFILE_SLOTS] = {"update", "score", "topk", "attend", "combine"};
+    return slot >= 0 && slot < RQ_PROFILE_SLOTS ? names[slot] : "";
 }
 
 int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_host,

@@ -465,18 +465,25 @@ int choose_splits(int BH, int n_idx, int sm_count)
 }
 
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
-                          int idx_stride, float scale, float *partial, int nsplit, void *o,
-                          cudaStream_t s)
+                          int idx_stride, float scale, float *partial, int nsplit, cudaStream_t s)
 {
     const int BH = a.B * a.H;
     const float scale_log2 = scale * 1.4426950408889634f;
     dim3 grid((unsigned)nsplit, (unsigned)BH);
 #define CALL_ATT(T, D, S)                                                                        \
     attend_kernel<T, D, S><<<grid, kAttendWarps * 32, 0, s>>>(a, (const T *)q, idx, n_idx,       \
-                                                              idx_stride, scale_log2, partial, nsplit); \
-    combine_kernel<T, D><<<BH, D, 0, s>>>(partial, nsplit, (T *)o)
+                                                              idx_stride, scale_log2, partial, nsplit)
     RQ_DISPATCH_TDS(a, CALL_ATT);
 #undef CALL_ATT
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const DecodeArgs &a, const float *partial, int nsplit, void *o, cudaStream_t s)
+{
+    const int BH = a.B * a.H;
+#define CALL_CMB(T, D, S) combine_kernel<T, D><<<BH, D, 0, s>>>(partial, nsplit, (T *)o)
+    RQ_DISPATCH_TDS(a, CALL_CMB);
+#undef CALL_CMB
     return cudaGetLastError();
 }
 

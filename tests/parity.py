@@ -4,8 +4,11 @@ Levels (tolerances are the ones the benchmark definition states):
   1. state     : fp32 running state vs the oracle's fp64 state, 1e-4 relative
                  (with an absolute floor of 1e-5 of the state's rms for channels
                  that are near zero by cancellation)
-  2. cache     : stored k~, v~ equal to the oracle's stored values or one
-                 storage-ulp apart, at least 99.9 % exactly equal;
+  2. cache     : bf16 storage: stored k~, v~ equal to the oracle's stored values
+                 or one storage-ulp apart, at least 99.9 % exactly equal (the
+                 fp32 state error is far below a bf16 ulp, so only values next
+                 to a rounding boundary can differ); fp32 storage: the stored
+                 value IS the fp32 state, so the state tolerance applies;
                  page bounds bit-exact against min/max of the device's own cache
   3. selection : the oracle's scoring + top-k run on the DEVICE's bounds and q
                  bits must give the same pages, except where the oracle flags a
@@ -75,13 +78,24 @@ def check_cache_level(cache, hd, b, h, dtype):
     assert_state_close(dev["state_v"], ex["state_v"], f"state_v[{b},{h}]")
     for name in ("k", "v"):
         a, r = dev[name], ex[name]
+        if dtype == torch.float32:
+            # fp32 storage keeps the fp32 state itself: the state tolerance applies
+            if a.size:
+                assert_state_close(a, r, f"stored {name}[{b},{h}]")
+            continue
         ne = a != r
         frac = ne.mean() if a.size else 0.0
         assert frac <= 1e-3, f"{name}[{b},{h}]: {frac:.2e} of stored values differ"
         if ne.any():
+            # one rounding step apart, or (for values that are near zero by cancellation, where
+            # an ulp is far below the fp32 state's absolute error) within the state tolerance
             gap = np.abs(a - r)[ne]
             ulp = storage_ulp(np.maximum(np.abs(a), np.abs(r)), dtype)[ne]
-            assert (gap <= ulp * 1.0000001).all(), f"{name}[{b},{h}]: a stored value is more than 1 ulp off"
+            rms = float(np.sqrt(np.mean(r ** 2)))
+            slack = (1e-4 * np.abs(r) + 1e-5 * rms)[ne]
+            bad = gap > np.maximum(ulp * 1.0000001, slack)
+            assert not bad.any(), (f"{name}[{b},{h}]: {bad.sum()} stored values are more than one "
+                                   f"rounding step off (worst gap {gap[bad].max():.3e})")
     # unused slots of the last page are defined (zero)
     assert not dev["k_tail"].any() and not dev["v_tail"].any()
     mn, mx = oracle.page_bounds(dev["k"], cache.cfg.page_size)

@@ -23,7 +23,7 @@ def run_case(w, T_prefill, steps=1, heads=None, n_sink=1, n_local=1, scale=0.0, 
     steps, checking every level after the prefill and after every step for the sampled heads."""
     stats = {} if stats is None else stats
     cap = T_prefill + steps + 3
-    maxK = max(w.pages(cap), 1)
+    maxK = max(w.pages(cap), budget or 1)
     cache = rq.Cache(w.B, w.H, w.D, w.S, cap, w.dtype, w.gdtype, n_sink, n_local, maxK)
     q0 = wl.make_query(w, DEV, 0)
     k, v, g = wl.make_prefill(w, DEV, T_prefill, q_for_needles=q0 if w.needles else None)
