@@ -1,0 +1,410 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse decode step (and, beside it, the prefill cache build).
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--workload NAME]
+
+One "step" is one rq_decode_step (state update + append, page scoring, top-k,
+sparse attention, combine) for every sequence of the batch at the workload's
+context length and budget.  The default workload is the one the headline
+metric is quoted on: batch 1, 32 heads x 128 dims, 128K context, page 16,
+budget 1/16 (512 pages per head), bf16 I/O with fp32 state and accumulation.
+
+Timing: CUDA events on the launching stream around exactly K steps after W
+warm-up steps, barrier + synchronize on both sides, max over ranks.  Several
+independent caches are rotated so that every step streams data that is not in
+L2 (their total is many times the L2 size), and every step uses a fresh query
+and token.  Prints ONE JSON line.
+
+With --gpus N > 1 the path does not shard (heads are independent and there is
+no exchange step): every rank runs an independent replica of the workload and
+`value` is the per-step time divided by N.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "sparse decode us/step at 128K ctx, 1/16 budget"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu
+# captures (profiles/): kernel -> bytes for the default workload, or None.
+NCU_TRAFFIC = {"score": None, "attend": None}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def pick_workload(name):
+    from paper_2605_28640_b200 import workloads as wl
+    import dataclasses
+    table = {"metric": wl.METRIC, "cfg1": wl.CONFIGS[1], "cfg2": wl.CONFIGS[2], "cfg4": wl.CONFIGS[4],
+             "cfg4-1/8": dataclasses.replace(wl.CONFIGS[4], budget_den=8),
+             "cfg4-1/4": dataclasses.replace(wl.CONFIGS[4], budget_den=4),
+             "half": dataclasses.replace(wl.METRIC, name="decode-64k-b1", T=65536),
+             "small": dataclasses.replace(wl.CONFIGS[1], name="small-16k")}
+    return table[name]
+
+
+def step_bytes(w, T):
+    """Algorithmic bytes one decode step must touch: all page bounds + the selected K/V pages."""
+    es = 2 if str(w.dtype).endswith("bfloat16") else 4
+    P, K = w.pages(T), w.budget_pages(T)
+    meta = w.B * w.H * P * 2 * w.D * es
+    kvb = w.B * w.H * min(K, P) * w.S * w.D * es * 2
+    return meta, kvb
+
+
+# ------------------------------------------------------------------------- oracle arm
+class OracleSample:
+    """The fp64 oracle, as it stands, on `n_heads` heads of batch item 0 of the workload:
+    prefill (untimed), then decode steps (append one token, score, select, attend) timed
+    per call.  Heads run on a thread pool (the C code releases the GIL)."""
+
+    def __init__(self, w, k, v, g, q, kt, vt, gt, n_heads, threads, max_steps):
+        import concurrent.futures as cf
+        import oracle
+        import torch
+        odt = oracle.BF16 if w.dtype == torch.bfloat16 else oracle.F32
+        T0 = k.shape[1]
+        self.K = w.budget_pages(T0 + 1)
+        self.scale = w.D ** -0.5
+        self.threads = threads
+        self.pool = cf.ThreadPoolExecutor(threads)
+
+        def f64(t):
+            return t.detach().to(torch.float64).cpu().numpy()
+
+        self.items = []
+        for h in range(n_heads):
+            hd = oracle.Head(w.D, w.S, T0 + max_steps + 1, odt)
+            self.items.append((hd, f64(q[0, h]), f64(kt[0, h]), f64(vt[0, h]), f64(gt[0, h])))
+        pre = [(self.items[h][0], f64(k[0, :, h]), f64(v[0, :, h]), f64(g[0, :, h])) for h in range(n_heads)]
+        list(self.pool.map(lambda it: it[0].append(it[1], it[2], it[3]), pre))
+
+    def _one(self, item):
+        hd, q, a, b, c = item
+        hd.append(a, b, c)
+        hd.query(q, self.K, self.scale)
+
+    def step(self):
+        """One decode step of every sampled head; returns wall seconds."""
+        t0 = time.perf_counter()
+        list(self.pool.map(self._one, self.items))
+        return time.perf_counter() - t0
+
+
+def oracle_sample_for(w, dev, n_heads, threads, max_steps, inputs=None):
+    import dataclasses
+    from paper_2605_28640_b200 import workloads as wl
+    ws = dataclasses.replace(w, B=1, H=n_heads, needles=0, resets=False)
+    if inputs is None:
+        k, v, g = wl.make_prefill(ws, dev, w.T - 1)
+    else:
+        k, v, g = inputs
+    q = wl.make_query(ws, dev)
+    kt, vt, gt = wl.make_token(ws, dev)
+    return OracleSample(ws, k, v, g, q, kt, vt, gt, n_heads, threads, max_steps)
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle timed on the host cores on a bounded sample."""
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    threads = n_heads = min(cores, 8, w.H)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    smp = oracle_sample_for(w, dev, n_heads, threads, args.warmup + args.steps)
+    for _ in range(args.warmup):
+        smp.step()
+    dt = sum(smp.step() for _ in range(args.steps)) / max(args.steps, 1)
+    rounds = -(-(w.B * w.H) // threads)          # a whole step = B*H heads, `threads` at a time
+    us = dt * rounds * 1e6
+    sample = (f"{n_heads} heads of batch item 0 at full context ({w.T} tokens), one decode step of each per "
+              f"timed step on {threads} threads; scaled by ceil(B*H/threads) = {rounds} to the whole step")
+    line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, 1),
+            "cpu_baseline": {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_config(w, ncopies):
+    return {"workload": w.name, "batch": w.B, "heads": w.H, "head_dim": w.D, "context": w.T,
+            "page_size": w.S, "budget": f"{w.budget_num}/{w.budget_den}", "budget_pages": w.budget_pages(),
+            "io_dtype": str(w.dtype).replace("torch.", ""), "state_dtype": "float32",
+            "l2": f"inputs larger than L2: {ncopies} independent caches rotated, fresh q/k/v/g every step"}
+
+
+# ------------------------------------------------------------------------- own arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="rq", choices=["rq", "reference"])
+    ap.add_argument("--workload", default="metric")
+    ap.add_argument("--copies", type=int, default=0, help="independent caches to rotate (0 = auto)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "rq" else args.warmup
+
+    w = pick_workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2605_28640_b200 as rq
+    from paper_2605_28640_b200 import build, workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    build.build_library()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    es = 2 if w.dtype == torch.bfloat16 else 4
+    T0 = w.T - 1                      # the first timed step brings the context to w.T
+    total_steps = args.warmup + args.steps
+    # caches: enough copies that their streamed bytes exceed L2 several times over
+    meta_b, kv_b = step_bytes(w, w.T)
+    l2 = torch.cuda.get_device_properties(local).L2_cache_size
+    ncopies = args.copies or max(2, min(8, -(-(4 * l2) // (meta_b + kv_b))))
+    # per copy: the timed loop, one more pass for the clock sampler, the profiled and e2e passes
+    per_copy = -(-total_steps // ncopies)
+    cap = T0 + 4 * per_copy + 64
+    K = w.budget_pages(w.T)
+    maxK = w.budget_pages(cap) + 1
+
+    caches, prefill_ms = [], []
+    q0 = wl.make_query(w, dev, 0)
+    import dataclasses
+    for c in range(ncopies):
+        wc = dataclasses.replace(w, seed=w.seed + 17 * c, resets=(c == 0))
+        k, v, g = wl.make_prefill(wc, dev, T0, q_for_needles=q0 if w.needles else None)
+        cache = rq.Cache(w.B, w.H, w.D, w.S, cap, w.dtype, w.gdtype, max_budget_pages=maxK, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        rq.rq_build_cache(cache.handle, k, v, g)
+        e1.record()
+        torch.cuda.synchronize()
+        prefill_ms.append(e0.elapsed_time(e1))
+        caches.append(cache)
+        if c == 0 and rank == 0 and not args.no_cpu_baseline:
+            nh = min(8, w.H)
+            sample_inputs = (k[:1, :, :nh].clone(), v[:1, :, :nh].clone(), g[:1, :, :nh].clone())
+        del k, v, g
+    torch.cuda.empty_cache()
+
+    # fresh inputs for every step, resident on the device before the timed region
+    pool = 64
+    qs = [wl.make_query(w, dev, s) for s in range(pool)]
+    toks = [wl.make_token(w, dev, s) for s in range(pool)]
+    outs = [torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=dev) for _ in range(4)]
+
+    def step(i):
+        kt, vt, gt = toks[i % pool]
+        rq.rq_decode_step(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[i % 4])
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        e0.record()
+        for i in range(args.warmup, total_steps):
+            step(i)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        # keep the sampler running over a second identical pass so that short runs get samples
+        t_end = time.time() + 0.6
+        j = total_steps
+        while time.time() < t_end and j < 2 * total_steps:
+            step(j)
+            j += 1
+            if j % 16 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = t.item() / args.steps
+    n_launches = args.steps * rq.binding.RQ_PROFILE_SLOTS
+
+    # ---- per-kernel times (separate pass, same rotation): events between the kernels of a step
+    prof = {}
+    nprof = min(args.steps, 50)
+    for i in range(nprof):
+        kt, vt, gt = toks[i % pool]
+        r = rq.rq_decode_step_profiled(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[0])
+        if i >= 3:
+            for name, us in r.items():
+                prof.setdefault(name, []).append(us)
+    kernel_us = {n: sum(v) / len(v) for n, v in prof.items()}
+
+    # ---- end to end through the host-buffer entry point (pinned host tensors, result read back)
+    hq = [q.cpu().pin_memory() for q in qs[:8]]
+    ht = [tuple(x.cpu().pin_memory() for x in tk) for tk in toks[:8]]
+    ho = torch.empty(w.B, w.H, w.D, dtype=w.dtype).pin_memory()
+    n_e2e = min(args.steps, 50)
+
+    def e2e_step(i):
+        kt, vt, gt = ht[i % 8]
+        rq.rq_decode_step_host(caches[i % ncopies].handle, hq[i % 8], kt, vt, gt, K, 0.0, ho)
+        torch.cuda.current_stream().synchronize()      # the caller reads the result before the next step
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    e0.record()
+    for i in range(n_e2e):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_us = t.item() / n_e2e * 1e3
+    in_bytes = w.B * w.H * w.D * (3 * es + (2 if w.gdtype == torch.bfloat16 else 4))
+    out_bytes = w.B * w.H * w.D * es
+
+    if rank != 0:
+        return
+
+    peak, peak_kind = measured_peak()
+    us = ms_per_step * 1e3
+    step_gbs = (meta_b + kv_b) / (us * 1e-6) / 1e9
+    kbytes = {"score": meta_b, "attend": kv_b}
+    dom = max(kbytes, key=lambda n: kernel_us.get(n, 0.0))
+    dom_gbs = kbytes[dom] / (kernel_us[dom] * 1e-6) / 1e9
+    line = {
+        "metric": METRIC, "value": us / world, "unit": "us/step", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w, ncopies),
+        "tokens_per_s": w.B * world / (us * 1e-6),
+        "step_hbm": {"algorithmic_bytes": meta_b + kv_b, "gbs": step_gbs, "frac_of_peak": step_gbs / peak,
+                     "frac_of_nominal_8tbs": step_gbs / 8000.0, "peak_gbs": peak, "peak_kind": peak_kind},
+        "kernels_us": kernel_us,
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": dom_gbs / peak, "peak_kind": peak_kind,
+                     "traffic": NCU_TRAFFIC.get(dom) if args.workload == "metric" else None,
+                     "bytes_per_launch": kbytes[dom],
+                     "others": {n: {"gbs": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9, "frac": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9 / peak}
+                                for n in kbytes if n != dom}},
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e_us / world, "unit": "us/step", "h2d_bytes_per_step": in_bytes,
+                "d2h_bytes_per_step": out_bytes},
+        "gpu_launches": n_launches,
+    }
+    if not args.no_prefill:
+        pm = sorted(prefill_ms)[len(prefill_ms) // 2]
+        gs = 2 if w.gdtype == torch.bfloat16 else 4
+        pbytes = w.B * w.H * T0 * w.D * (2 * es + gs + 2 * es) + w.B * w.H * w.pages(T0) * 2 * w.D * es
+        line["prefill"] = {"ms": pm, "tokens_per_s": w.B * T0 / (pm * 1e-3), "algorithmic_bytes": pbytes,
+                           "gbs": pbytes / (pm * 1e-3) / 1e9, "frac_of_peak": pbytes / (pm * 1e-3) / 1e9 / peak,
+                           "runs_ms": prefill_ms}
+    if not args.no_cpu_baseline:
+        nh = min(8, w.H)
+        threads = min(os.cpu_count() or 1, nh)
+        reps = 60
+        smp = oracle_sample_for(w, dev, nh, threads, reps + 2, inputs=sample_inputs)
+        smp.step()
+        wall = sum(smp.step() for _ in range(reps))
+        rounds_sample = -(-nh // threads)
+        rounds_full = -(-(w.B * w.H) // threads)
+        line["cpu_baseline"] = {
+            "value": wall / reps / rounds_sample * rounds_full * 1e6, "unit": "us/step", "cores": threads,
+            "kind": "oracle",
+            "sample": (f"{nh} heads of batch item 0 at full context, {reps} decode steps each on {threads} "
+                       f"threads ({wall:.1f} s wall); scaled to all {w.B * w.H} heads")}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

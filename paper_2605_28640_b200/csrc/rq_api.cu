@@ -37,6 +37,7 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     w.scan_chunks_cap = (c.capacity_tokens + ct - 1) / ct + 1;
     size_t off = 0;
     w.status = off;  off += align256(64 * sizeof(int32_t));
+    w.tickets = off; off += align256(BH * sizeof(int32_t));
     w.scores = off;  off += align256(BH * pc * sizeof(float));
     w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
     w.partial = off; off += align256(BH * kMaxSplits * (size_t)(c.head_dim + 2) * sizeof(float));
@@ -107,11 +108,10 @@ static int attend_from(const rq_cache *c, int64_t len, const void *q, const int3
     float *partial = (float *)((char *)c->workspace + w.partial);
     if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
     const int nsplit = choose_splits(a.B * a.H, n_idx, sm_count());
-    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, s) != cudaSuccess)
+    int32_t *tickets = (int32_t *)((char *)c->workspace + w.tickets);
+    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, tickets, o, s) != cudaSuccess)
         return RQ_ERR_CUDA;
     mark(ev, 4, s);
-    if (launch_combine(a, partial, nsplit, o, s) != cudaSuccess) return RQ_ERR_CUDA;
-    mark(ev, 5, s);
     return RQ_OK;
 }
 
@@ -187,7 +187,8 @@ int rq_cache_reset(rq_cache *cache, void *stream)
     const WorkspaceLayout w = workspace_layout(cache->cfg);
     if (cudaMemsetAsync(cache->state, 0, BH * 2 * cache->cfg.head_dim * sizeof(float), s) != cudaSuccess)
         return RQ_ERR_CUDA;
-    if (cudaMemsetAsync((char *)cache->workspace + w.status, 0, 64 * sizeof(int32_t), s) != cudaSuccess)
+    // status word and the split-K arrival counters (adjacent regions)
+    if (cudaMemsetAsync((char *)cache->workspace + w.status, 0, w.scores - w.status, s) != cudaSuccess)
         return RQ_ERR_CUDA;
     cache->len = 0;
     return RQ_OK;
@@ -257,7 +258,7 @@ int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t, con
 
 const char *rq_profile_slot_name(int slot)
 {
-    static const char *names[RQ_PROFILE_SLOTS] = {"update", "score", "topk", "attend", "combine"};
+    static const char *names[RQ_PROFILE_SLOTS] = {"update", "score", "topk", "attend"};
     return slot >= 0 && slot < RQ_PROFILE_SLOTS ? names[slot] : "";
 }
 

@@ -5,8 +5,8 @@
 //             every page (Eq. 3 with the min/max representatives of App. A.1)
 //   topk    — per (b,h) selection of the budget's pages, forced first/local
 //             pages inside the budget, ties to the lower page index, ascending
-//   attend  — split-K flash-decode over the selected pages only (Eq. 4) and
-//             the combine of the split partials
+//   attend  — split-K flash-decode over the selected pages only (Eq. 4); the
+//             split that finishes last for a head combines the partials
 // All of it is bandwidth-bound GEMV-like work on plain ALUs with fp32
 // accumulation; no tensor cores.
 #include <math_constants.h>
@@ -128,20 +128,31 @@ __global__ void __launch_bounds__(kScoreThreads) score_kernel(DecodeArgs a, cons
 
 // ---------------------------------------------------------------- top-k
 // One CTA per (b,h).  Scores become order-preserving 32-bit keys held in
-// registers (KPT consecutive pages per thread); forced pages get the largest
-// key.  The k-th largest key is found bit by bit (32 counting rounds, one
-// barrier each); pages with a larger key are taken, pages with an equal key
-// are taken in index order until the budget is full.  A block-wide prefix sum
-// over the per-thread counts gives each taken page its slot, so the output is
+// registers (consecutive pages per thread).  Forced pages (first / newest) are
+// taken outright and count inside the budget.  Among the rest, the k-th
+// largest key is found by a most-significant-digit radix select: the bits
+// that all keys share are skipped, then each pass histograms one 8-bit digit
+// of the keys that still match the prefix found so far (one private histogram
+// per warp in shared memory, so equal keys only collide inside a warp) and
+// walks the bins from the top until the remaining budget is used up.  Pages
+// with a larger key are taken; pages with an equal key are taken in index
+// order until the budget is full.  A block-wide prefix sum over the
+// per-thread counts gives each taken page its slot, so the output is
 // ascending and unique whatever the thread timing.
+constexpr uint32_t kKeyForced = 0xffffffffu;   // above every score key
+constexpr uint32_t kKeyPad = 0u;               // below every score key
+
 template <int KPT>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
                                                             int P, int K, int n_sink, int n_local,
                                                             int32_t *idx, int idx_stride, int budget)
 {
     constexpr int NTH = kTopkThreads, NWP = NTH / 32;
-    __shared__ int cnt[2][NWP];
-    __shared__ uint32_t wsum[NWP];
+    static_assert(NWP == 32, "second-level reductions are one warp wide");
+    __shared__ uint32_t hist[NWP][256];
+    __shared__ uint32_t red[NWP];
+    __shared__ uint32_t bins[256];
+    __shared__ uint32_t s_digit, s_krem;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
 
@@ -150,35 +161,89 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         return;
     }
     const float *sc = scores + (int64_t)bh * score_stride;
+    const int nk = (P + NTH - 1) / NTH;              // pages per thread in use (<= KPT)
+    const int base = tid * nk;
     uint32_t key[KPT];
-    const int base = tid * KPT;
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
 #pragma unroll
     for (int j = 0; j < KPT; ++j) {
         const int p = base + j;
-        uint32_t kx = 0;                             // below every real key
-        if (p < P) {
-            kx = order_key(sc[p]);
-            if (kx == 0xffffffffu) kx = 0xfffffffeu; // keep the top key for forced pages
-            if (kx == 0u) kx = 1u;
-            if (p < n_sink || p >= P - n_local) kx = 0xffffffffu;
+        uint32_t kx = kKeyPad;
+        if (j < nk && p < P) {
+            if (p < n_sink || p >= P - n_local) {
+                kx = kKeyForced;
+            } else {
+                kx = order_key(sc[p]);
+                kx = min(max(kx, 1u), 0xfffffffeu);  // stay clear of the two reserved keys
+                kmin = min(kmin, kx);
+                kmax = max(kmax, kx);
+            }
         }
         key[j] = kx;
     }
+    int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
 
-    // k-th largest key: largest tau with count(key >= tau) >= K
-    uint32_t tau = 0;
-    for (int bit = 31; bit >= 0; --bit) {
-        const uint32_t cand = tau | (1u << bit);
-        int c = 0;
+    // range of the score keys -> bits they all share
+    kmin = __reduce_min_sync(0xffffffffu, kmin);
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    if (lane == 0) { red[warp] = kmin; bins[warp] = kmax; }
+    __syncthreads();
+    kmin = __reduce_min_sync(0xffffffffu, red[lane]);
+    kmax = __reduce_max_sync(0xffffffffu, bins[lane]);
+    __syncthreads();
+
+    uint32_t tau;                                    // k-th largest key among the non-forced pages
+    if (k_rem <= 0) {
+        tau = 0xfffffffeu + 1u;                      // nothing but forced pages fits: take none of the rest
+    } else if (kmin == kmax) {
+        tau = kmin;
+    } else {
+        int hb = 31 - __clz(kmin ^ kmax);            // highest bit in which keys differ
+        tau = hb == 31 ? 0u : (kmax >> (hb + 1)) << (hb + 1);   // shared leading bits
+        while (hb >= 0) {
+            const int lo = hb >= 7 ? hb - 7 : 0;     // this pass decides bits hb .. lo
+            const int nb = hb - lo + 1;
+            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) c += key[j] >= cand;
-        c = __reduce_add_sync(0xffffffffu, c);
-        if (lane == 0) cnt[bit & 1][warp] = c;
-        __syncthreads();
-        int tot = 0;
+            for (int i = 0; i < 8; ++i) hist[warp][lane + 32 * i] = 0u;
+            __syncwarp();
 #pragma unroll
-        for (int w = 0; w < NWP; ++w) tot += cnt[bit & 1][w];
-        if (tot >= K) tau = cand;
+            for (int j = 0; j < KPT; ++j) {
+                if (j >= nk) break;
+                const uint32_t kx = key[j];
+                if (kx != kKeyForced && kx != kKeyPad && (kx & himask) == (tau & himask))
+                    atomicAdd(&hist[warp][(kx >> lo) & ((1u << nb) - 1u)], 1u);
+            }
+            __syncthreads();
+            // bin totals, then suffix sums from the top bin down
+            uint32_t c = 0;
+            if (tid < 256) {
+#pragma unroll 8
+                for (int w = 0; w < NWP; ++w) c += hist[w][tid];
+            }
+            uint32_t suf = c;                        // inclusive suffix sum inside the warp
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t t = __shfl_down_sync(0xffffffffu, suf, off);
+                if (lane + off < 32) suf += t;
+            }
+            if (tid < 256 && lane == 0) red[warp] = suf;   // warp totals (8 warps cover 256 bins)
+            __syncthreads();
+            if (tid < 256) {
+                uint32_t above = 0;                  // keys in the warps that hold higher bins
+                for (int w = warp + 1; w < 8; ++w) above += red[w];
+                const uint32_t s_incl = suf + above; // keys in bins >= tid
+                const uint32_t s_excl = s_incl - c;  // keys in bins >  tid
+                if (s_incl >= (uint32_t)k_rem && s_excl < (uint32_t)k_rem) {
+                    s_digit = (uint32_t)tid;
+                    s_krem = (uint32_t)k_rem - s_excl;
+                }
+            }
+            __syncthreads();
+            tau |= s_digit << lo;
+            k_rem = (int)s_krem;
+            hb = lo - 1;
+        }
     }
 
     // per-thread counts of "greater" (low half) and "equal" (high half)
@@ -191,15 +256,17 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
         if (lane >= off) incl += t;
     }
-    if (lane == 31) wsum[warp] = incl;
+    if (lane == 31) red[warp] = incl;
     __syncthreads();
-    uint32_t before = 0, total = 0;
+    const uint32_t wv = red[lane];
+    uint32_t winc = wv;                              // inclusive scan of the warp totals
 #pragma unroll
-    for (int w = 0; w < NWP; ++w) {
-        const uint32_t t = wsum[w];
-        if (w < warp) before += t;
-        total += t;
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, winc, off);
+        if (lane >= off) winc += t;
     }
+    const uint32_t total = __shfl_sync(0xffffffffu, winc, 31);
+    const uint32_t before = __shfl_sync(0xffffffffu, winc - wv, warp);
     const uint32_t excl = before + incl - mine;
     const int n_gt = (int)(total & 0xffffu);
     const int r = K - n_gt;                          // how many equal keys to take
@@ -209,7 +276,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         if (key[j] > tau) {
             out[gt_before + min(eq_before, r)] = base + j;
             ++gt_before;
-        } else if (key[j] == tau && tau != 0u) {
+        } else if (key[j] == tau && key[j] != kKeyPad) {
             if (eq_before < r) out[gt_before + eq_before] = base + j;
             ++eq_before;
         }
@@ -230,7 +297,8 @@ template <typename T, int D, int S>
 __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a, const T *q,
                                                                    const int32_t *idx, int n_idx,
                                                                    int idx_stride, float scale_log2,
-                                                                   float *partial, int nsplit)
+                                                                   float *partial, int nsplit,
+                                                                   int32_t *tickets, T *o)
 {
     constexpr int CH = VecOf<T>::N;
     constexpr int LPR = D / CH;                 // lanes per row
@@ -243,6 +311,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
 
     __shared__ float sm_m[NW], sm_l[NW];
     __shared__ float sm_acc[NW][D];
+    __shared__ int sm_last;
 
     const int split = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -356,24 +425,41 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
         dst[0] = m_all;
         dst[1] = l;
     }
-}
 
-// grid B*H, D threads: o = sum_s 2^(m_s-m) acc_s / sum_s 2^(m_s-m) l_s
-template <typename T, int D>
-__global__ void combine_kernel(const float *partial, int nsplit, T *o)
-{
-    const int bh = blockIdx.x, d = threadIdx.x;
-    const float *src = partial + (int64_t)bh * nsplit * (D + 2);
-    float m = -CUDART_INF_F;
-    for (int s = 0; s < nsplit; ++s) m = fmaxf(m, src[(int64_t)s * (D + 2)]);
-    float num = 0.0f, den = 0.0f;
-    for (int s = 0; s < nsplit; ++s) {
-        const float ms = src[(int64_t)s * (D + 2)];
-        const float f = ms == -CUDART_INF_F ? 0.0f : exp2f(ms - m);
-        num = fmaf(f, src[(int64_t)s * (D + 2) + 2 + d], num);
-        den = fmaf(f, src[(int64_t)s * (D + 2) + 1], den);
+    // The split that finishes last for this (b,h) combines all partials:
+    // o = sum_s 2^(m_s-m) acc_s / sum_s 2^(m_s-m) l_s.  No CTA waits for another.
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int t = atomicAdd(tickets + bh, 1);
+        sm_last = (t == nsplit - 1);
+        if (sm_last) tickets[bh] = 0;               // leave the counter ready for the next call
     }
-    store1<T>(o + (int64_t)bh * D + d, num / den);
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    const float *src = partial + (int64_t)bh * nsplit * (D + 2);
+    float *wgt = &sm_acc[0][0];                      // reuse: per-split weights (nsplit <= kMaxSplits <= D)
+    float m = -CUDART_INF_F;
+    for (int s2 = lane; s2 < nsplit; s2 += 32) m = fmaxf(m, __ldcg(src + (int64_t)s2 * (D + 2)));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    float den = 0.0f;
+    for (int s2 = lane; s2 < nsplit; s2 += 32) {
+        const float ms = __ldcg(src + (int64_t)s2 * (D + 2));
+        const float f = ms == -CUDART_INF_F ? 0.0f : exp2f(ms - m);
+        if (warp == 0) wgt[s2] = f;
+        den = fmaf(f, __ldcg(src + (int64_t)s2 * (D + 2) + 1), den);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+    __syncthreads();
+    for (int d = threadIdx.x; d < D; d += NW * 32) {
+        float num = 0.0f;
+#pragma unroll 8
+        for (int s2 = 0; s2 < nsplit; ++s2) num = fmaf(wgt[s2], __ldcg(src + (int64_t)s2 * (D + 2) + 2 + d), num);
+        store1<T>(o + (int64_t)bh * D + d, num / den);
+    }
 }
 
 // ---------------------------------------------------------------- dispatch helpers
@@ -465,25 +551,18 @@ int choose_splits(int BH, int n_idx, int sm_count)
 }
 
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
-                          int idx_stride, float scale, float *partial, int nsplit, cudaStream_t s)
+                          int idx_stride, float scale, float *partial, int nsplit, int32_t *tickets,
+                          void *o, cudaStream_t s)
 {
     const int BH = a.B * a.H;
     const float scale_log2 = scale * 1.4426950408889634f;
     dim3 grid((unsigned)nsplit, (unsigned)BH);
 #define CALL_ATT(T, D, S)                                                                        \
     attend_kernel<T, D, S><<<grid, kAttendWarps * 32, 0, s>>>(a, (const T *)q, idx, n_idx,       \
-                                                              idx_stride, scale_log2, partial, nsplit)
+                                                              idx_stride, scale_log2, partial, nsplit, \
+                                                              tickets, (T *)o)
     RQ_DISPATCH_TDS(a, CALL_ATT);
 #undef CALL_ATT
-    return cudaGetLastError();
-}
-
-cudaError_t launch_combine(const DecodeArgs &a, const float *partial, int nsplit, void *o, cudaStream_t s)
-{
-    const int BH = a.B * a.H;
-#define CALL_CMB(T, D, S) combine_kernel<T, D><<<BH, D, 0, s>>>(partial, nsplit, (T *)o)
-    RQ_DISPATCH_TDS(a, CALL_CMB);
-#undef CALL_CMB
     return cudaGetLastError();
 }
 

@@ -36,6 +36,7 @@ constexpr int kTargetSMs = 148;        // B200
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
     size_t status;    // int32[64]
+    size_t tickets;   // int32[BH]: split-K arrival counters, zero between calls
     size_t scores;    // float [BH][page_capacity]
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][kMaxSplits][D + 2]
@@ -73,8 +74,8 @@ cudaError_t launch_score(const DecodeArgs &a, const void *q, float *scores, cuda
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
                         int idx_stride, cudaStream_t s);
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
-                          int idx_stride, float scale, float *partial, int nsplit, cudaStream_t s);
-cudaError_t launch_combine(const DecodeArgs &a, const float *partial, int nsplit, void *o, cudaStream_t s);
+                          int idx_stride, float scale, float *partial, int nsplit, int32_t *tickets,
+                          void *o, cudaStream_t s);
 int choose_splits(int BH, int n_idx, int sm_count);
 
 }  // namespace rq
