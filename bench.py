@@ -317,7 +317,7 @@ def main():
 
     # ---- per-kernel times (separate pass, same rotation): events between the kernels of a step
     prof = {}
-    nprof = min(args.steps, 50)
+    nprof = min(args.steps, 50) + 3
     for i in range(nprof):
         kt, vt, gt = toks[i % pool]
         r = rq.rq_decode_step_profiled(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[0])
