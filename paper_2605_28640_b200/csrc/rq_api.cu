@@ -37,10 +37,11 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     w.scan_chunks_cap = (c.capacity_tokens + ct - 1) / ct + 1;
     size_t off = 0;
     w.status = off;  off += align256(64 * sizeof(int32_t));
-    w.tickets = off; off += align256(BH * sizeof(int32_t));
+    w.tickets = off; off += align256(BH * (size_t)kCtrStride * sizeof(int32_t));
     w.scores = off;  off += align256(BH * pc * sizeof(float));
     w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
-    w.partial = off; off += align256(BH * kMaxSplits * (size_t)(c.head_dim + 2) * sizeof(float));
+    const size_t slots = (size_t)attend_slots_per_head((int64_t)c.max_budget_pages * (c.page_size / 16));
+    w.partial = off; off += align256(BH * slots * (size_t)(c.head_dim + 4) * sizeof(float));
     w.agg = off;     off += align256(BH * (size_t)w.scan_chunks_cap * 3 * c.head_dim * sizeof(float));
     w.staging = off; off += align256(5 * BH * (size_t)c.head_dim * 4);
     w.total = off;
@@ -95,7 +96,8 @@ static int select_into(const rq_cache *c, int64_t len, const void *q, int budget
     DecodeArgs a = decode_args(c, len);
     if (launch_score(a, q, scores, s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 2, s);
-    if (launch_topk(a, scores, budget, idx, idx_stride, s) != cudaSuccess) return RQ_ERR_CUDA;
+    int32_t *attend_ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
+    if (launch_topk(a, scores, budget, idx, idx_stride, attend_ctr, s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 3, s);
     return RQ_OK;
 }
@@ -107,9 +109,9 @@ static int attend_from(const rq_cache *c, int64_t len, const void *q, const int3
     const WorkspaceLayout w = workspace_layout(c->cfg);
     float *partial = (float *)((char *)c->workspace + w.partial);
     if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
-    const int nsplit = choose_splits(a.B * a.H, n_idx, sm_count());
     int32_t *tickets = (int32_t *)((char *)c->workspace + w.tickets);
-    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, nsplit, tickets, o, s) != cudaSuccess)
+    const AttendCounters ctr = {tickets, tickets + 1, tickets + 2};
+    if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, ctr, o, sm_count(), s) != cudaSuccess)
         return RQ_ERR_CUDA;
     mark(ev, 4, s);
     return RQ_OK;
@@ -329,6 +331,10 @@ int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t 
     if (rc != RQ_OK) return rc;
     if (!q || !idx || !o || n_idx < 1 || cache->len < 1) return RQ_ERR_INVALID_ARG;
     if (n_idx > cache->cfg.max_budget_pages) return RQ_ERR_CAPACITY;
+    // the flash-decode counters must be zero at launch (in a decode step the selection kernel does this)
+    const WorkspaceLayout w = workspace_layout(cache->cfg);
+    if (cudaMemsetAsync((char *)cache->workspace + w.tickets, 0, w.scores - w.tickets, (cudaStream_t)stream) != cudaSuccess)
+        return RQ_ERR_CUDA;
     return attend_from(cache, cache->len, q, idx, n_idx, n_idx, scale, o, (cudaStream_t)stream);
 }
 

@@ -1,0 +1,543 @@
+// Sparse flash-decode over the selected pages only (Eq. 4), split-K with the
+// combine folded into the same launch.
+//
+// Work decomposition.  The unit of work is a tile: 16 consecutive token rows
+// of one selected page, i.e. a 16 x D block of decayed keys and the matching
+// block of decayed values (for 16-token pages a tile is the whole page and its
+// keys and values are adjacent in the cache).  A head's tiles are numbered in
+// the order of its index list and handed out one at a time through a per-head
+// ticket counter.  The grid is sized to what the GPU holds at once.  With at
+// least one CTA per head (the usual case) head h is served by the CTAs h,
+// h + BH, h + 2 BH, ...: they sit on SMs all over the chip, so every head's
+// group is equally fast, and inside a group a warp that the memory system
+// serves more slowly simply pulls fewer tickets; everybody finishes together.
+// With fewer CTAs than heads every warp sweeps forward over the heads from its
+// own starting head.  The per-head counters are zero at launch: the selection
+// kernel clears them (a memset does when this kernel is launched on its own).
+//
+// Data movement.  Each warp runs its own pipeline: lane 0 issues one bulk
+// (TMA, 1-D) copy for the key block and one for the value block of a tile into
+// the warp's ring of shared-memory stages, completion is counted on the
+// stage's mbarrier, and the warp consumes the stages in issue order and
+// refills a stage as soon as it has been read.  The first tickets of a warp
+// are its own by position, later ones come from the counter, and the ticket
+// and the page index of a refill are fetched one refill ahead, so neither the
+// atomic nor the index load is waited for.  No warp waits for another warp
+// inside the stream.
+//
+// Arithmetic (plain fp32 ALU work; a decode query is a GEMV): a warp-wide
+// 16-byte shared-memory read covers whole rows, lane -> (row, channel group);
+// row dot products are reduced over the lanes of a row, the softmax runs
+// online per warp in the exp2 domain, V is accumulated per lane for its
+// channel group.  At the end the warps of a CTA are merged through shared
+// memory into one partial (m, l, acc[D]) per head; the arrival that completes
+// a head's count combines the head's partials into the output row.
+#include <limits.h>
+#include <math_constants.h>
+
+#include "rq_async.cuh"
+#include "rq_device.cuh"
+#include "rq_internal.h"
+
+namespace rq {
+
+namespace {
+
+constexpr int kTileRows = 16;
+constexpr int kDoneTileBits = 20;                  // low bits of a head's done word count tiles
+constexpr int kDoneTileMask = (1 << kDoneTileBits) - 1;
+
+template <typename T, int D, int S>
+struct AttendGeom {
+    static constexpr int CH = VecOf<T>::N;         // elements per 16-byte vector
+    static constexpr int LPR = D / CH;             // lanes per row
+    static constexpr int RPI = 32 / LPR;           // rows per warp-wide read
+    static constexpr int TR = kTileRows;           // rows per tile
+    static constexpr int TPP = S / TR;             // tiles per page
+    static constexpr int NI = TR / RPI;            // warp-wide reads per tile and tensor
+    static constexpr int TILE_BYTES = TR * D * (int)sizeof(T);
+    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    static constexpr int NW = kAttendWarps;
+    static constexpr int DEPTH_RAW = kAttendRingBytes / (NW * STAGE_BYTES);
+    static constexpr int DEPTH = DEPTH_RAW < 2 ? 2 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
+    static constexpr int RING_BYTES = NW * DEPTH * STAGE_BYTES;
+    // ring | barriers | (head, valid rows) per stage | per-warp m, l, tiles, head | per-warp acc
+    static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 8 + 4 * NW * 4 + NW * D * 4;
+    static_assert(LPR <= 32 && TR % RPI == 0 && S % TR == 0, "unsupported geometry");
+    static_assert(TILE_BYTES % 16 == 0, "bulk copies move multiples of 16 bytes");
+};
+
+// Combine n partials of a head (one warp): o = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s.
+// Lane -> (channel group g = lane % 8 of D/8 channels, subset j = lane / 8): a lane sweeps the
+// partials s = j, j+4, ... with a running maximum, three records per round trip (their loads are
+// all issued before the first is used); the four subsets are merged with two shuffle steps.
+// A record is [m, l, -, -, acc[D]]; an empty one has m = -inf and zeros.
+template <typename T, int D>
+__device__ __forceinline__ void combine_head(const float *src, int n, T *o_row, int lane)
+{
+    constexpr int CPL = D / 8;                     // channels per lane
+    constexpr int NV = CPL / 4;                    // 16-byte vectors per lane and record
+    constexpr int U = 3;                           // records in flight per lane
+    const int g = lane & 7, j = lane >> 3;
+    float M = -CUDART_INF_F, L = 0.0f, A[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) A[c] = 0.0f;
+    for (int s0 = j; s0 < n; s0 += 4 * U) {
+        float2 ml[U];
+        float4 v[U][NV];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int s = s0 + 4 * u;
+            const float *rec = src + (int64_t)(s < n ? s : s0) * (D + 4);
+            ml[u] = ld_cg_now(reinterpret_cast<const float2 *>(rec));
+            if (s >= n) ml[u].x = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < NV; ++c) v[u][c] = ld_cg_now(reinterpret_cast<const float4 *>(rec + 4 + g * CPL) + c);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            // branch-free; an empty partial or a record past the end gets weight 0
+            const float Mn = fmaxf(M, ml[u].x);
+            const float fo = M == -CUDART_INF_F ? 0.0f : exp2f(M - Mn);
+            const float fn = ml[u].x == -CUDART_INF_F ? 0.0f : exp2f(ml[u].x - Mn);
+            L = fmaf(L, fo, ml[u].y * fn);
+#pragma unroll
+            for (int c = 0; c < NV; ++c) {
+                A[4 * c + 0] = fmaf(A[4 * c + 0], fo, v[u][c].x * fn);
+                A[4 * c + 1] = fmaf(A[4 * c + 1], fo, v[u][c].y * fn);
+                A[4 * c + 2] = fmaf(A[4 * c + 2], fo, v[u][c].z * fn);
+                A[4 * c + 3] = fmaf(A[4 * c + 3], fo, v[u][c].w * fn);
+            }
+            M = Mn;
+        }
+    }
+#pragma unroll
+    for (int off = 8; off < 32; off <<= 1) {
+        const float Mo = __shfl_xor_sync(0xffffffffu, M, off);
+        const float Lo = __shfl_xor_sync(0xffffffffu, L, off);
+        const float Mn = fmaxf(M, Mo);
+        const float fa = M == -CUDART_INF_F ? 0.0f : exp2f(M - Mn), fb = Mo == -CUDART_INF_F ? 0.0f : exp2f(Mo - Mn);
+        L = L * fa + Lo * fb;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) A[c] = A[c] * fa + __shfl_xor_sync(0xffffffffu, A[c], off) * fb;
+        M = Mn;
+    }
+    if (j == 0) {
+        const float inv = 1.0f / L;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) store1<T>(o_row + g * CPL + c, A[c] * inv);
+    }
+}
+
+template <typename T, int D, int S>
+__global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a, const T *q,
+                                                                   const int32_t *idx, int n_idx,
+                                                                   int idx_stride, float scale_log2,
+                                                                   float *partial, int slots_per_head,
+                                                                   AttendCounters ctr, T *o)
+{
+    using G = AttendGeom<T, D, S>;
+    constexpr int CH = G::CH, LPR = G::LPR, RPI = G::RPI, TR = G::TR, TPP = G::TPP, NI = G::NI;
+    constexpr int NW = G::NW, DEPTH = G::DEPTH;
+    constexpr unsigned FULL = 0xffffffffu;
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *ring = smem;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ring + G::RING_BYTES);
+    int2 *infos = reinterpret_cast<int2 *>(bars + NW * DEPTH);       // x: head (-1 = end), y: valid rows
+    float *sm_m = reinterpret_cast<float *>(infos + NW * DEPTH);
+    float *sm_l = sm_m + NW;
+    int *sm_t = reinterpret_cast<int *>(sm_l + NW);
+    int *sm_h = sm_t + NW;
+    float *sm_acc = reinterpret_cast<float *>(sm_h + NW);            // [NW][D]
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int rsub = lane / LPR, cgp = lane % LPR;
+    const int BH = a.B * a.H;
+    const int64_t P = (a.len + S - 1) / S;
+    const int per_head = n_idx * TPP;                // tiles per head (host: < 2^20)
+    const int NC = gridDim.x;                        // CTAs in the grid
+    const int TW = NC * NW;                          // warps in the grid
+    const int wg = blockIdx.x * NW + warp;
+
+    uint64_t *mybars = bars + warp * DEPTH;
+    int2 *myinfo = infos + warp * DEPTH;
+    unsigned char *myring = ring + (size_t)warp * DEPTH * G::STAGE_BYTES;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < DEPTH; ++s) mbar_init(&mybars[s], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    grid_dependency_wait();          // the index list and the cache come from earlier kernels
+    grid_launch_dependents();
+
+    const T *kvbase = static_cast<const T *>(a.kv);
+
+    // ------------------------------------------------------------ issue side
+    // fixed: at least one CTA per head; all warps of CTA c serve head c % BH and never change.
+    const bool fixed = NC >= BH;
+    const int h0 = fixed ? (int)(blockIdx.x % BH) : (int)((int64_t)wg * BH / TW);
+    // Warps that start on head h.  Each owns DEPTH tickets by position, so its ring fills
+    // without waiting for an atomic; the counter hands out the tickets after those.
+    auto owners = [&](int h) -> int {
+        if (fixed) return ((NC - h + BH - 1) / BH) * NW;
+        const int w = (int)(((int64_t)h * TW + BH - 1) / BH);
+        return w < TW && (int)((int64_t)w * BH / TW) == h ? 1 : 0;
+    };
+    int k = 0;                                       // sweep position: head (h0 + k) % BH
+    int ih = h0;                                     // head being pulled from
+    int base = owners(h0) * DEPTH;                   // first ticket of head ih that the counter hands out
+    bool drained = false;                            // no head has tiles left
+    int n_own = DEPTH;                               // own tickets not yet issued
+    int t_own = (fixed ? (int)(blockIdx.x / BH) * NW + warp : 0) * DEPTH;   // next own ticket
+    int pg_own = -1;                                 // lane j < DEPTH: page of own ticket j
+    if (lane < DEPTH && t_own + lane < per_head)
+        pg_own = __ldg(idx + (int64_t)h0 * idx_stride + (t_own + lane) / TPP);
+    int tA = 0, pgA = -1, tB = 0;                    // lane 0: next ticket + its page, ticket after it
+
+    auto prime = [&]() {                             // lane 0: first two counter tickets of head ih
+        tA = base + atomicAdd(ctr.next + ih * kCtrStride, 2);
+        tB = tA + 1;
+        pgA = tA < per_head ? __ldg(idx + (int64_t)ih * idx_stride + tA / TPP) : -1;
+    };
+    // move to the next head of the sweep that still has tickets
+    auto advance = [&]() {
+        for (;;) {
+            if (fixed || k + 1 >= BH) { drained = true; return; }
+            const int j = k + 1 + lane;
+            int c = INT_MAX;
+            if (j < BH) {
+                const int h = (h0 + j) % BH;
+                c = owners(h) * DEPTH + ld_volatile(ctr.next + h * kCtrStride);
+            }
+            const unsigned m = __ballot_sync(FULL, c < per_head);
+            if (m) {
+                k += __ffs(m);
+                ih = (h0 + k) % BH;
+                base = owners(ih) * DEPTH;
+                if (lane == 0) prime();
+                return;
+            }
+            k = min(k + 32, BH - 1);
+        }
+    };
+    // lane 0: start the copies of tile t of head h (page pg) into a stage
+    auto start_copies = [&](int stage, int h, int t, int pg) {
+        const int tile = t % TPP;
+        int valid = 0;
+        if (pg >= 0) {
+            if (pg < P) {
+                const int64_t left = a.len - ((int64_t)pg * S + tile * TR);
+                valid = left >= TR ? TR : (left > 0 ? (int)left : 0);
+            } else {
+                atomicExch(a.status, RQ_ERR_INVALID_ARG);
+            }
+        }
+        myinfo[stage] = make_int2(h, valid);
+        if (valid > 0) {
+            const T *kb = kvbase + (((int64_t)h * a.page_cap + pg) * 2) * S * D + tile * TR * D;
+            unsigned char *dst = myring + (size_t)stage * G::STAGE_BYTES;
+            mbar_arrive_expect_tx(&mybars[stage], G::STAGE_BYTES);
+            bulk_g2s(dst, kb, G::TILE_BYTES, &mybars[stage]);
+            bulk_g2s(dst + G::TILE_BYTES, kb + (int64_t)S * D, G::TILE_BYTES, &mybars[stage]);
+        }
+    };
+    // put the next tile into a stage (or the end mark); called by the whole warp
+    auto refill = [&](int stage) {
+        while (n_own > 0) {                          // own tickets first
+            const int t = t_own, pg = __shfl_sync(FULL, pg_own, DEPTH - n_own);
+            ++t_own;
+            --n_own;
+            if (t < per_head) {
+                if (lane == 0) start_copies(stage, h0, t, pg);
+                return;
+            }
+        }
+        for (;;) {
+            if (drained) {
+                if (lane == 0) myinfo[stage] = make_int2(-1, 0);
+                return;
+            }
+            int t = 0, pg = -1;
+            if (lane == 0) {
+                t = tA;
+                pg = pgA;
+                tA = tB;
+                pgA = tA < per_head ? __ldg(idx + (int64_t)ih * idx_stride + tA / TPP) : -1;
+                tB = base + atomicAdd(ctr.next + ih * kCtrStride, 1);
+            }
+            t = __shfl_sync(FULL, t, 0);
+            if (t < per_head) {
+                if (lane == 0) start_copies(stage, ih, t, pg);
+                return;
+            }
+            advance();                               // this head has no tickets left
+        }
+    };
+
+    if (lane == 0) prime();
+#pragma unroll
+    for (int s = 0; s < DEPTH; ++s) refill(s);
+    __syncwarp();
+
+    // ------------------------------------------------------------ consume side
+    int cur = -1;                                    // head of the running accumulation
+    int tiles = 0;                                   // tiles of `cur` consumed by this warp
+    int slot = 0;                                    // lane 0, sweeping only: this warp's partial slot in `cur`
+    float qf[CH], acc[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) { qf[c] = 0.0f; acc[c] = 0.0f; }
+    float m_run = -CUDART_INF_F, l_run = 0.0f;
+    int stage = 0;
+    uint32_t phase = 0;                              // one parity bit per stage
+    bool dead = false;                               // a wait ran out: stop streaming, finish cleanly
+
+    // sum the row groups of the warp (they share m_run); lanes < LPR end up with the channel sums
+    auto merge_rows = [&]() {
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1) {
+            l_run += __shfl_xor_sync(FULL, l_run, off);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) acc[c] += __shfl_xor_sync(FULL, acc[c], off);
+        }
+    };
+    // after a partial of head h has been written by this warp: count it, and combine if it was the last
+    auto arrive = [&](int h, int count_word, int expect_ctas, int n_fixed) {
+        __threadfence();
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+            const int now = atomicAdd(ctr.done + h * kCtrStride, count_word) + count_word;
+            last = (now & kDoneTileMask) == per_head && (now >> kDoneTileBits) == expect_ctas;
+        }
+        last = __shfl_sync(FULL, last, 0);
+        if (last) {
+            __threadfence();
+            const int n = n_fixed >= 0 ? n_fixed : min(ld_volatile(ctr.nslot + h * kCtrStride), slots_per_head);
+            combine_head<T, D>(partial + (int64_t)h * slots_per_head * (D + 4), n, o + (int64_t)h * D, lane);
+        }
+    };
+    // sweeping mode: the warp writes its own partial for head h
+    auto flush_warp = [&](int h) {
+        merge_rows();
+        const int s = __shfl_sync(FULL, slot, 0);
+        if (s >= slots_per_head) {                   // cannot happen: a warp joins a head by holding one of its tiles
+            if (lane == 0) atomicExch(a.status, RQ_ERR_CAPACITY);
+            return;
+        }
+        float *dst = partial + ((int64_t)h * slots_per_head + s) * (D + 4);
+        if (lane == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m_run, l_run);
+        if (lane < LPR) {
+#pragma unroll
+            for (int c = 0; c < CH; c += 4)
+                *reinterpret_cast<float4 *>(dst + 4 + cgp * CH + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+        }
+        arrive(h, tiles, 0, -1);
+    };
+
+    for (;;) {
+        const int2 inf = myinfo[stage];
+        if (inf.x < 0) break;
+        if (inf.x != cur) {
+            if (cur >= 0) flush_warp(cur);           // only a sweeping warp changes head
+            cur = inf.x;
+            tiles = 0;
+            if (!fixed && lane == 0) slot = atomicAdd(ctr.nslot + cur * kCtrStride, 1);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                qf[c] = load1<T>(q + (int64_t)cur * D + cgp * CH + c) * scale_log2;
+                acc[c] = 0.0f;
+            }
+            m_run = -CUDART_INF_F;
+            l_run = 0.0f;
+        }
+        const int valid = inf.y;
+        if (valid > 0 && !dead) {
+            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u)) {
+                // give the copies still in flight the same bounded chance to land, then stop
+                for (int s = 0; s < DEPTH; ++s)
+                    if (s != stage && myinfo[s].x >= 0 && myinfo[s].y > 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
+                if (lane == 0) atomicExch(a.status, RQ_ERR_TIMEOUT);
+                dead = true;
+            }
+            phase ^= 1u << stage;
+        }
+        if (valid > 0 && !dead) {
+            const T *ks = reinterpret_cast<const T *>(myring + (size_t)stage * G::STAGE_BYTES);
+            const T *vs = ks + TR * D;
+            float s[NI];
+            float m_new = m_run;
+#pragma unroll
+            for (int n = 0; n < NI; ++n) {
+                float kf[CH];
+                unpack16<T>(lds16(ks + (n * 32 + lane) * CH), kf);
+                float d = 0.0f;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) d = fmaf(qf[c], kf[c], d);
+#pragma unroll
+                for (int off = LPR / 2; off > 0; off >>= 1) d += __shfl_xor_sync(FULL, d, off);
+                const int row = n * RPI + rsub;
+                s[n] = row < valid ? d : -CUDART_INF_F;
+                m_new = fmaxf(m_new, s[n]);
+            }
+#pragma unroll
+            for (int off = LPR; off < 32; off <<= 1) m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, off));
+            const float alpha = exp2f(m_run - m_new);    // 0 on the first tile (m_run = -inf)
+            m_run = m_new;
+            l_run *= alpha;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) acc[c] *= alpha;
+#pragma unroll
+            for (int n = 0; n < NI; ++n) {
+                const float p = exp2f(s[n] - m_new);     // 0 for masked rows
+                l_run += p;
+                float vf[CH];
+                unpack16<T>(lds16(vs + (n * 32 + lane) * CH), vf);
+#pragma unroll
+                for (int c = 0; c < CH; ++c) acc[c] = fmaf(p, vf[c], acc[c]);
+            }
+        }
+        ++tiles;
+        __syncwarp();                                // every lane is done with the stage
+        if (dead) drained = true;
+        refill(stage);
+        __syncwarp();
+        stage = stage + 1 == DEPTH ? 0 : stage + 1;
+    }
+
+    if (!fixed) {
+        if (cur >= 0 && !dead) flush_warp(cur);
+        return;
+    }
+
+    // fixed mode: merge the CTA's warps (all on head h0) into one partial in slot blockIdx / BH
+    merge_rows();
+    if (dead || cur < 0) { m_run = -CUDART_INF_F; l_run = 0.0f; tiles = 0; }
+    if (lane == 0) { sm_m[warp] = m_run; sm_l[warp] = l_run; sm_t[warp] = tiles; sm_h[warp] = dead; }
+    if (lane < LPR) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) sm_acc[warp * D + cgp * CH + c] = (dead || cur < 0) ? 0.0f : acc[c];
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    constexpr int CPL = D / 32;                      // channels per lane in the merge
+    float m_all = -CUDART_INF_F, l_all = 0.0f;
+    int t_all = 0, any_dead = 0;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { m_all = fmaxf(m_all, sm_m[w]); t_all += sm_t[w]; any_dead |= sm_h[w]; }
+    float out[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) out[c] = 0.0f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+        const float f = sm_m[w] == -CUDART_INF_F ? 0.0f : exp2f(sm_m[w] - m_all);
+        l_all = fmaf(f, sm_l[w], l_all);
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) out[c] = fmaf(f, sm_acc[w * D + lane * CPL + c], out[c]);
+    }
+    if (any_dead) return;                            // status already says why; the head stays incomplete
+    const int rank = blockIdx.x / BH;
+    float *dst = partial + ((int64_t)h0 * slots_per_head + rank) * (D + 4);
+    if (lane == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m_all, l_all);
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) dst[4 + lane * CPL + c] = out[c];
+    const int team = (NC - h0 + BH - 1) / BH;        // CTAs on this head; each arrives exactly once
+    arrive(h0, t_all + (1 << kDoneTileBits), team, team);
+}
+
+}  // namespace
+
+namespace {
+
+// CTAs of this kernel one SM holds at once, found once per device.
+template <typename T, int D, int S>
+cudaError_t attend_occupancy(int *ctas_per_sm)
+{
+    using G = AttendGeom<T, D, S>;
+    static int cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cached[dev] == 0) {
+        e = cudaFuncSetAttribute(attend_kernel<T, D, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, attend_kernel<T, D, S>, G::NW * 32, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        cached[dev] = n > 0 ? n : 1;
+    }
+    *ctas_per_sm = cached[dev];
+    return cudaSuccess;
+}
+
+template <typename T, int D, int S>
+cudaError_t launch_attend_t(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx, int idx_stride,
+                            float scale, float *partial, const AttendCounters &ctr, void *o, int sm_count,
+                            cudaStream_t s)
+{
+    using G = AttendGeom<T, D, S>;
+    const int64_t per_head = (int64_t)n_idx * G::TPP;
+    const int64_t W = (int64_t)a.B * a.H * per_head;
+    if (W <= 0 || per_head > kDoneTileMask) return cudaErrorInvalidValue;
+    int occ = 1;
+    cudaError_t e = attend_occupancy<T, D, S>(&occ);
+    if (e != cudaSuccess) return e;
+    const int grid = attend_grid(W, occ * sm_count);
+    const int slots = attend_slots_per_head(per_head);
+    const float scale_log2 = scale * 1.4426950408889634f;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(G::NW * 32);
+    cfg.dynamicSmemBytes = G::SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, attend_kernel<T, D, S>, a, (const T *)q, idx, n_idx, idx_stride, scale_log2,
+                              partial, slots, ctr, (T *)o);
+}
+
+}  // namespace
+
+int attend_grid(int64_t tiles, int resident_ctas)
+{
+    // every warp should get at least two tiles, every CTA at least one
+    int64_t g = tiles / (2 * kAttendWarps);
+    if (g > resident_ctas) g = resident_ctas;
+    if (g > kAttendMaxWarps / kAttendWarps) g = kAttendMaxWarps / kAttendWarps;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+int attend_slots_per_head(int64_t tiles_per_head)
+{
+    // A head gets one partial per CTA that serves it (fewer than its tiles / 8, see attend_grid)
+    // or, when warps sweep over heads, one per warp that held one of its tiles.
+    return (int)(tiles_per_head < kAttendMaxWarps ? tiles_per_head : kAttendMaxWarps);
+}
+
+cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx, int idx_stride,
+                          float scale, float *partial, const AttendCounters &ctr, void *o, int sm_count,
+                          cudaStream_t s)
+{
+#define RQ_ATT(T, D, S) return launch_attend_t<T, D, S>(a, q, idx, n_idx, idx_stride, scale, partial, ctr, o, sm_count, s)
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128 && a.S == 16) RQ_ATT(bf16, 128, 16);
+        if (a.D == 128 && a.S == 64) RQ_ATT(bf16, 128, 64);
+        if (a.D == 64 && a.S == 16) RQ_ATT(bf16, 64, 16);
+        if (a.D == 64 && a.S == 64) RQ_ATT(bf16, 64, 64);
+    } else {
+        if (a.D == 128 && a.S == 16) RQ_ATT(float, 128, 16);
+        if (a.D == 128 && a.S == 64) RQ_ATT(float, 128, 64);
+        if (a.D == 64 && a.S == 16) RQ_ATT(float, 64, 16);
+        if (a.D == 64 && a.S == 64) RQ_ATT(float, 64, 64);
+    }
+#undef RQ_ATT
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace rq

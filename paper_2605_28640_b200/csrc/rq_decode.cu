@@ -5,8 +5,6 @@
 //             every page (Eq. 3 with the min/max representatives of App. A.1)
 //   topk    — per (b,h) selection of the budget's pages, forced first/local
 //             pages inside the budget, ties to the lower page index, ascending
-//   attend  — split-K flash-decode over the selected pages only (Eq. 4); the
-//             split that finishes last for a head combines the partials
 // All of it is bandwidth-bound GEMV-like work on plain ALUs with fp32
 // accumulation; no tensor cores.
 #include <math_constants.h>
@@ -145,7 +143,8 @@ constexpr uint32_t kKeyPad = 0u;               // below every score key
 template <int KPT>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
                                                             int P, int K, int n_sink, int n_local,
-                                                            int32_t *idx, int idx_stride, int budget)
+                                                            int32_t *idx, int idx_stride, int budget,
+                                                            int32_t *attend_ctr)
 {
     constexpr int NTH = kTopkThreads, NWP = NTH / 32;
     static_assert(NWP == 32, "second-level reductions are one warp wide");
@@ -155,6 +154,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     __shared__ uint32_t s_digit, s_krem;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
+    if (tid < 3) attend_ctr[bh * kCtrStride + tid] = 0;   // the flash-decode kernel's counters of this head
 
     if (K >= P) {                                    // dense: every page, in order
         for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
@@ -284,184 +284,6 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
-// ---------------------------------------------------------------- attend
-// grid (nsplit, B*H), kAttendWarps warps.  Split s owns a contiguous range of
-// the head's index list; its warps take the pages of that range round-robin.
-// A warp reads a page's K block and V block with fully coalesced 16-byte
-// loads: one load instruction covers RPI whole rows, lane -> (row, channel
-// group).  Row dot products are reduced over the LPR lanes of a row; the
-// softmax runs online per warp in the exp2 domain; V is accumulated per lane
-// for its channel group over the rows it loaded, and the row groups are
-// merged once at the end.
-template <typename T, int D, int S>
-__global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a, const T *q,
-                                                                   const int32_t *idx, int n_idx,
-                                                                   int idx_stride, float scale_log2,
-                                                                   float *partial, int nsplit,
-                                                                   int32_t *tickets, T *o)
-{
-    constexpr int CH = VecOf<T>::N;
-    constexpr int LPR = D / CH;                 // lanes per row
-    constexpr int RPI = 32 / LPR;               // rows per load instruction
-    constexpr int TR = 16;                      // rows handled per register tile
-    constexpr int NTILE = S / TR;               // register tiles per page
-    constexpr int NI = TR / RPI;                // load instructions per tile and tensor
-    constexpr int NW = kAttendWarps;
-    static_assert(LPR <= 32 && TR % RPI == 0 && S % TR == 0, "unsupported geometry");
-
-    __shared__ float sm_m[NW], sm_l[NW];
-    __shared__ float sm_acc[NW][D];
-    __shared__ int sm_last;
-
-    const int split = blockIdx.x, bh = blockIdx.y;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int rsub = lane / LPR, cgp = lane % LPR;
-    const int64_t P = (a.len + S - 1) / S;
-
-    float qf[CH];
-#pragma unroll
-    for (int i = 0; i < CH; ++i) qf[i] = load1<T>(q + (int64_t)bh * D + cgp * CH + i) * scale_log2;
-
-    const int lo = (int)((int64_t)n_idx * split / nsplit);
-    const int hi = (int)((int64_t)n_idx * (split + 1) / nsplit);
-    const int32_t *list = idx + (int64_t)bh * idx_stride;
-    const T *kvb = static_cast<const T *>(a.kv) + (int64_t)bh * a.page_cap * 2 * S * D;
-
-    float m_run = -CUDART_INF_F, l_run = 0.0f;
-    float acc[CH];
-#pragma unroll
-    for (int i = 0; i < CH; ++i) acc[i] = 0.0f;
-
-    for (int it = lo + warp; it < hi; it += NW) {
-        const int page = list[it];
-        if (page < 0) continue;
-        if (page >= P) {
-            if (lane == 0) atomicExch(a.status, RQ_ERR_INVALID_ARG);
-            continue;
-        }
-        const int valid = (int)min((int64_t)S, a.len - (int64_t)page * S);
-        const T *kb = kvb + (int64_t)page * 2 * S * D;
-        const T *vb = kb + S * D;
-#pragma unroll 1
-        for (int tile = 0; tile < NTILE; ++tile) {
-            if (tile * TR >= valid) break;          // the rest of the page holds no token
-            uint4 rk[NI], rv[NI];
-#pragma unroll
-            for (int i = 0; i < NI; ++i) rk[i] = ldcs16(kb + ((tile * NI + i) * 32 + lane) * CH);
-#pragma unroll
-            for (int i = 0; i < NI; ++i) rv[i] = ldcs16(vb + ((tile * NI + i) * 32 + lane) * CH);
-
-            float s[NI];
-            float m_new = m_run;
-#pragma unroll
-            for (int i = 0; i < NI; ++i) {
-                float kf[CH];
-                unpack16<T>(rk[i], kf);
-                float d = 0.0f;
-#pragma unroll
-                for (int c = 0; c < CH; ++c) d = fmaf(qf[c], kf[c], d);
-#pragma unroll
-                for (int off = LPR / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
-                const int row = tile * TR + i * RPI + rsub;
-                s[i] = row < valid ? d : -CUDART_INF_F;
-                m_new = fmaxf(m_new, s[i]);
-            }
-#pragma unroll
-            for (int off = LPR; off < 32; off <<= 1)
-                m_new = fmaxf(m_new, __shfl_xor_sync(0xffffffffu, m_new, off));
-            const float alpha = exp2f(m_run - m_new);    // 0 on the first tile (m_run = -inf)
-            m_run = m_new;
-            l_run *= alpha;
-#pragma unroll
-            for (int c = 0; c < CH; ++c) acc[c] *= alpha;
-#pragma unroll
-            for (int i = 0; i < NI; ++i) {
-                const float p = exp2f(s[i] - m_new);     // 0 for masked rows
-                l_run += p;
-                float vf[CH];
-                unpack16<T>(rv[i], vf);
-#pragma unroll
-                for (int c = 0; c < CH; ++c) acc[c] = fmaf(p, vf[c], acc[c]);
-            }
-        }
-    }
-
-    // merge the row groups of the warp (they share m_run); every lane of a row
-    // added the same p, so the warp's l is the sum over one lane per row group
-#pragma unroll
-    for (int off = LPR; off < 32; off <<= 1) {
-        l_run += __shfl_xor_sync(0xffffffffu, l_run, off);
-#pragma unroll
-        for (int c = 0; c < CH; ++c) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], off);
-    }
-    if (lane == 0) { sm_m[warp] = m_run; sm_l[warp] = l_run; }
-    if (lane < LPR) {
-#pragma unroll
-        for (int c = 0; c < CH; ++c) sm_acc[warp][cgp * CH + c] = acc[c];
-    }
-    __syncthreads();
-
-    // merge the warps and write this split's partial: [m, l, acc[D]]
-    float m_all = -CUDART_INF_F;
-#pragma unroll
-    for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, sm_m[w]);
-    float *dst = partial + ((int64_t)bh * nsplit + split) * (D + 2);
-    for (int d = threadIdx.x; d < D; d += NW * 32) {
-        float o = 0.0f;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) {
-            const float f = sm_m[w] == -CUDART_INF_F ? 0.0f : exp2f(sm_m[w] - m_all);
-            o = fmaf(f, sm_acc[w][d], o);
-        }
-        dst[2 + d] = o;
-    }
-    if (threadIdx.x == 0) {
-        float l = 0.0f;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) {
-            const float f = sm_m[w] == -CUDART_INF_F ? 0.0f : exp2f(sm_m[w] - m_all);
-            l = fmaf(f, sm_l[w], l);
-        }
-        dst[0] = m_all;
-        dst[1] = l;
-    }
-
-    // The split that finishes last for this (b,h) combines all partials:
-    // o = sum_s 2^(m_s-m) acc_s / sum_s 2^(m_s-m) l_s.  No CTA waits for another.
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const int t = atomicAdd(tickets + bh, 1);
-        sm_last = (t == nsplit - 1);
-        if (sm_last) tickets[bh] = 0;               // leave the counter ready for the next call
-    }
-    __syncthreads();
-    if (!sm_last) return;
-    __threadfence();
-    const float *src = partial + (int64_t)bh * nsplit * (D + 2);
-    float *wgt = &sm_acc[0][0];                      // reuse: per-split weights (nsplit <= kMaxSplits <= D)
-    float m = -CUDART_INF_F;
-    for (int s2 = lane; s2 < nsplit; s2 += 32) m = fmaxf(m, __ldcg(src + (int64_t)s2 * (D + 2)));
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-    float den = 0.0f;
-    for (int s2 = lane; s2 < nsplit; s2 += 32) {
-        const float ms = __ldcg(src + (int64_t)s2 * (D + 2));
-        const float f = ms == -CUDART_INF_F ? 0.0f : exp2f(ms - m);
-        if (warp == 0) wgt[s2] = f;
-        den = fmaf(f, __ldcg(src + (int64_t)s2 * (D + 2) + 1), den);
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
-    __syncthreads();
-    for (int d = threadIdx.x; d < D; d += NW * 32) {
-        float num = 0.0f;
-#pragma unroll 8
-        for (int s2 = 0; s2 < nsplit; ++s2) num = fmaf(wgt[s2], __ldcg(src + (int64_t)s2 * (D + 2) + 2 + d), num);
-        store1<T>(o + (int64_t)bh * D + d, num / den);
-    }
-}
-
 // ---------------------------------------------------------------- dispatch helpers
 #define RQ_DISPATCH_TDS(a, CALL)                                                         \
     do {                                                                                 \
@@ -515,7 +337,7 @@ cudaError_t launch_score(const DecodeArgs &a, const void *q, float *scores, cuda
 }
 
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, cudaStream_t s)
+                        int idx_stride, int32_t *attend_ctr, cudaStream_t s)
 {
     const int P = (int)((a.len + a.S - 1) / a.S);
     const int K = budget < P ? budget : P;
@@ -527,7 +349,7 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     if (nl > P - ns) nl = P - ns;
     const int per = (P + kTopkThreads - 1) / kTopkThreads;
 #define CALL_TOPK(KPT) \
-    topk_kernel<KPT><<<BH, kTopkThreads, 0, s>>>(scores, a.page_cap, P, K, ns, nl, idx, idx_stride, budget)
+    topk_kernel<KPT><<<BH, kTopkThreads, 0, s>>>(scores, a.page_cap, P, K, ns, nl, idx, idx_stride, budget, attend_ctr)
     if (per <= 1) CALL_TOPK(1);
     else if (per <= 2) CALL_TOPK(2);
     else if (per <= 4) CALL_TOPK(4);
@@ -536,33 +358,6 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     else if (per <= 32) CALL_TOPK(32);
     else return cudaErrorInvalidValue;
 #undef CALL_TOPK
-    return cudaGetLastError();
-}
-
-int choose_splits(int BH, int n_idx, int sm_count)
-{
-    // aim at four resident CTAs per SM in total
-    int target = sm_count * 4;
-    int ns = (target + BH - 1) / BH;
-    if (ns > kMaxSplits) ns = kMaxSplits;
-    if (ns > n_idx) ns = n_idx;
-    if (ns < 1) ns = 1;
-    return ns;
-}
-
-cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
-                          int idx_stride, float scale, float *partial, int nsplit, int32_t *tickets,
-                          void *o, cudaStream_t s)
-{
-    const int BH = a.B * a.H;
-    const float scale_log2 = scale * 1.4426950408889634f;
-    dim3 grid((unsigned)nsplit, (unsigned)BH);
-#define CALL_ATT(T, D, S)                                                                        \
-    attend_kernel<T, D, S><<<grid, kAttendWarps * 32, 0, s>>>(a, (const T *)q, idx, n_idx,       \
-                                                              idx_stride, scale_log2, partial, nsplit, \
-                                                              tickets, (T *)o)
-    RQ_DISPATCH_TDS(a, CALL_ATT);
-#undef CALL_ATT
     return cudaGetLastError();
 }
 

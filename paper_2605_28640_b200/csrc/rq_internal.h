@@ -27,8 +27,10 @@ inline int scan_chunk_tokens(int head_dim, int dtype)
 }
 
 // ---- decode-side geometry ----
-constexpr int kMaxSplits = 64;         // most split-K partials per (b,h)
-constexpr int kAttendWarps = 4;        // warps per flash-decode CTA
+constexpr int kAttendWarps = 4;        // warps per flash-decode CTA, each with its own copy pipeline
+constexpr int kAttendRingBytes = 96 * 1024;  // shared-memory ring of one flash-decode CTA (all warps)
+constexpr int kAttendMaxWarps = 1536;  // upper bound of the warps of a flash-decode grid
+constexpr int kCtrStride = 64;         // int32 between the counters of two heads (256 bytes: different L2 lines)
 constexpr int kTopkThreads = 1024;     // threads of the selection CTA
 constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
 constexpr int kTargetSMs = 148;        // B200
@@ -36,10 +38,10 @@ constexpr int kTargetSMs = 148;        // B200
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
     size_t status;    // int32[64]
-    size_t tickets;   // int32[BH]: split-K arrival counters, zero between calls
+    size_t tickets;   // int32[BH * kCtrStride]: flash-decode ticket / slot / done counters of every head
     size_t scores;    // float [BH][page_capacity]
     size_t sel;       // int32 [BH][max_budget]
-    size_t partial;   // float [BH][kMaxSplits][D + 2]
+    size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
     size_t agg;       // float [BH][scan chunks][3][D]
     size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
     size_t total;
@@ -71,11 +73,22 @@ struct DecodeArgs {
 cudaError_t launch_update(const DecodeArgs &a, const void *k_t, const void *v_t, const void *g_t,
                           cudaStream_t s);
 cudaError_t launch_score(const DecodeArgs &a, const void *q, float *scores, cudaStream_t s);
+// attend_ctr: the flash-decode counters (cleared here, one head per CTA)
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, cudaStream_t s);
+                        int idx_stride, int32_t *attend_ctr, cudaStream_t s);
+// per-head counters of the flash-decode kernel, kCtrStride int32 apart from head to head; all
+// zero at launch
+struct AttendCounters {
+    int32_t *next;    // next tile ticket that the counter hands out
+    int32_t *nslot;   // partial records handed out to sweeping warps
+    int32_t *done;    // tiles whose partial has been written (low 20 bits) | CTA arrivals (high bits)
+};
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
-                          int idx_stride, float scale, float *partial, int nsplit, int32_t *tickets,
-                          void *o, cudaStream_t s);
-int choose_splits(int BH, int n_idx, int sm_count);
+                          int idx_stride, float scale, float *partial, const AttendCounters &ctr, void *o,
+                          int sm_count, cudaStream_t s);
+// flash-decode grid for a number of tiles and the CTAs the device holds at once
+int attend_grid(int64_t tiles, int resident_ctas);
+// partial records a head can need when it has this many tiles
+int attend_slots_per_head(int64_t tiles_per_head);
 
 }  // namespace rq
