@@ -180,17 +180,17 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     const int h0 = fixed ? (int)(blockIdx.x % BH) : (int)((int64_t)wg * BH / TW);
     // Warps that start on head h.  Each owns DEPTH tickets by position, so its ring fills
     // without waiting for an atomic; the counter hands out the tickets after those.
+    auto first_warp = [&](int h) -> int { return (int)(((int64_t)h * TW + BH - 1) / BH); };   // sweeping mode
     auto owners = [&](int h) -> int {
         if (fixed) return ((NC - h + BH - 1) / BH) * NW;
-        const int w = (int)(((int64_t)h * TW + BH - 1) / BH);
-        return w < TW && (int)((int64_t)w * BH / TW) == h ? 1 : 0;
+        return first_warp(h + 1) - first_warp(h);
     };
     int k = 0;                                       // sweep position: head (h0 + k) % BH
     int ih = h0;                                     // head being pulled from
     int base = owners(h0) * DEPTH;                   // first ticket of head ih that the counter hands out
     bool drained = false;                            // no head has tiles left
     int n_own = DEPTH;                               // own tickets not yet issued
-    int t_own = (fixed ? (int)(blockIdx.x / BH) * NW + warp : 0) * DEPTH;   // next own ticket
+    int t_own = (fixed ? (int)(blockIdx.x / BH) * NW + warp : wg - first_warp(h0)) * DEPTH;   // next own ticket
     int pg_own = -1;                                 // lane j < DEPTH: page of own ticket j
     if (lane < DEPTH && t_own + lane < per_head)
         pg_own = __ldg(idx + (int64_t)h0 * idx_stride + (t_own + lane) / TPP);
