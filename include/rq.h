@@ -169,7 +169,7 @@ RQ_API int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *
  * rq_profile_slot_name(i) names slot i.  The computation and its results are
  * those of rq_decode_step [Eq. 1, Eq. 3, Eq. 4].
  * Errors: as rq_decode_step; INVALID_ARG for NULL kernel_us. */
-#define RQ_PROFILE_SLOTS 4
+#define RQ_PROFILE_SLOTS 3
 RQ_API int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t,
                                    const void *v_t, const void *g_t, int32_t budget_pages,
                                    float scale, void *o, int32_t *sel_idx_out,

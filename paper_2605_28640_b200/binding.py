@@ -132,7 +132,7 @@ def rq_decode_step_host(cache: rq_cache, q, k_t, v_t, g_t, budget_pages, scale, 
            "rq_decode_step_host")
 
 
-RQ_PROFILE_SLOTS = 4
+RQ_PROFILE_SLOTS = 3
 
 
 def rq_decode_step_profiled(cache: rq_cache, q, k_t, v_t, g_t, budget_pages, scale, o, sel_idx_out=None,

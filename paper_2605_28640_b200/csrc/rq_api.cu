@@ -89,16 +89,18 @@ static void mark(cudaEvent_t *ev, int i, cudaStream_t s)
     if (ev) cudaEventRecord(ev[i], s);
 }
 
-// score + select into `idx` (device, stride idx_stride), for a cache of length len
-static int select_into(const rq_cache *c, int64_t len, const void *q, int budget, float *scores,
-                       int32_t *idx, int idx_stride, cudaStream_t s, cudaEvent_t *ev = nullptr)
+// (optionally append a token, then) score + select into `idx` (device, stride idx_stride), for a
+// cache of length len after the append
+static int select_into(const rq_cache *c, int64_t len, const void *q, const void *k_t, const void *v_t,
+                       const void *g_t, int do_update, int budget, float *scores, int32_t *idx, int idx_stride,
+                       cudaStream_t s, cudaEvent_t *ev = nullptr)
 {
     DecodeArgs a = decode_args(c, len);
-    if (launch_score(a, q, scores, s) != cudaSuccess) return RQ_ERR_CUDA;
+    int32_t *ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
+    if (launch_score(a, q, k_t, v_t, g_t, scores, ctr + 3, do_update, sm_count(), s) != cudaSuccess) return RQ_ERR_CUDA;
+    mark(ev, 1, s);
+    if (launch_topk(a, scores, budget, idx, idx_stride, ctr, s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 2, s);
-    int32_t *attend_ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
-    if (launch_topk(a, scores, budget, idx, idx_stride, attend_ctr, s) != cudaSuccess) return RQ_ERR_CUDA;
-    mark(ev, 3, s);
     return RQ_OK;
 }
 
@@ -113,7 +115,7 @@ static int attend_from(const rq_cache *c, int64_t len, const void *q, const int3
     const AttendCounters ctr = {tickets, tickets + 1, tickets + 2};
     if (launch_attend(a, q, idx, n_idx, idx_stride, scale, partial, ctr, o, sm_count(), s) != cudaSuccess)
         return RQ_ERR_CUDA;
-    mark(ev, 4, s);
+    mark(ev, 3, s);
     return RQ_OK;
 }
 
@@ -131,13 +133,10 @@ static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, con
     float *scores = (float *)((char *)cache->workspace + w.scores);
     int32_t *sel = sel_idx_out ? sel_idx_out : (int32_t *)((char *)cache->workspace + w.sel);
 
-    DecodeArgs a = decode_args(cache, cache->len);
     mark(ev, 0, s);
-    if (launch_update(a, k_t, v_t, g_t, s) != cudaSuccess) return RQ_ERR_CUDA;
-    mark(ev, 1, s);
     cache->len += 1;
     const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
-    int st = select_into(cache, cache->len, q, budget_pages, scores, sel, budget_pages, s, ev);
+    int st = select_into(cache, cache->len, q, k_t, v_t, g_t, 1, budget_pages, scores, sel, budget_pages, s, ev);
     if (st != RQ_OK) return st;
     const int n_idx = (int)(budget_pages < P ? budget_pages : P);
     return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s, ev);
@@ -260,7 +259,7 @@ int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t, con
 
 const char *rq_profile_slot_name(int slot)
 {
-    static const char *names[RQ_PROFILE_SLOTS] = {"update", "score", "topk", "attend"};
+    static const char *names[RQ_PROFILE_SLOTS] = {"score", "topk", "attend"};
     return slot >= 0 && slot < RQ_PROFILE_SLOTS ? names[slot] : "";
 }
 
@@ -311,7 +310,7 @@ int rq_select_pages(rq_cache *cache, const void *q, int32_t budget_pages, float 
     cudaStream_t s = (cudaStream_t)stream;
     const WorkspaceLayout w = workspace_layout(c);
     float *scores = (float *)((char *)cache->workspace + w.scores);
-    const int st = select_into(cache, cache->len, q, budget_pages, scores, idx_out, budget_pages, s);
+    const int st = select_into(cache, cache->len, q, nullptr, nullptr, nullptr, 0, budget_pages, scores, idx_out, budget_pages, s);
     if (st != RQ_OK) return st;
     if (scores_out) {
         const int64_t P = (cache->len + c.page_size - 1) / c.page_size;

@@ -27,6 +27,8 @@ inline int scan_chunk_tokens(int head_dim, int dtype)
 }
 
 // ---- decode-side geometry ----
+constexpr int kScoreWarps = 4;         // warps per scoring CTA, each with its own copy pipeline
+constexpr int kScoreRingBytes = 96 * 1024;   // shared-memory ring of one scoring CTA (all warps)
 constexpr int kAttendWarps = 4;        // warps per flash-decode CTA, each with its own copy pipeline
 constexpr int kAttendRingBytes = 96 * 1024;  // shared-memory ring of one flash-decode CTA (all warps)
 constexpr int kAttendMaxWarps = 1536;  // upper bound of the warps of a flash-decode grid
@@ -38,7 +40,7 @@ constexpr int kTargetSMs = 148;        // B200
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
     size_t status;    // int32[64]
-    size_t tickets;   // int32[BH * kCtrStride]: flash-decode ticket / slot / done counters of every head
+    size_t tickets;   // int32[BH * kCtrStride]: per head, flash-decode ticket / slot / done counters (+0..2) and the scoring ticket counter (+3)
     size_t scores;    // float [BH][page_capacity]
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
@@ -70,10 +72,12 @@ struct DecodeArgs {
     int n_sink, n_local;
     int32_t *status;
 };
-cudaError_t launch_update(const DecodeArgs &a, const void *k_t, const void *v_t, const void *g_t,
-                          cudaStream_t s);
-cudaError_t launch_score(const DecodeArgs &a, const void *q, float *scores, cudaStream_t s);
-// attend_ctr: the flash-decode counters (cleared here, one head per CTA)
+// a.len is the length the scores are for.  do_update: first append the token (k_t, v_t, g_t) as
+// position a.len - 1 (state, cache row, newest page's bounds).  next: the scoring ticket counters
+// (head h at next[h * kCtrStride]), zero at launch.
+cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                         float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s);
+// attend_ctr: the ticket counters of the streaming kernels (cleared here, one head per CTA)
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
                         int idx_stride, int32_t *attend_ctr, cudaStream_t s);
 // per-head counters of the flash-decode kernel, kCtrStride int32 apart from head to head; all

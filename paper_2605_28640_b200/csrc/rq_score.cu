@@ -1,0 +1,395 @@
+// First kernel of a decode step: the single-token state update (Eq. 1) fused
+// with the scoring of every page by the query's upper bound (Eq. 3 with the
+// per-page min/max representatives of App. A.1).
+//
+// Scoring.  U_p = sum_i max(q_i min_p[i], q_i max_p[i]).  A page's bounds are
+// one contiguous record [min row][max row] of 2*D elements and a head's
+// records are contiguous, so scoring is one long stream per head.  Since
+// min <= max, max(q*min, q*max) = q*max for q >= 0 and q*min for q < 0: a lane
+// that holds part of a max row multiplies by max(q, 0), a lane that holds part
+// of a min row by min(q, 0); every loaded byte is used and a record's score is
+// a sum over the lanes that share it.
+//
+// Data movement is the flash-decode kernel's: the unit of work is 8 KiB of
+// consecutive records of one head, a head's units are handed out through a
+// per-head ticket counter (own tickets by position first), head h is served by
+// the CTAs h, h + BH, ... (or, with fewer CTAs than heads, warps sweep over
+// the heads), and every warp streams its units through its own ring of
+// shared-memory stages filled by bulk (TMA, 1-D) copies.  The ticket counters
+// are zero at launch; the selection kernel, which always runs next, clears
+// them.
+//
+// Update.  When a token is appended, the CTAs h, h + gridDim, ... first do head
+// h's recurrence step on the fp32 state, append the rounded state to the
+// cache, merge it into the newest page's bounds, and write that page's score
+// from the merged bounds they hold; the stream leaves the newest page out, so
+// nobody reads a record while it is being rewritten.
+#include <limits.h>
+#include <math_constants.h>
+
+#include "rq_async.cuh"
+#include "rq_device.cuh"
+#include "rq_internal.h"
+
+namespace rq {
+
+namespace {
+
+constexpr int kUnitBytes = 8192;
+
+template <typename T, int D>
+struct ScoreGeom {
+    static constexpr int CH = VecOf<T>::N;           // elements per 16-byte vector
+    static constexpr int REC_BYTES = 2 * D * (int)sizeof(T);
+    static constexpr int VPR = REC_BYTES / 16;       // 16-byte vectors per record
+    static constexpr int RU = kUnitBytes / REC_BYTES;   // records per unit
+    static constexpr int LPP = VPR > 32 ? 32 : VPR;  // lanes that share one record in a warp-wide read
+    static constexpr int VPL = VPR / LPP;            // vectors per lane and record (1 or 2)
+    static constexpr int PPW = 32 / LPP;             // records per warp-wide read
+    static constexpr int NR = RU / PPW;              // record groups per unit
+    static constexpr int NW = kScoreWarps;
+    static constexpr int DEPTH_RAW = kScoreRingBytes / (NW * kUnitBytes);
+    static constexpr int DEPTH = DEPTH_RAW < 2 ? 2 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
+    static constexpr int RING_BYTES = NW * DEPTH * kUnitBytes;
+    // ring | barriers | (head, first record, records) per stage | reduction scratch of the update
+    static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 16 + 64;
+    static_assert(VPL == 1 || VPL == 2, "unsupported record width");
+    static_assert(D <= NW * 32, "the update uses one thread per channel");
+};
+
+// One step of Eq. 1 for head h (thread d < D owns channel d): new state, cache row, bounds of
+// the newest page, and that page's score.  `len` is the length AFTER the append.
+template <typename T, int D>
+__device__ __forceinline__ void update_head(const DecodeArgs &a, int h, const T *q, const T *k_t, const T *v_t,
+                                            const void *g_t, float *scores, float *red)
+{
+    const int d = threadIdx.x;
+    const int S = a.S;
+    const int64_t pos = a.len - 1;
+    const int64_t page = pos / S;
+    const int slot = (int)(pos % S);
+    float term = 0.0f;
+    if (d < D) {
+        float *st = a.state + (int64_t)h * 2 * D;
+        const float g = a.gate_dtype == RQ_BF16 ? load1<bf16>(static_cast<const bf16 *>(g_t) + (int64_t)h * D + d)
+                                                : load1<float>(static_cast<const float *>(g_t) + (int64_t)h * D + d);
+        const float om = 1.0f - g;
+        const float sk = fmaf(g, st[d], om * load1<T>(k_t + (int64_t)h * D + d));
+        const float sv = fmaf(g, st[D + d], om * load1<T>(v_t + (int64_t)h * D + d));
+        st[d] = sk;
+        st[D + d] = sv;
+        T *pg = static_cast<T *>(a.kv) + (((int64_t)h * a.page_cap + page) * 2) * S * D;
+        store1<T>(pg + (int64_t)slot * D + d, sk);
+        store1<T>(pg + (int64_t)(S + slot) * D + d, sv);
+        const float r = round_storage<T>(sk);
+        T *m = static_cast<T *>(a.meta) + (((int64_t)h * a.page_cap + page) * 2) * D;
+        float mn = r, mx = r;
+        if (slot == 0) {
+            // a fresh page: clear its unused slots so that later reads are defined
+            for (int s2 = 1; s2 < S; ++s2) {
+                store1<T>(pg + (int64_t)s2 * D + d, 0.0f);
+                store1<T>(pg + (int64_t)(S + s2) * D + d, 0.0f);
+            }
+        } else {
+            mn = fminf(load1<T>(m + d), r);
+            mx = fmaxf(load1<T>(m + D + d), r);
+        }
+        store1<T>(m + d, mn);
+        store1<T>(m + D + d, mx);
+        const float qd = load1<T>(q + (int64_t)h * D + d);
+        term = fmaxf(qd * mn, qd * mx);
+    }
+    // score of the newest page: sum of the D terms
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) term += __shfl_xor_sync(0xffffffffu, term, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = term;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.0f;
+        for (int w = 0; w < (D + 31) / 32; ++w) s += red[w];
+        scores[(int64_t)h * a.page_cap + page] = s;
+    }
+    __syncthreads();
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, const T *q, const T *k_t,
+                                                                 const T *v_t, const void *g_t, float *scores,
+                                                                 int32_t *next, int do_update)
+{
+    using G = ScoreGeom<T, D>;
+    constexpr int CH = G::CH, VPR = G::VPR, RU = G::RU, LPP = G::LPP, VPL = G::VPL, PPW = G::PPW, NR = G::NR;
+    constexpr int NW = G::NW, DEPTH = G::DEPTH;
+    constexpr unsigned FULL = 0xffffffffu;
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *ring = smem;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(ring + G::RING_BYTES);
+    int4 *infos = reinterpret_cast<int4 *>(bars + NW * DEPTH);       // x: head (-1 = end), y: first record, z: records
+    float *red = reinterpret_cast<float *>(infos + NW * DEPTH);
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int sub = lane / LPP, c = lane % LPP;
+    const int BH = a.B * a.H;
+    const int P = (int)((a.len + a.S - 1) / a.S);
+    const int Ps = do_update ? P - 1 : P;            // records per head that are streamed
+    const int per_head = (Ps + RU - 1) / RU;         // units per head
+    const int NC = gridDim.x, TW = NC * NW;
+    const int wg = blockIdx.x * NW + warp;
+
+    uint64_t *mybars = bars + warp * DEPTH;
+    int4 *myinfo = infos + warp * DEPTH;
+    unsigned char *myring = ring + (size_t)warp * DEPTH * kUnitBytes;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < DEPTH; ++s) mbar_init(&mybars[s], 1);
+        mbar_init_fence();
+    }
+    __syncthreads();
+    grid_dependency_wait();          // earlier kernels may still read what the update rewrites
+    grid_launch_dependents();
+
+    if (do_update)
+        for (int h = blockIdx.x; h < BH; h += NC) update_head<T, D>(a, h, q, k_t, v_t, g_t, scores, red);
+
+    const T *meta = static_cast<const T *>(a.meta);
+
+    // ------------------------------------------------------------ issue side (as in the flash-decode kernel)
+    const bool fixed = NC >= BH;
+    const int h0 = fixed ? (int)(blockIdx.x % BH) : (int)((int64_t)wg * BH / TW);
+    auto first_warp = [&](int h) -> int { return (int)(((int64_t)h * TW + BH - 1) / BH); };   // sweeping mode
+    auto owners = [&](int h) -> int {                // warps that start on head h; each owns DEPTH tickets
+        if (fixed) return ((NC - h + BH - 1) / BH) * NW;
+        return first_warp(h + 1) - first_warp(h);
+    };
+    int k = 0;                                       // sweep position: head (h0 + k) % BH
+    int ih = h0;                                     // head being pulled from
+    int base = owners(h0) * DEPTH;                   // first ticket of head ih that the counter hands out
+    bool drained = false;
+    int n_own = DEPTH;                               // own tickets not yet issued
+    int t_own = (fixed ? (int)(blockIdx.x / BH) * NW + warp : wg - first_warp(h0)) * DEPTH;
+    int tA = 0;                                      // lane 0: next counter ticket
+
+    auto advance = [&]() {                           // next head of the sweep that still has tickets
+        for (;;) {
+            if (fixed || k + 1 >= BH) { drained = true; return; }
+            const int j = k + 1 + lane;
+            int cnt = INT_MAX;
+            if (j < BH) {
+                const int h = (h0 + j) % BH;
+                cnt = owners(h) * DEPTH + ld_volatile(next + h * kCtrStride);
+            }
+            const unsigned m = __ballot_sync(FULL, cnt < per_head);
+            if (m) {
+                k += __ffs(m);
+                ih = (h0 + k) % BH;
+                base = owners(ih) * DEPTH;
+                if (lane == 0) tA = base + atomicAdd(next + ih * kCtrStride, 1);
+                return;
+            }
+            k = min(k + 32, BH - 1);
+        }
+    };
+    auto start_copy = [&](int stage, int h, int t) { // lane 0
+        const int first = t * RU;
+        const int n = min(RU, Ps - first);
+        myinfo[stage] = make_int4(h, first, n, 0);
+        const T *src = meta + ((int64_t)h * a.page_cap + first) * 2 * D;
+        mbar_arrive_expect_tx(&mybars[stage], n * G::REC_BYTES);
+        bulk_g2s(myring + (size_t)stage * kUnitBytes, src, n * G::REC_BYTES, &mybars[stage]);
+    };
+    auto refill = [&](int stage) {                   // whole warp
+        while (n_own > 0) {
+            const int t = t_own;
+            ++t_own;
+            --n_own;
+            if (t < per_head) {
+                if (lane == 0) start_copy(stage, h0, t);
+                return;
+            }
+        }
+        for (;;) {
+            if (drained) {
+                if (lane == 0) myinfo[stage] = make_int4(-1, 0, 0, 0);
+                return;
+            }
+            int t = 0;
+            if (lane == 0) {
+                t = tA;
+                tA = base + atomicAdd(next + ih * kCtrStride, 1);
+            }
+            t = __shfl_sync(FULL, t, 0);
+            if (t < per_head) {
+                if (lane == 0) start_copy(stage, ih, t);
+                return;
+            }
+            advance();
+        }
+    };
+
+    if (lane == 0) tA = base + atomicAdd(next + ih * kCtrStride, 1);
+#pragma unroll
+    for (int s = 0; s < DEPTH; ++s) refill(s);
+    __syncwarp();
+
+    // ------------------------------------------------------------ consume side
+    int cur = -1;
+    float qs[VPL][CH];                               // this lane's slice of q, split by sign
+#pragma unroll
+    for (int v = 0; v < VPL; ++v)
+#pragma unroll
+        for (int i = 0; i < CH; ++i) qs[v][i] = 0.0f;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool dead = false;
+
+    for (;;) {
+        const int4 inf = myinfo[stage];
+        if (inf.x < 0) break;
+        if (inf.x != cur) {
+            cur = inf.x;
+#pragma unroll
+            for (int v = 0; v < VPL; ++v) {
+                const int vec = c + v * LPP;         // vector index inside the record
+                const bool is_max = vec >= VPR / 2;
+                const int ch0 = (vec % (VPR / 2)) * CH;
+#pragma unroll
+                for (int i = 0; i < CH; ++i) {
+                    const float x = load1<T>(q + (int64_t)cur * D + ch0 + i);
+                    qs[v][i] = is_max ? fmaxf(x, 0.0f) : fminf(x, 0.0f);
+                }
+            }
+        }
+        if (!dead) {
+            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u)) {
+                for (int s = 0; s < DEPTH; ++s)
+                    if (s != stage && myinfo[s].x >= 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
+                if (lane == 0) atomicExch(a.status, RQ_ERR_TIMEOUT);
+                dead = true;
+            }
+            phase ^= 1u << stage;
+        }
+        if (!dead) {
+            const unsigned char *ub = myring + (size_t)stage * kUnitBytes;
+            float val[NR];
+#pragma unroll
+            for (int gi = 0; gi < NR; ++gi) {
+                const unsigned char *rec = ub + (size_t)(gi * PPW + sub) * G::REC_BYTES;
+                float s = 0.0f;
+#pragma unroll
+                for (int v = 0; v < VPL; ++v) {
+                    float m[CH];
+                    unpack16<T>(lds16(rec + (c + v * LPP) * 16), m);
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) s = fmaf(qs[v][i], m[i], s);
+                }
+                val[gi] = s;
+            }
+            // sum over the LPP lanes of a record; while more than one value is left a step also
+            // halves the values a lane carries, so the whole reduction costs about NR shuffles
+            int n = NR;
+#pragma unroll
+            for (int off = LPP / 2; off > 0; off >>= 1) {
+                if (n > 1) {
+                    const int half = n / 2;
+                    const bool hi = (lane & off) != 0;
+#pragma unroll
+                    for (int i = 0; i < NR / 2; ++i) {
+                        if (i < half) {
+                            const float send = hi ? val[i] : val[i + half];
+                            const float keep = hi ? val[i + half] : val[i];
+                            val[i] = keep + __shfl_xor_sync(FULL, send, off);
+                        }
+                    }
+                    n = half;
+                } else {
+                    val[0] += __shfl_xor_sync(FULL, val[0], off);
+                }
+            }
+            // the lane now holds the sum of record group `gi` if its low lane bits are zero
+            constexpr int LOG_LPP = LPP == 32 ? 5 : (LPP == 16 ? 4 : (LPP == 8 ? 3 : 2));
+            constexpr int LOG_NR = NR == 32 ? 5 : (NR == 16 ? 4 : (NR == 8 ? 3 : (NR == 4 ? 2 : (NR == 2 ? 1 : 0))));
+            static_assert((1 << LOG_LPP) == LPP && (1 << LOG_NR) == NR && LOG_NR <= LOG_LPP, "unsupported reduction shape");
+            const int gi = (c >> (LOG_LPP - LOG_NR)) & (NR - 1);
+            const bool writer = (c & ((1 << (LOG_LPP - LOG_NR)) - 1)) == 0;
+            const int r = gi * PPW + sub;
+            if (writer && r < inf.z) scores[(int64_t)cur * a.page_cap + inf.y + r] = val[0];
+        }
+        __syncwarp();
+        if (dead) drained = true;
+        refill(stage);
+        __syncwarp();
+        stage = stage + 1 == DEPTH ? 0 : stage + 1;
+    }
+}
+
+}  // namespace
+
+namespace {
+
+template <typename T, int D>
+cudaError_t score_occupancy(int *ctas_per_sm)
+{
+    using G = ScoreGeom<T, D>;
+    static int cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cached[dev] == 0) {
+        e = cudaFuncSetAttribute(score_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, score_kernel<T, D>, G::NW * 32, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        cached[dev] = n > 0 ? n : 1;
+    }
+    *ctas_per_sm = cached[dev];
+    return cudaSuccess;
+}
+
+template <typename T, int D>
+cudaError_t launch_score_t(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                           float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s)
+{
+    using G = ScoreGeom<T, D>;
+    const int64_t P = (a.len + a.S - 1) / a.S;
+    const int64_t Ps = do_update ? P - 1 : P;
+    const int64_t units = (int64_t)a.B * a.H * ((Ps + G::RU - 1) / G::RU);
+    int occ = 1;
+    cudaError_t e = score_occupancy<T, D>(&occ);
+    if (e != cudaSuccess) return e;
+    int64_t grid = units / (2 * G::NW);              // every warp should get at least two units
+    if (grid > (int64_t)occ * sm_count) grid = (int64_t)occ * sm_count;
+    if (grid < 1) grid = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(G::NW * 32);
+    cfg.dynamicSmemBytes = G::SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, score_kernel<T, D>, a, (const T *)q, (const T *)k_t, (const T *)v_t, g_t, scores,
+                              next, do_update);
+}
+
+}  // namespace
+
+cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                         float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s)
+{
+    if (a.len <= 0) return cudaSuccess;
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128) return launch_score_t<bf16, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+        if (a.D == 64) return launch_score_t<bf16, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+    } else {
+        if (a.D == 128) return launch_score_t<float, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+        if (a.D == 64) return launch_score_t<float, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace rq
