@@ -3,6 +3,7 @@
 // budget (App. A.1), ties to the lower page index, output ascending.
 #include <math_constants.h>
 
+#include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
 
@@ -11,35 +12,45 @@ namespace rq {
 namespace {
 
 // ---------------------------------------------------------------- top-k
-// One CTA per (b,h).  Scores become order-preserving 32-bit keys held in
-// registers (consecutive pages per thread).  Forced pages (first / newest) are
-// taken outright and count inside the budget.  Among the rest, the k-th
-// largest key is found by a most-significant-digit radix select: the bits
-// that all keys share are skipped, then each pass histograms one 8-bit digit
-// of the keys that still match the prefix found so far (one private histogram
-// per warp in shared memory, so equal keys only collide inside a warp) and
-// walks the bins from the top until the remaining budget is used up.  Pages
-// with a larger key are taken; pages with an equal key are taken in index
-// order until the budget is full.  A block-wide prefix sum over the
-// per-thread counts gives each taken page its slot, so the output is
-// ascending and unique whatever the thread timing.
+// One CTA per (b,h).  Scores become order-preserving 32-bit keys in shared
+// memory.  Forced pages (first / newest) are taken outright and count inside
+// the budget.  Among the rest, the k-th largest key is found by a
+// most-significant-digit radix select: the bits that all keys share are
+// skipped, then each pass histograms one 11-bit digit of the keys that still
+// match the prefix found so far and walks the bins from the top until the
+// remaining budget is used up; a pass whose chosen bin is wanted whole ends
+// the search early.  Pages with a larger key are taken; pages with an equal
+// key are taken in index order until the budget is full.  For the output,
+// warp w owns a contiguous range of pages and walks it row by row (row j:
+// pages base_w + 32 j + lane): warp ballots give every taken page its rank
+// inside the warp and a scan over the warp totals its rank in the head, so the
+// output is ascending and unique whatever the thread timing.
+//
+// Every CTA runs this code once on an SM whose instruction cache holds another
+// kernel's code, so the loops are kept rolled: fetching the instructions is a
+// visible part of the run time.
 constexpr uint32_t kKeyForced = 0xffffffffu;   // above every score key
-constexpr uint32_t kKeyPad = 0u;               // below every score key
+constexpr int kDigitBits = 11;
+constexpr int kBins = 1 << kDigitBits;
 
-template <int KPT>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
                                                             int P, int K, int n_sink, int n_local,
                                                             int32_t *idx, int idx_stride, int budget,
                                                             int32_t *attend_ctr)
 {
     constexpr int NTH = kTopkThreads, NWP = NTH / 32;
+    constexpr unsigned FULL = 0xffffffffu;
     static_assert(NWP == 32, "second-level reductions are one warp wide");
-    __shared__ uint32_t hist[NWP][256];
-    __shared__ uint32_t red[NWP];
-    __shared__ uint32_t bins[256];
-    __shared__ uint32_t s_digit, s_krem;
+    static_assert(kBins == 2 * NTH, "a thread owns two bins in the suffix scan");
+    constexpr int NH = 2;                            // histogram copies; warp w adds to copy w % NH
+    extern __shared__ __align__(16) uint32_t skey[]; // [P] keys of the head
+    __shared__ __align__(16) uint32_t hist[NH][kBins];   // read back as 8-byte pairs
+    __shared__ uint32_t red[NWP], red2[NWP];
+    __shared__ uint32_t s_digit, s_krem, s_cnt;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
+    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
+    grid_launch_dependents();
     if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
 
     if (K >= P) {                                    // dense: every page, in order
@@ -47,36 +58,27 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         return;
     }
     const float *sc = scores + (int64_t)bh * score_stride;
-    const int nk = (P + NTH - 1) / NTH;              // pages per thread in use (<= KPT)
-    const int base = tid * nk;
-    uint32_t key[KPT];
     uint32_t kmin = 0xffffffffu, kmax = 0u;
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        const int p = base + j;
-        uint32_t kx = kKeyPad;
-        if (j < nk && p < P) {
-            if (p < n_sink || p >= P - n_local) {
-                kx = kKeyForced;
-            } else {
-                kx = order_key(sc[p]);
-                kx = min(max(kx, 1u), 0xfffffffeu);  // stay clear of the two reserved keys
-                kmin = min(kmin, kx);
-                kmax = max(kmax, kx);
-            }
+#pragma unroll 4
+    for (int p = tid; p < P; p += NTH) {
+        uint32_t kx = kKeyForced;
+        if (p >= n_sink && p < P - n_local) {
+            kx = order_key(__ldcg(sc + p));
+            kx = min(max(kx, 1u), 0xfffffffeu);      // stay clear of the reserved key
+            kmin = min(kmin, kx);
+            kmax = max(kmax, kx);
         }
-        key[j] = kx;
+        skey[p] = kx;
     }
     int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
 
     // range of the score keys -> bits they all share
-    kmin = __reduce_min_sync(0xffffffffu, kmin);
-    kmax = __reduce_max_sync(0xffffffffu, kmax);
-    if (lane == 0) { red[warp] = kmin; bins[warp] = kmax; }
+    kmin = __reduce_min_sync(FULL, kmin);
+    kmax = __reduce_max_sync(FULL, kmax);
+    if (lane == 0) { red[warp] = kmin; red2[warp] = kmax; }
     __syncthreads();
-    kmin = __reduce_min_sync(0xffffffffu, red[lane]);
-    kmax = __reduce_max_sync(0xffffffffu, bins[lane]);
-    __syncthreads();
+    kmin = __reduce_min_sync(FULL, red[lane]);
+    kmax = __reduce_max_sync(FULL, red2[lane]);
 
     uint32_t tau;                                    // k-th largest key among the non-forced pages
     if (k_rem <= 0) {
@@ -86,86 +88,97 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     } else {
         int hb = 31 - __clz(kmin ^ kmax);            // highest bit in which keys differ
         tau = hb == 31 ? 0u : (kmax >> (hb + 1)) << (hb + 1);   // shared leading bits
+#pragma unroll 1
         while (hb >= 0) {
-            const int lo = hb >= 7 ? hb - 7 : 0;     // this pass decides bits hb .. lo
-            const int nb = hb - lo + 1;
+            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
+            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
             const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) hist[warp][lane + 32 * i] = 0u;
-            __syncwarp();
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                if (j >= nk) break;
-                const uint32_t kx = key[j];
-                if (kx != kKeyForced && kx != kKeyPad && (kx & himask) == (tau & himask))
-                    atomicAdd(&hist[warp][(kx >> lo) & ((1u << nb) - 1u)], 1u);
+            __syncthreads();                         // the previous pass (and red/red2) has been read
+#pragma unroll 1
+            for (int i = tid; i < NH * kBins; i += NTH) (&hist[0][0])[i] = 0u;
+            __syncthreads();
+#pragma unroll 2
+            for (int p = tid; p < P; p += NTH) {
+                const uint32_t kx = skey[p];
+                if (kx != kKeyForced && (kx & himask) == (tau & himask)) atomicAdd(&hist[warp % NH][(kx >> lo) & dmask], 1u);
             }
             __syncthreads();
-            // bin totals, then suffix sums from the top bin down
-            uint32_t c = 0;
-            if (tid < 256) {
-#pragma unroll 8
-                for (int w = 0; w < NWP; ++w) c += hist[w][tid];
+            // thread t owns bins 2t and 2t+1; suffix sums from the top bin down
+            uint32_t c0 = 0, c1 = 0;
+#pragma unroll
+            for (int w = 0; w < NH; ++w) {
+                const uint2 v = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
+                c0 += v.x;
+                c1 += v.y;
             }
-            uint32_t suf = c;                        // inclusive suffix sum inside the warp
+            uint32_t suf = c0 + c1;                  // inclusive suffix sum over the threads of the warp
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t t = __shfl_down_sync(0xffffffffu, suf, off);
+                const uint32_t t = __shfl_down_sync(FULL, suf, off);
                 if (lane + off < 32) suf += t;
             }
-            if (tid < 256 && lane == 0) red[warp] = suf;   // warp totals (8 warps cover 256 bins)
+            if (lane == 0) red[warp] = suf;          // warp totals
             __syncthreads();
-            if (tid < 256) {
-                uint32_t above = 0;                  // keys in the warps that hold higher bins
-                for (int w = warp + 1; w < 8; ++w) above += red[w];
-                const uint32_t s_incl = suf + above; // keys in bins >= tid
-                const uint32_t s_excl = s_incl - c;  // keys in bins >  tid
-                if (s_incl >= (uint32_t)k_rem && s_excl < (uint32_t)k_rem) {
-                    s_digit = (uint32_t)tid;
-                    s_krem = (uint32_t)k_rem - s_excl;
-                }
+            const uint32_t wtot = red[lane];
+            uint32_t wsuf = wtot;                    // suffix sum over the warps, every warp on its own
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+                if (lane + off < 32) wsuf += t;
             }
+            const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+            const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
+            const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
+            const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
+            const uint32_t kr = (uint32_t)k_rem;
+            if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
+            if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
             __syncthreads();
             tau |= s_digit << lo;
             k_rem = (int)s_krem;
+            // every key of the chosen bin is wanted: the bin's lowest possible key is a valid
+            // threshold and the remaining digits need not be resolved
+            if (s_cnt == s_krem) break;
             hb = lo - 1;
         }
     }
 
-    // per-thread counts of "greater" (low half) and "equal" (high half)
-    uint32_t mine = 0;
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) mine += (key[j] > tau ? 1u : 0u) + (key[j] == tau ? 0x10000u : 0u);
-    uint32_t incl = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += t;
+    // rank of every taken page: ballots inside the warp, a scan over the warp totals across warps
+    const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp
+    const int base = warp * 32 * rows + lane;        // this lane's page in row 0
+    uint32_t wgt = 0, weq = 0;                       // this warp's counts of "greater" and "equal"
+#pragma unroll 1
+    for (int j = 0; j < rows; ++j) {
+        const int p = base + 32 * j;
+        const uint32_t kx = p < P ? skey[p] : 0u;    // 0 is below every key
+        wgt += __popc(__ballot_sync(FULL, kx > tau));
+        weq += __popc(__ballot_sync(FULL, kx == tau));
     }
-    if (lane == 31) red[warp] = incl;
     __syncthreads();
-    const uint32_t wv = red[lane];
-    uint32_t winc = wv;                              // inclusive scan of the warp totals
+    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
+    __syncthreads();
+    uint32_t g_inc = red[lane], e_inc = red2[lane];  // inclusive scans over the warps
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xffffffffu, winc, off);
-        if (lane >= off) winc += t;
+        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
+        if (lane >= off) { g_inc += tg; e_inc += te; }
     }
-    const uint32_t total = __shfl_sync(0xffffffffu, winc, 31);
-    const uint32_t before = __shfl_sync(0xffffffffu, winc - wv, warp);
-    const uint32_t excl = before + incl - mine;
-    const int n_gt = (int)(total & 0xffffu);
+    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
     const int r = K - n_gt;                          // how many equal keys to take
-    int gt_before = (int)(excl & 0xffffu), eq_before = (int)(excl >> 16);
-#pragma unroll
-    for (int j = 0; j < KPT; ++j) {
-        if (key[j] > tau) {
-            out[gt_before + min(eq_before, r)] = base + j;
-            ++gt_before;
-        } else if (key[j] == tau && key[j] != kKeyPad) {
-            if (eq_before < r) out[gt_before + eq_before] = base + j;
-            ++eq_before;
-        }
+    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
+    int eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll 1
+    for (int j = 0; j < rows; ++j) {
+        const int p = base + 32 * j;
+        const uint32_t kx = p < P ? skey[p] : 0u;
+        const bool is_gt = kx > tau, is_eq = kx == tau;
+        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
+        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
+        if (is_gt) out[gb + min(eb, r)] = p;
+        else if (is_eq && eb < r) out[gb + eb] = p;
+        gt_run += __popc(bg);
+        eq_run += __popc(be);
     }
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
@@ -183,18 +196,31 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     if (ns > P) ns = P;
     int nl = a.n_local < K - ns ? a.n_local : K - ns;
     if (nl > P - ns) nl = P - ns;
-    const int per = (P + kTopkThreads - 1) / kTopkThreads;
-#define CALL_TOPK(KPT) \
-    topk_kernel<KPT><<<BH, kTopkThreads, 0, s>>>(scores, a.page_cap, P, K, ns, nl, idx, idx_stride, budget, attend_ctr)
-    if (per <= 1) CALL_TOPK(1);
-    else if (per <= 2) CALL_TOPK(2);
-    else if (per <= 4) CALL_TOPK(4);
-    else if (per <= 8) CALL_TOPK(8);
-    else if (per <= 16) CALL_TOPK(16);
-    else if (per <= 32) CALL_TOPK(32);
-    else return cudaErrorInvalidValue;
-#undef CALL_TOPK
-    return cudaGetLastError();
+    if (P > kTopkThreads * kTopkMaxPerThread) return cudaErrorInvalidValue;
+    // the keys of a head live in dynamic shared memory: allow the largest head once per device
+    static bool ready[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!ready[dev]) {
+        e = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kTopkThreads * kTopkMaxPerThread * (int)sizeof(uint32_t));
+        if (e != cudaSuccess) return e;
+        ready[dev] = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)BH);
+    cfg.blockDim = dim3(kTopkThreads);
+    cfg.dynamicSmemBytes = (size_t)P * sizeof(uint32_t);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int64_t stride = a.page_cap;
+    return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr);
 }
 
 }  // namespace rq
