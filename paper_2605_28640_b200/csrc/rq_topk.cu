@@ -32,6 +32,13 @@ namespace {
 constexpr uint32_t kKeyForced = 0xffffffffu;   // above every score key
 constexpr int kDigitBits = 11;
 constexpr int kBins = 1 << kDigitBits;
+constexpr int kCandMax = 1024;                 // candidates ranked directly; a fuller bucket goes through the key bits
+
+// the score a key was made from (inverse of order_key)
+__device__ __forceinline__ float key_value(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
                                                             int P, int K, int n_sink, int n_local,
@@ -46,7 +53,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     extern __shared__ __align__(16) uint32_t skey[]; // [P] keys of the head
     __shared__ __align__(16) uint32_t hist[NH][kBins];   // read back as 8-byte pairs
     __shared__ uint32_t red[NWP], red2[NWP];
-    __shared__ uint32_t s_digit, s_krem, s_cnt;
+    __shared__ uint32_t s_digit, s_krem, s_cnt, s_ncand, s_tau;
+    __shared__ uint32_t cand[kCandMax];              // keys of the chosen bucket
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
     grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
@@ -80,66 +88,137 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     kmin = __reduce_min_sync(FULL, red[lane]);
     kmax = __reduce_max_sync(FULL, red2[lane]);
 
+    // One histogram pass over the non-forced keys for which `in(key)` holds: bins by `bin(key)`,
+    // walked from the top until k_rem keys are covered.  Leaves the chosen bin in s_digit, the
+    // rank wanted inside it in s_krem and its population in s_cnt.
+    auto select_bin = [&](auto in, auto bin) {
+        __syncthreads();                             // earlier readers of hist / red / s_* are done
+#pragma unroll 1
+        for (int i = tid; i < NH * kBins; i += NTH) (&hist[0][0])[i] = 0u;
+        __syncthreads();
+#pragma unroll 2
+        for (int p = tid; p < P; p += NTH) {
+            const uint32_t kx = skey[p];
+            if (kx != kKeyForced && in(kx)) atomicAdd(&hist[warp % NH][bin(kx)], 1u);
+        }
+        __syncthreads();
+        // thread t owns bins 2t and 2t+1; suffix sums from the top bin down
+        uint32_t c0 = 0, c1 = 0;
+#pragma unroll
+        for (int w = 0; w < NH; ++w) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
+            c0 += v.x;
+            c1 += v.y;
+        }
+        uint32_t suf = c0 + c1;                      // inclusive suffix sum over the threads of the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, suf, off);
+            if (lane + off < 32) suf += t;
+        }
+        if (lane == 0) red[warp] = suf;              // warp totals
+        __syncthreads();
+        const uint32_t wtot = red[lane];
+        uint32_t wsuf = wtot;                        // suffix sum over the warps, every warp on its own
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+            if (lane + off < 32) wsuf += t;
+        }
+        const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+        const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
+        const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
+        const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
+        const uint32_t kr = (uint32_t)k_rem;
+        if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
+        if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
+        __syncthreads();
+    };
+    // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
+    // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
+    auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
+        if (lo_key == hi_key) return lo_key;
+        int hb = 31 - __clz(lo_key ^ hi_key);        // highest bit in which the keys differ
+        uint32_t t = hb == 31 ? 0u : (hi_key >> (hb + 1)) << (hb + 1);   // shared leading bits
+#pragma unroll 1
+        while (hb >= 0) {
+            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
+            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
+            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
+            select_bin([&](uint32_t kx) { return in(kx) && (kx & himask) == (t & himask); },
+                       [&](uint32_t kx) { return (kx >> lo) & dmask; });
+            t |= s_digit << lo;
+            k_rem = (int)s_krem;
+            // every key of the chosen bin is wanted: the bin's lowest possible key is a valid
+            // threshold and the remaining digits need not be resolved
+            if (s_cnt == s_krem) break;
+            hb = lo - 1;
+        }
+        return t;
+    };
+
     uint32_t tau;                                    // k-th largest key among the non-forced pages
     if (k_rem <= 0) {
         tau = 0xfffffffeu + 1u;                      // nothing but forced pages fits: take none of the rest
     } else if (kmin == kmax) {
         tau = kmin;
     } else {
-        int hb = 31 - __clz(kmin ^ kmax);            // highest bit in which keys differ
-        tau = hb == 31 ? 0u : (kmax >> (hb + 1)) << (hb + 1);   // shared leading bits
-#pragma unroll 1
-        while (hb >= 0) {
-            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
-            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
-            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
-            __syncthreads();                         // the previous pass (and red/red2) has been read
-#pragma unroll 1
-            for (int i = tid; i < NH * kBins; i += NTH) (&hist[0][0])[i] = 0u;
+        // First pass on the score VALUES: 2048 equal-width buckets between the smallest and the
+        // largest score.  The map score -> bucket is monotone, so every key of a higher bucket is
+        // larger than every key of a lower one, and unlike a digit of the key bits the buckets
+        // resolve the bulk of the scores evenly whatever their sign and exponent.
+        const float v_lo = key_value(kmin);
+        const float scale = (float)(kBins - 1) / (key_value(kmax) - v_lo);
+        auto bucket = [&](uint32_t kx) -> uint32_t {
+            const float f = (key_value(kx) - v_lo) * scale;
+            return (uint32_t)min(max((int)f, 0), kBins - 1);
+        };
+        if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
+            tau = radix_select([](uint32_t) { return true; }, kmin, kmax);      // range too wide for a float
+        } else {
+            select_bin([](uint32_t) { return true; }, bucket);
+            const uint32_t b = s_digit, cnt = s_cnt;
+            k_rem = (int)s_krem;
+            // the candidates: keys of the chosen bucket, usually a handful
+            if (tid == 0) s_ncand = 0;
             __syncthreads();
+            uint32_t cmin = 0xffffffffu, cmax = 0u;
 #pragma unroll 2
             for (int p = tid; p < P; p += NTH) {
                 const uint32_t kx = skey[p];
-                if (kx != kKeyForced && (kx & himask) == (tau & himask)) atomicAdd(&hist[warp % NH][(kx >> lo) & dmask], 1u);
+                if (kx != kKeyForced && bucket(kx) == b) {
+                    cmin = min(cmin, kx);
+                    cmax = max(cmax, kx);
+                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = kx;
+                }
             }
             __syncthreads();
-            // thread t owns bins 2t and 2t+1; suffix sums from the top bin down
-            uint32_t c0 = 0, c1 = 0;
-#pragma unroll
-            for (int w = 0; w < NH; ++w) {
-                const uint2 v = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
-                c0 += v.x;
-                c1 += v.y;
+            if (cnt <= (uint32_t)kCandMax) {
+                // rank every candidate against all others; the wanted one has fewer than k_rem
+                // candidates above it and at least k_rem at or above it
+                if (tid < (int)cnt) {
+                    const uint32_t mine = cand[tid];
+                    uint32_t g = 0, ge = 0;
+#pragma unroll 4
+                    for (uint32_t j = 0; j < cnt; ++j) {
+                        const uint32_t o = cand[j];
+                        g += o > mine;
+                        ge += o >= mine;
+                    }
+                    if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) s_tau = mine;
+                }
+                __syncthreads();
+                tau = s_tau;
+            } else {
+                // an unusually full bucket (many equal scores): finish on the key bits
+                cmin = __reduce_min_sync(FULL, cmin);
+                cmax = __reduce_max_sync(FULL, cmax);
+                if (lane == 0) { red[warp] = cmin; red2[warp] = cmax; }
+                __syncthreads();
+                cmin = __reduce_min_sync(FULL, red[lane]);
+                cmax = __reduce_max_sync(FULL, red2[lane]);
+                tau = radix_select([&](uint32_t kx) { return bucket(kx) == b; }, cmin, cmax);
             }
-            uint32_t suf = c0 + c1;                  // inclusive suffix sum over the threads of the warp
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t t = __shfl_down_sync(FULL, suf, off);
-                if (lane + off < 32) suf += t;
-            }
-            if (lane == 0) red[warp] = suf;          // warp totals
-            __syncthreads();
-            const uint32_t wtot = red[lane];
-            uint32_t wsuf = wtot;                    // suffix sum over the warps, every warp on its own
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
-                if (lane + off < 32) wsuf += t;
-            }
-            const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
-            const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
-            const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
-            const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
-            const uint32_t kr = (uint32_t)k_rem;
-            if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
-            if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
-            __syncthreads();
-            tau |= s_digit << lo;
-            k_rem = (int)s_krem;
-            // every key of the chosen bin is wanted: the bin's lowest possible key is a valid
-            // threshold and the remaining digits need not be resolved
-            if (s_cnt == s_krem) break;
-            hb = lo - 1;
         }
     }
 
