@@ -48,6 +48,20 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     return w;
 }
 
+}  // namespace rq (reopened below)
+
+int rq::stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_cta, int max_ctas)
+{
+    int64_t g = units / (2 * warps_per_cta);
+    if (g > resident_ctas) g = resident_ctas;
+    if (g > max_ctas) g = max_ctas;
+    if (g >= heads && heads > 0) g -= g % heads;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+namespace rq {
+
 static int sm_count()
 {
     static int cached = 0;

@@ -484,7 +484,7 @@ cudaError_t launch_attend_t(const DecodeArgs &a, const void *q, const int32_t *i
     int occ = 1;
     cudaError_t e = attend_occupancy<T, D, S>(&occ);
     if (e != cudaSuccess) return e;
-    const int grid = attend_grid(W, occ * sm_count);
+    const int grid = attend_grid(W, a.B * a.H, occ * sm_count);
     const int slots = attend_slots_per_head(per_head);
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
@@ -503,14 +503,9 @@ cudaError_t launch_attend_t(const DecodeArgs &a, const void *q, const int32_t *i
 
 }  // namespace
 
-int attend_grid(int64_t tiles, int resident_ctas)
+int attend_grid(int64_t tiles, int heads, int resident_ctas)
 {
-    // every warp should get at least two tiles, every CTA at least one
-    int64_t g = tiles / (2 * kAttendWarps);
-    if (g > resident_ctas) g = resident_ctas;
-    if (g > kAttendMaxWarps / kAttendWarps) g = kAttendMaxWarps / kAttendWarps;
-    if (g < 1) g = 1;
-    return (int)g;
+    return stream_grid(tiles, heads, resident_ctas, kAttendWarps, kAttendMaxWarps / kAttendWarps);
 }
 
 int attend_slots_per_head(int64_t tiles_per_head)

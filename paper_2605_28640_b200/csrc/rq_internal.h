@@ -90,8 +90,12 @@ struct AttendCounters {
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
                           int idx_stride, float scale, float *partial, const AttendCounters &ctr, void *o,
                           int sm_count, cudaStream_t s);
+// Grid of a streaming kernel for a number of work units spread evenly over `heads` heads: at
+// most what the device holds at once, at least two units per warp, and, once there is a CTA per
+// head, a whole number of CTAs per head (heads served by more CTAs than others would finish early).
+int stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_cta, int max_ctas);
 // flash-decode grid for a number of tiles and the CTAs the device holds at once
-int attend_grid(int64_t tiles, int resident_ctas);
+int attend_grid(int64_t tiles, int heads, int resident_ctas);
 // partial records a head can need when it has this many tiles
 int attend_slots_per_head(int64_t tiles_per_head);
 

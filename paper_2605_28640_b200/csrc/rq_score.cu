@@ -359,9 +359,7 @@ cudaError_t launch_score_t(const DecodeArgs &a, const void *q, const void *k_t, 
     int occ = 1;
     cudaError_t e = score_occupancy<T, D>(&occ);
     if (e != cudaSuccess) return e;
-    int64_t grid = units / (2 * G::NW);              // every warp should get at least two units
-    if (grid > (int64_t)occ * sm_count) grid = (int64_t)occ * sm_count;
-    if (grid < 1) grid = 1;
+    const int grid = stream_grid(units, a.B * a.H, occ * sm_count, G::NW, INT_MAX);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(G::NW * 32);
