@@ -252,9 +252,9 @@ def main():
     meta_b, kv_b = step_bytes(w, w.T)
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
     ncopies = args.copies or max(2, min(8, -(-(4 * l2) // (meta_b + kv_b))))
-    # per copy: the timed loop, one more pass for the clock sampler, the profiled and e2e passes
+    # per copy: the timed loop, two more passes for the clock sampler, the profiled and e2e passes
     per_copy = -(-total_steps // ncopies)
-    cap = T0 + 4 * per_copy + 64
+    cap = T0 + 5 * per_copy + 128
     K = w.budget_pages(w.T)
     maxK = w.budget_pages(cap) + 1
 
@@ -300,11 +300,19 @@ def main():
         e1.record()
         barrier()
         ms = e0.elapsed_time(e1)
-        # keep the sampler running over a second identical pass so that short runs get samples
-        t_end = time.time() + 0.6
+        # keep the sampler running over more of the same work so that a short timed region still
+        # gets clock samples under load: decode steps while the caches have room, then the same
+        # selection and attention kernels without the append
+        t_end = time.time() + 1.5
         j = total_steps
-        while time.time() < t_end and j < 2 * total_steps:
-            step(j)
+        idx_keep = torch.empty(w.B, w.H, K, dtype=torch.int32, device=dev)
+        while time.time() < t_end:
+            if j < 3 * total_steps:
+                step(j)
+            else:
+                c = caches[j % ncopies].handle
+                rq.rq_select_pages(c, qs[j % pool], K, None, idx_keep)
+                rq.rq_attend_pages(c, qs[j % pool], idx_keep, K, 0.0, outs[j % 4])
             j += 1
             if j % 16 == 0:
                 torch.cuda.synchronize()
@@ -390,9 +398,10 @@ def main():
     if not args.no_cpu_baseline:
         nh = min(8, w.H)
         threads = min(os.cpu_count() or 1, nh)
-        reps = 60
-        smp = oracle_sample_for(w, dev, nh, threads, reps + 2, inputs=sample_inputs)
+        smp = oracle_sample_for(w, dev, nh, threads, 4096, inputs=sample_inputs)
         smp.step()
+        probe = sum(smp.step() for _ in range(3)) / 3
+        reps = int(max(10, min(4000, 12.0 / max(probe, 1e-6))))    # about 12 s of host work
         wall = sum(smp.step() for _ in range(reps))
         rounds_sample = -(-nh // threads)
         rounds_full = -(-(w.B * w.H) // threads)
