@@ -10,7 +10,8 @@ Levels (tolerances are the ones the benchmark definition states):
                  to a rounding boundary can differ); fp32 storage: the stored
                  value IS the fp32 state, so the state tolerance applies;
                  page bounds bit-exact against min/max of the device's own cache
-  3. selection : the oracle's scoring + top-k run on the DEVICE's bounds and q
+  3. selection : scores within 2e-6 of the sum of the products' magnitudes;
+                 the oracle's scoring + top-k run on the DEVICE's bounds and q
                  bits must give the same pages, except where the oracle flags a
                  near-tie (1e-5 relative) at the cut — those are counted
   4. attention : the oracle's attention over the device's pages and stored
@@ -113,8 +114,12 @@ def check_query_level(dev, hd, cache, b, h, q, K, scale, o, idx, scores, dtype, 
     if scores is not None:
         gU = f64(scores[b, h])
         assert gU.shape == U.shape
-        denom = np.maximum(np.abs(U), 1e-3 * np.sqrt(np.mean(U ** 2)) + 1e-30)
-        assert (np.abs(gU - U) / denom).max() <= 1e-5, f"scores[{b},{h}] off by {(np.abs(gU - U) / denom).max():.2e}"
+        # fp32 summation of the 2*D products (tree over the lanes, then sequential inside a lane):
+        # the error is bounded by about 13 * 2^-24 of the sum of the products' magnitudes, which
+        # is what matters when positive and negative terms cancel; allow 2e-6 of that sum
+        mag = np.maximum(np.abs(q64 * dev["min"]), np.abs(q64 * dev["max"])).sum(axis=1)
+        excess = np.abs(gU - U) - 2e-6 * mag
+        assert excess.max() <= 0, f"scores[{b},{h}] off by {np.abs(gU - U).max():.2e} (allowed {2e-6 * mag.max():.2e})"
     want, near = oracle.select_pages(U, K, n_sink, n_local)
     got = idx[b, h].cpu().numpy().astype(np.int64)
     n = len(want)
