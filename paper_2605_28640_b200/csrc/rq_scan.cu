@@ -48,8 +48,10 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cg = tid % NCG, sl = tid / NCG;
-    const int bh = blockIdx.y, b = bh / a.H, h = bh % a.H;
-    const int64_t chunk = chunk0 + blockIdx.x;
+    // heads vary fastest over the grid: CTAs that run together read neighbouring head rows of the
+    // same tokens, i.e. one contiguous stretch of the [B][T][H][D] inputs
+    const int bh = blockIdx.x, b = bh / a.H, h = bh % a.H;
+    const int64_t chunk = chunk0 + blockIdx.y;
     const int64_t pos0 = chunk * CT + (int64_t)sl * TS;
     const int64_t end = a.len0 + a.T;
 
@@ -133,7 +135,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
         }
     }
 
-    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + blockIdx.x) * 3 * D;
+    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + blockIdx.y) * 3 * D;
 
     if constexpr (MODE == 0) {
         // the chunk's map = (last warp's total) o (everything before the last warp)
@@ -300,7 +302,7 @@ cudaError_t run(const ScanArgs &a, cudaStream_t s)
     const int64_t nchunks = c1 - c0;
     if (nchunks <= 0) return cudaSuccess;
     if (nchunks > a.chunks_cap) return cudaErrorInvalidValue;
-    dim3 grid((unsigned)nchunks, (unsigned)(a.B * a.H));
+    dim3 grid((unsigned)(a.B * a.H), (unsigned)nchunks);
     scan_kernel<T, G, D, S, 0><<<grid, NT, 0, s>>>(a, c0);
     scan_carry_kernel<16><<<a.B * a.H, D, 0, s>>>(a.agg, a.state, D, nchunks, a.chunks_cap);
     scan_kernel<T, G, D, S, 1><<<grid, NT, 0, s>>>(a, c0);
