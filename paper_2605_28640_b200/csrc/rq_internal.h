@@ -44,7 +44,9 @@ struct WorkspaceLayout {
     size_t scores;    // float [BH][page_capacity]
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
-    size_t agg;       // float [BH][scan chunks][3][D]
+    size_t agg;       // float [BH][scan chunks][3][D] prefill chunk maps
+    size_t inc;       // float [BH][scan chunks][2][D] prefill chunk end states
+    size_t flags;     // int32 [BH][scan chunks] + ticket counter
     size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
     size_t total;
     int64_t scan_chunks_cap;
@@ -57,7 +59,12 @@ struct ScanArgs {
     const void *k, *v, *g;
     int64_t sb, st, sh;     // element strides of k, v, g
     void *kv, *meta;
-    float *state, *agg;
+    float *state;
+    float *agg;             // [BH][chunks_cap][3][D] chunk maps
+    float *inc;             // [BH][chunks_cap][2][D] state at the end of a chunk
+    int32_t *flags;         // [BH][chunks_cap] 0 = nothing, 1 = map published, 2 = end state published
+    int32_t *ticket;        // next (chunk, head) to hand out
+    int32_t *status;
     int B, H, D, S, dtype, gate_dtype;
     int64_t len0, T, page_cap, chunks_cap;
 };

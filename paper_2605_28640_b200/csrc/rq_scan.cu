@@ -1,6 +1,6 @@
-// Prefill: chunked parallel scan of the gated decay recurrence (Eq. 1) fused
-// with the paged cache write and the per-page min/max of the stored keys
-// (Appendix A.1, "Sparse inference settings").
+// Prefill: single-pass chained scan of the gated decay recurrence (Eq. 1)
+// fused with the paged cache write and the per-page min/max of the stored keys
+// (Appendix A.1, "Sparse inference settings").  Every input byte is read once.
 //
 // The recurrence x~_t = g_t x~_{t-1} + (1-g_t) x_t is a first-order linear
 // recurrence, so a run of tokens acts on the incoming state as the affine map
@@ -16,12 +16,22 @@
 // between the slices of a warp moves with warp shuffles; warps exchange their
 // totals through shared memory.
 //
-// Three launches: (0) every chunk's (A, Bk, Bv) -> workspace; (carry) a
-// sequential pass over the chunk maps per channel turns them into the state
-// entering each chunk; (1) every chunk re-reads its inputs and applies the
-// recurrence from the true incoming state, rounds to the storage type, writes
-// the pages and the page bounds, and the last token's owner leaves the fp32
-// state behind.
+// Chaining.  A CTA takes its (chunk, head) from a ticket counter, chunk-major
+// with the heads varying fastest, so every chunk before its own was taken
+// earlier by a CTA that is running or done, and CTAs that run together read
+// one contiguous stretch of the [B][T][H][D] inputs.  It loads its tokens,
+// reduces them to the chunk's map, publishes the map (flag 1), then looks back
+// over the records of the chunks before it, composing their maps until it
+// meets one that already knows the state at its own end (flag 2); that gives
+// the state entering the chunk.  Which chunks are composed is fixed by the
+// chunk's number (back to the last multiple of eight), not by timing, so the
+// result is the same bits on every run.  It publishes its own end state (flag 2)
+// before the heavy part, the token-by-token application with rounding, page
+// writes and page bounds, so later chunks never wait for that.  Waits on a
+// flag are bounded: when the limit runs out the kernel records
+// RQ_ERR_TIMEOUT in the status word and carries on with a zero carry instead
+// of spinning.
+#include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
 
@@ -30,9 +40,22 @@ namespace rq {
 namespace {
 
 constexpr int NT = kScanThreads;
+constexpr int kLookWindow = 8;                  // chunks examined per look-back round
+constexpr int kFlagPollLimit = 1 << 20;         // polls of one flag before giving up
 
-template <typename T, typename G, int D, int S, int MODE>
-__global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
+__device__ __forceinline__ int ld_acquire(const int32_t *p)
+{
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int32_t *p, int v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <typename T, typename G, int D, int S>
+__global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
 {
     constexpr int CH = VecOf<T>::N;
     constexpr int NCG = D / CH;
@@ -44,14 +67,19 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
     static_assert(NCG <= 32 && 32 % NCG == 0, "a warp must hold whole slices");
 
     __shared__ float wtot[NW][3][D];
-    __shared__ float mm[MODE == 1 ? NSL : 1][2][D];
+    __shared__ float mm[NSL][2][D];
+    __shared__ float sm_agg[3][D];               // the chunk's map
+    __shared__ float sm_in[2][D];                // state entering the chunk
+    __shared__ int sm_ticket;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cg = tid % NCG, sl = tid / NCG;
-    // heads vary fastest over the grid: CTAs that run together read neighbouring head rows of the
-    // same tokens, i.e. one contiguous stretch of the [B][T][H][D] inputs
-    const int bh = blockIdx.x, b = bh / a.H, h = bh % a.H;
-    const int64_t chunk = chunk0 + blockIdx.y;
+    const int BH = a.B * a.H;
+    if (tid == 0) sm_ticket = atomicAdd(a.ticket, 1);
+    __syncthreads();
+    const int rel = sm_ticket / BH;              // chunk number inside this call
+    const int bh = sm_ticket % BH, b = bh / a.H, h = bh % a.H;
+    const int64_t chunk = chunk0 + rel;
     const int64_t pos0 = chunk * CT + (int64_t)sl * TS;
     const int64_t end = a.len0 + a.T;
 
@@ -135,27 +163,101 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
         }
     }
 
-    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + blockIdx.y) * 3 * D;
+    // ---- the chunk's map = (last warp's total) o (everything before the last warp)
+    if (warp == NW - 1 && lane >= 32 - NCG) {
+#pragma unroll
+        for (int c = 0; c < CH; ++c) {
+            sm_agg[0][cg * CH + c] = A[c] * Ap[c];
+            sm_agg[1][cg * CH + c] = fmaf(A[c], Pk[c], Bk[c]);
+            sm_agg[2][cg * CH + c] = fmaf(A[c], Pv[c], Bv[c]);
+        }
+    }
+    __syncthreads();
 
-    if constexpr (MODE == 0) {
-        // the chunk's map = (last warp's total) o (everything before the last warp)
-        if (warp == NW - 1 && lane >= 32 - NCG) {
-            float oa[CH], ok[CH], ov[CH];
+    // ---- publish the map, find the state entering the chunk, publish the state leaving it
+    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + rel) * 3 * D;
+    float *inc = a.inc + ((int64_t)bh * a.chunks_cap + rel) * 2 * D;
+    int32_t *flags = a.flags + (int64_t)bh * a.chunks_cap;
+    if (tid < D) {
+        const int d = tid;
+        const float ca = sm_agg[0][d], cbk = sm_agg[1][d], cbv = sm_agg[2][d];
+        float in_k, in_v;
+        if (rel == 0) {
+            in_k = a.state[(int64_t)bh * 2 * D + d];
+            in_v = a.state[(int64_t)bh * 2 * D + D + d];
+        } else {
+            agg[d] = ca;
+            agg[D + d] = cbk;
+            agg[2 * D + d] = cbv;
+            __threadfence();
+        }
+        // the D publishing threads are whole warps: D is a multiple of 32
+        asm volatile("bar.sync 1, %0;" ::"n"(D));
+        if (rel != 0) {
+            if (d == 0) st_release(flags + rel, 1);
+            // Look back to the anchor: the last chunk before this one whose number is a multiple
+            // of kLookWindow.  The state entering this chunk is the anchor's end state pushed
+            // through the maps of the chunks in between, always in the same order, so the result
+            // does not depend on which chunk happened to finish first.
+            const int base = (rel - 1) / kLookWindow * kLookWindow;
+            const int n = rel - 1 - base;          // maps to compose: chunks base+1 .. rel-1
+            bool timed_out = false;
+            auto wait_for = [&](int idx, int need) {
+                int polls = 0;
+                while (ld_acquire(flags + idx) < need) {
+                    if (++polls > kFlagPollLimit) { timed_out = true; return; }
+                    __nanosleep(64);
+                }
+            };
 #pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                ok[c] = fmaf(A[c], Pk[c], Bk[c]);
-                ov[c] = fmaf(A[c], Pv[c], Bv[c]);
-                oa[c] = A[c] * Ap[c];
+            for (int u = 0; u < kLookWindow - 1; ++u)
+                if (u < n && !timed_out) wait_for(rel - 1 - u, 1);
+            __threadfence();
+            const float *pa = a.agg + ((int64_t)bh * a.chunks_cap + (rel - 1)) * 3 * D + d;
+            float ra[kLookWindow - 1], rbk[kLookWindow - 1], rbv[kLookWindow - 1];
+#pragma unroll
+            for (int u = 0; u < kLookWindow - 1; ++u) {
+                if (u < n && !timed_out) {
+                    ra[u] = __ldcg(pa - (int64_t)u * 3 * D);
+                    rbk[u] = __ldcg(pa - (int64_t)u * 3 * D + D);
+                    rbv[u] = __ldcg(pa - (int64_t)u * 3 * D + 2 * D);
+                }
             }
+            float acc_a = 1.0f, acc_k = 0.0f, acc_v = 0.0f;     // map of the chunks base+1 .. rel-1
 #pragma unroll
-            for (int c = 0; c < CH; c += 4) {
-                *reinterpret_cast<float4 *>(agg + 0 * D + cg * CH + c) = make_float4(oa[c], oa[c + 1], oa[c + 2], oa[c + 3]);
-                *reinterpret_cast<float4 *>(agg + 1 * D + cg * CH + c) = make_float4(ok[c], ok[c + 1], ok[c + 2], ok[c + 3]);
-                *reinterpret_cast<float4 *>(agg + 2 * D + cg * CH + c) = make_float4(ov[c], ov[c + 1], ov[c + 2], ov[c + 3]);
+            for (int u = 0; u < kLookWindow - 1; ++u) {
+                if (u < n && !timed_out) {           // acc = acc o map(rel-1-u): the older map acts first
+                    acc_k = fmaf(acc_a, rbk[u], acc_k);
+                    acc_v = fmaf(acc_a, rbv[u], acc_v);
+                    acc_a *= ra[u];
+                }
+            }
+            if (!timed_out) wait_for(base, 2);
+            __threadfence();
+            in_k = 0.0f;
+            in_v = 0.0f;
+            if (!timed_out) {
+                const float *pi = a.inc + ((int64_t)bh * a.chunks_cap + base) * 2 * D + d;
+                in_k = fmaf(acc_a, __ldcg(pi), acc_k);
+                in_v = fmaf(acc_a, __ldcg(pi + D), acc_v);
+            }
+            if (timed_out) {
+                atomicExch(a.status, RQ_ERR_TIMEOUT);
+                in_k = 0.0f;
+                in_v = 0.0f;
             }
         }
-        return;
-    } else {
+        inc[d] = fmaf(ca, in_k, cbk);
+        inc[D + d] = fmaf(ca, in_v, cbv);
+        __threadfence();
+        sm_in[0][d] = in_k;
+        sm_in[1][d] = in_v;
+        asm volatile("bar.sync 1, %0;" ::"n"(D));
+        if (d == 0) st_release(flags + rel, 2);
+    }
+    __syncthreads();
+
+    {
         // ---- exclusive map inside the warp = inclusive map of the previous slice
         float sk[CH], sv[CH];
 #pragma unroll
@@ -164,9 +266,9 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
             float ek = __shfl_up_sync(0xffffffffu, Bk[c], NCG % 32);
             float ev = __shfl_up_sync(0xffffffffu, Bv[c], NCG % 32);
             if (NCG == 32 || lane < NCG) { ea = 1.0f; ek = 0.0f; ev = 0.0f; }
-            // state entering the chunk (left by the carry pass in slots 1 and 2)
-            const float ck = agg[1 * D + cg * CH + c];
-            const float cv = agg[2 * D + cg * CH + c];
+            // state entering the chunk
+            const float ck = sm_in[0][cg * CH + c];
+            const float cv = sm_in[1][cg * CH + c];
             // entering this warp, then entering this slice
             const float wk = fmaf(Ap[c], ck, Pk[c]);
             const float wv = fmaf(Ap[c], cv, Pv[c]);
@@ -259,38 +361,6 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t chunk0)
     }
 }
 
-// Sequential composition of the chunk maps, one thread per (b, h, channel):
-// slot 1/2 of every chunk's record is overwritten with the state entering it.
-template <int BATCH>
-__global__ void scan_carry_kernel(float *agg, const float *state, int D, int64_t nchunks,
-                                  int64_t chunks_cap)
-{
-    const int bh = blockIdx.x, d = threadIdx.x;
-    if (d >= D) return;
-    float sk = state[(int64_t)bh * 2 * D + d];
-    float sv = state[(int64_t)bh * 2 * D + D + d];
-    float *base = agg + (int64_t)bh * chunks_cap * 3 * D + d;
-    for (int64_t c0 = 0; c0 < nchunks; c0 += BATCH) {
-        float A[BATCH], Bk[BATCH], Bv[BATCH];
-#pragma unroll
-        for (int j = 0; j < BATCH; ++j) {
-            if (c0 + j < nchunks) {
-                const float *r = base + (c0 + j) * 3 * D;
-                A[j] = r[0]; Bk[j] = r[D]; Bv[j] = r[2 * D];
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < BATCH; ++j) {
-            if (c0 + j < nchunks) {
-                float *r = base + (c0 + j) * 3 * D;
-                r[D] = sk; r[2 * D] = sv;
-                sk = fmaf(A[j], sk, Bk[j]);
-                sv = fmaf(A[j], sv, Bv[j]);
-            }
-        }
-    }
-}
-
 template <typename T, typename G, int D, int S>
 cudaError_t run(const ScanArgs &a, cudaStream_t s)
 {
@@ -302,10 +372,14 @@ cudaError_t run(const ScanArgs &a, cudaStream_t s)
     const int64_t nchunks = c1 - c0;
     if (nchunks <= 0) return cudaSuccess;
     if (nchunks > a.chunks_cap) return cudaErrorInvalidValue;
-    dim3 grid((unsigned)(a.B * a.H), (unsigned)nchunks);
-    scan_kernel<T, G, D, S, 0><<<grid, NT, 0, s>>>(a, c0);
-    scan_carry_kernel<16><<<a.B * a.H, D, 0, s>>>(a.agg, a.state, D, nchunks, a.chunks_cap);
-    scan_kernel<T, G, D, S, 1><<<grid, NT, 0, s>>>(a, c0);
+    const int64_t ctas = nchunks * a.B * a.H;
+    if (ctas >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    // the ticket counter and this call's flags start at zero
+    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(int32_t), s);
+    if (e != cudaSuccess) return e;
+    e = cudaMemsetAsync(a.flags, 0, (size_t)a.B * a.H * a.chunks_cap * sizeof(int32_t), s);
+    if (e != cudaSuccess) return e;
+    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, 0, s>>>(a, c0);
     return cudaGetLastError();
 }
 
