@@ -43,12 +43,6 @@ constexpr int NT = kScanThreads;
 constexpr int kLookWindow = 8;                  // chunks examined per look-back round
 constexpr int kFlagPollLimit = 1 << 20;         // polls of one flag before giving up
 
-__device__ __forceinline__ int ld_acquire(const int32_t *p)
-{
-    int v;
-    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
 __device__ __forceinline__ void st_release(int32_t *p, int v)
 {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -189,9 +183,9 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
             agg[d] = ca;
             agg[D + d] = cbk;
             agg[2 * D + d] = cbv;
-            __threadfence();
         }
-        // the D publishing threads are whole warps: D is a multiple of 32
+        // the D publishing threads are whole warps (D is a multiple of 32); the barrier orders their
+        // stores before thread 0's release store of the flag
         asm volatile("bar.sync 1, %0;" ::"n"(D));
         if (rel != 0) {
             if (d == 0) st_release(flags + rel, 1);
@@ -202,16 +196,21 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
             const int base = (rel - 1) / kLookWindow * kLookWindow;
             const int n = rel - 1 - base;          // maps to compose: chunks base+1 .. rel-1
             bool timed_out = false;
-            auto wait_for = [&](int idx, int need) {
-                int polls = 0;
-                while (ld_acquire(flags + idx) < need) {
-                    if (++polls > kFlagPollLimit) { timed_out = true; return; }
-                    __nanosleep(64);
-                }
-            };
+            // all flags are read together (relaxed loads, one round trip), then only the ones that
+            // are not there yet are polled; the fence after the loop makes the reads acquire
+            int f[kLookWindow];                    // f[u], u < n: chunk rel-1-u; f[n]: the anchor
 #pragma unroll
-            for (int u = 0; u < kLookWindow - 1; ++u)
-                if (u < n && !timed_out) wait_for(rel - 1 - u, 1);
+            for (int u = 0; u < kLookWindow; ++u) f[u] = u <= n ? ld_volatile(flags + (rel - 1 - u)) : 2;
+#pragma unroll
+            for (int u = 0; u < kLookWindow; ++u) {
+                const int need = u == n ? 2 : 1;
+                int polls = 0;
+                while (u <= n && f[u] < need && !timed_out) {
+                    if (++polls > kFlagPollLimit) timed_out = true;
+                    __nanosleep(32);
+                    f[u] = ld_volatile(flags + (rel - 1 - u));
+                }
+            }
             __threadfence();
             const float *pa = a.agg + ((int64_t)bh * a.chunks_cap + (rel - 1)) * 3 * D + d;
             float ra[kLookWindow - 1], rbk[kLookWindow - 1], rbv[kLookWindow - 1];
@@ -232,8 +231,6 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
                     acc_a *= ra[u];
                 }
             }
-            if (!timed_out) wait_for(base, 2);
-            __threadfence();
             in_k = 0.0f;
             in_v = 0.0f;
             if (!timed_out) {
@@ -249,7 +246,6 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
         }
         inc[d] = fmaf(ca, in_k, cbk);
         inc[D + d] = fmaf(ca, in_v, cbv);
-        __threadfence();
         sm_in[0][d] = in_k;
         sm_in[1][d] = in_v;
         asm volatile("bar.sync 1, %0;" ::"n"(D));
