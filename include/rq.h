@@ -194,6 +194,38 @@ RQ_API int rq_select_pages(rq_cache *cache, const void *q, int32_t budget_pages,
 RQ_API int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t n_idx,
                     float scale, void *o, void *stream);
 
+/* The paper has no counterpart to this entry point; it exists for one kind of caller.
+ *
+ * rq_attend_pages for callers that are not allowed to allocate device memory and therefore
+ * have no workspace to hand over: a plug-in inside a serving engine that owns every byte of
+ * the GPU, code on a latency path where cudaMalloc is banned because it synchronises the
+ * device, a process whose memory pool is already carved up.  Such a caller passes only the
+ * inputs (the paged cache it already holds, the query, the page list) and the output; the
+ * partial results and counters of the kernel live in a fixed 4 MiB array that is part of the
+ * library's image on every GPU that loads it, until the process exits.
+ *   cfg      : the configuration the cache was built with (host memory)
+ *   kv       : the paged cache, layout as above (device)
+ *   len      : tokens in every sequence, 1 .. cfg->capacity_tokens
+ *   q, o     : [B][H][D] of cfg->dtype (device);  idx : int32 [B][H][n_idx] as in rq_attend_pages,
+ *              except that an entry >= P is skipped without being reported
+ *   scale    : softmax scale; <= 0 selects 1/sqrt(D)
+ * Limit: 256 + B*H*256 + B*H*r*(D+4)*4 bytes must fit in the 4 MiB, where r is the number of
+ * partial records per head (CTAs per head, about 2 * SMs / (B*H), when B*H is at most the
+ * number of resident CTAs; otherwise up to 4 per CTA); the headline shape (B*H = 32, D = 128)
+ * needs 0.16 MiB.  A shape beyond the limit is refused with RQ_ERR_CAPACITY before anything is
+ * enqueued.  The call allocates nothing and calls no allocating routine; it enqueues one small
+ * memset (status and counters must start at zero: the array keeps what the last call left) and
+ * one kernel on `stream` and returns without synchronising.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and
+ * sets a kernel attribute; make that first call outside any stream capture.
+ * All calls share the one array: two calls whose kernels overlap on the GPU (different streams,
+ * or different host threads) race on it and give wrong results; calls on one stream are safe.
+ * Errors: as rq_sizes for cfg; INVALID_ARG (NULL pointer, n_idx < 1, len out of range);
+ * CAPACITY (shape beyond the limit); CUDA. */
+RQ_API int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int64_t len, const void *q,
+                                   const int32_t *idx, int32_t n_idx, float scale, void *o,
+                                   void *stream);
+
 /* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
 RQ_API int64_t rq_cache_len(const rq_cache *cache);
 

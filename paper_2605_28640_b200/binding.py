@@ -47,6 +47,7 @@ SIGNATURES = {
     "rq_profile_slot_name": (C.c_char_p, [C.c_int]),
     "rq_select_pages": (C.c_int, [_cachep, _vp, _i32, _vp, _vp, _vp]),
     "rq_attend_pages": (C.c_int, [_cachep, _vp, _vp, _i32, _f, _vp, _vp]),
+    "rq_attend_pages_noalloc": (C.c_int, [_cfgp, _vp, _i64, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
     "rq_device_status": (C.c_int, [_cachep, C.POINTER(C.c_int32), _vp]),
     "rq_status_string": (C.c_char_p, [C.c_int]),
@@ -153,6 +154,13 @@ def rq_select_pages(cache: rq_cache, q, budget_pages, scores_out, idx_out, strea
 def rq_attend_pages(cache: rq_cache, q, idx, n_idx, scale, o, stream=None):
     _check(lib().rq_attend_pages(C.byref(cache), _ptr(q), _ptr(idx), n_idx, scale, _ptr(o),
                                  _stream(stream)), "rq_attend_pages")
+
+
+def rq_attend_pages_noalloc(cfg: rq_config, kv, length, q, idx, n_idx, scale, o, stream=None):
+    """rq_attend_pages without a workspace, for callers that may not allocate device memory: the
+    kernel's scratch is a fixed array inside the library (shapes beyond its 4 MiB are refused)."""
+    _check(lib().rq_attend_pages_noalloc(C.byref(cfg), _ptr(kv), length, _ptr(q), _ptr(idx), n_idx, scale,
+                                         _ptr(o), _stream(stream)), "rq_attend_pages_noalloc")
 
 
 def rq_cache_len(cache: rq_cache) -> int:

@@ -33,7 +33,10 @@
 // memory into one partial (m, l, acc[D]) per head; the arrival that completes
 // a head's count combines the head's partials into the output row.
 #include <limits.h>
+#include <math.h>
 #include <math_constants.h>
+
+#include <algorithm>
 
 #include "rq_async.cuh"
 #include "rq_device.cuh"
@@ -501,6 +504,47 @@ cudaError_t launch_attend_t(const DecodeArgs &a, const void *q, const int32_t *i
                               partial, slots, ctr, (T *)o);
 }
 
+// the same launch with the number of partial records per head given by the caller
+template <typename T, int D, int S>
+cudaError_t launch_attend_slots_t(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx, int idx_stride,
+                                  float scale, float *partial, int slots, const AttendCounters &ctr, void *o,
+                                  int sm_count, cudaStream_t s)
+{
+    using G = AttendGeom<T, D, S>;
+    const int64_t W = (int64_t)a.B * a.H * n_idx * G::TPP;
+    int occ = 1;
+    cudaError_t e = attend_occupancy<T, D, S>(&occ);
+    if (e != cudaSuccess) return e;
+    const int grid = attend_grid(W, a.B * a.H, occ * sm_count);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(G::NW * 32);
+    cfg.dynamicSmemBytes = G::SMEM_BYTES;
+    cfg.stream = s;
+    return cudaLaunchKernelEx(&cfg, attend_kernel<T, D, S>, a, (const T *)q, idx, n_idx, idx_stride,
+                              scale * 1.4426950408889634f, partial, slots, ctr, (T *)o);
+}
+
+cudaError_t launch_attend_slots(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx, int idx_stride,
+                                float scale, float *partial, int slots, const AttendCounters &ctr, void *o,
+                                int sm_count, cudaStream_t s)
+{
+#define RQ_ATT(T, D, S) return launch_attend_slots_t<T, D, S>(a, q, idx, n_idx, idx_stride, scale, partial, slots, ctr, o, sm_count, s)
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128 && a.S == 16) RQ_ATT(bf16, 128, 16);
+        if (a.D == 128 && a.S == 64) RQ_ATT(bf16, 128, 64);
+        if (a.D == 64 && a.S == 16) RQ_ATT(bf16, 64, 16);
+        if (a.D == 64 && a.S == 64) RQ_ATT(bf16, 64, 64);
+    } else {
+        if (a.D == 128 && a.S == 16) RQ_ATT(float, 128, 16);
+        if (a.D == 128 && a.S == 64) RQ_ATT(float, 128, 64);
+        if (a.D == 64 && a.S == 16) RQ_ATT(float, 64, 16);
+        if (a.D == 64 && a.S == 64) RQ_ATT(float, 64, 64);
+    }
+#undef RQ_ATT
+    return cudaErrorInvalidValue;
+}
+
 }  // namespace
 
 int attend_grid(int64_t tiles, int heads, int resident_ctas)
@@ -535,4 +579,93 @@ cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx
     return cudaErrorInvalidValue;
 }
 
+// ---------------------------------------------------------------- attention without a workspace
+// Scratch of rq_attend_pages_noalloc: lives in the library's image, so every GPU that loads the
+// library holds these 4 MiB until the process exits.  Layout: status word (256 bytes), then the
+// per-head counters, then the partial records.
+constexpr size_t kStaticScratchBytes = (size_t)4 << 20;
+static __device__ __align__(256) unsigned char g_attend_scratch[kStaticScratchBytes];
+
+// Device address of the scratch array on the current device (the array's name is only a handle in
+// host code).  Looked up once per device.
+static cudaError_t static_scratch(unsigned char **out)
+{
+    static unsigned char *cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!cached[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_attend_scratch);
+        if (e != cudaSuccess) return e;
+        cached[dev] = static_cast<unsigned char *>(p);
+    }
+    *out = cached[dev];
+    return cudaSuccess;
+}
+
 }  // namespace rq
+
+extern "C" int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int64_t len, const void *q,
+                                       const int32_t *idx, int32_t n_idx, float scale, void *o, void *stream)
+{
+    using namespace rq;
+    const int rc = rq_sizes(cfg, nullptr, nullptr, nullptr, nullptr);      // validates the configuration
+    if (rc != RQ_OK) return rc;
+    if (!kv || !q || !idx || !o || n_idx < 1 || len < 1 || len > cfg->capacity_tokens) return RQ_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int BH = cfg->batch * cfg->heads;
+    const int tpp = cfg->page_size / kTileRows;
+    const int64_t per_head = (int64_t)n_idx * tpp;
+    if (per_head > kDoneTileMask) return RQ_ERR_CAPACITY;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return RQ_ERR_CUDA;
+
+    DecodeArgs a = {};
+    a.kv = const_cast<void *>(kv);
+    a.B = cfg->batch; a.H = cfg->heads; a.D = cfg->head_dim; a.S = cfg->page_size;
+    a.dtype = cfg->dtype; a.gate_dtype = cfg->gate_dtype;
+    a.len = len;
+    a.page_cap = (cfg->capacity_tokens + cfg->page_size - 1) / cfg->page_size;
+
+    // The grid and the number of partial records per head follow from the shape alone; the
+    // ordinary entry point sizes its workspace for the worst case, here the exact need counts.
+    int occ = 1;
+    cudaError_t e = cudaErrorInvalidValue;
+#define RQ_OCC(T, D, S) e = attend_occupancy<T, D, S>(&occ)
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128 && a.S == 16) RQ_OCC(bf16, 128, 16);
+        else if (a.D == 128 && a.S == 64) RQ_OCC(bf16, 128, 64);
+        else if (a.D == 64 && a.S == 16) RQ_OCC(bf16, 64, 16);
+        else if (a.D == 64 && a.S == 64) RQ_OCC(bf16, 64, 64);
+    } else {
+        if (a.D == 128 && a.S == 16) RQ_OCC(float, 128, 16);
+        else if (a.D == 128 && a.S == 64) RQ_OCC(float, 128, 64);
+        else if (a.D == 64 && a.S == 16) RQ_OCC(float, 64, 16);
+        else if (a.D == 64 && a.S == 64) RQ_OCC(float, 64, 64);
+    }
+#undef RQ_OCC
+    if (e != cudaSuccess) return RQ_ERR_CUDA;
+    const int grid = attend_grid((int64_t)BH * per_head, BH, occ * sms);
+    const int64_t slots = grid >= BH ? grid / BH : std::min<int64_t>((int64_t)grid * kAttendWarps, per_head);
+    const size_t ctr_bytes = (size_t)BH * kCtrStride * sizeof(int32_t);
+    const size_t need = 256 + ctr_bytes + (size_t)BH * slots * (a.D + 4) * sizeof(float);
+    if (need > kStaticScratchBytes) return RQ_ERR_CAPACITY;
+
+    unsigned char *scratch = nullptr;
+    if (static_scratch(&scratch) != cudaSuccess) return RQ_ERR_CUDA;
+    // the array keeps what the last call left: status and counters must start at zero
+    if (cudaMemsetAsync(scratch, 0, 256 + ctr_bytes, s) != cudaSuccess) return RQ_ERR_CUDA;
+    a.status = reinterpret_cast<int32_t *>(scratch);
+    int32_t *ctr = reinterpret_cast<int32_t *>(scratch + 256);
+    float *partial = reinterpret_cast<float *>(scratch + 256 + ctr_bytes);
+    if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
+    const AttendCounters c = {ctr, ctr + 1, ctr + 2};
+    if (launch_attend_slots(a, q, idx, n_idx, n_idx, scale, partial, (int)slots, c, o, sms, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    return RQ_OK;
+}
