@@ -62,7 +62,7 @@ struct AttendGeom {
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
     static constexpr int NW = kAttendWarps;
     static constexpr int DEPTH_RAW = kAttendRingBytes / (NW * STAGE_BYTES);
-    static constexpr int DEPTH = DEPTH_RAW < 2 ? 2 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
+    static constexpr int DEPTH = DEPTH_RAW < 1 ? 1 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
     static constexpr int RING_BYTES = NW * DEPTH * STAGE_BYTES;
     // ring | barriers | (head, valid rows) per stage | per-warp m, l, tiles, head | per-warp acc
     static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 8 + 4 * NW * 4 + NW * D * 4;

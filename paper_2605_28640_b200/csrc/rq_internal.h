@@ -28,9 +28,9 @@ inline int scan_chunk_tokens(int head_dim, int dtype)
 
 // ---- decode-side geometry ----
 constexpr int kScoreWarps = 4;         // warps per scoring CTA, each with its own copy pipeline
-constexpr int kScoreRingBytes = 96 * 1024;   // shared-memory ring of one scoring CTA (all warps)
+constexpr int kScoreRingBytes = 64 * 1024;   // shared-memory ring of one scoring CTA (all warps): three CTAs per SM
 constexpr int kAttendWarps = 4;        // warps per flash-decode CTA, each with its own copy pipeline
-constexpr int kAttendRingBytes = 96 * 1024;  // shared-memory ring of one flash-decode CTA (all warps)
+constexpr int kAttendRingBytes = 64 * 1024;  // shared-memory ring of one flash-decode CTA (all warps): three CTAs per SM
 constexpr int kAttendMaxWarps = 1536;  // upper bound of the warps of a flash-decode grid
 constexpr int kCtrStride = 64;         // int32 between the counters of two heads (256 bytes: different L2 lines)
 constexpr int kTopkThreads = 1024;     // threads of the selection CTA

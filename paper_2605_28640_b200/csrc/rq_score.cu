@@ -49,7 +49,7 @@ struct ScoreGeom {
     static constexpr int NR = RU / PPW;              // record groups per unit
     static constexpr int NW = kScoreWarps;
     static constexpr int DEPTH_RAW = kScoreRingBytes / (NW * kUnitBytes);
-    static constexpr int DEPTH = DEPTH_RAW < 2 ? 2 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
+    static constexpr int DEPTH = DEPTH_RAW < 1 ? 1 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
     static constexpr int RING_BYTES = NW * DEPTH * kUnitBytes;
     // ring | barriers | (head, first record, records) per stage | reduction scratch of the update
     static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 16 + 64;
