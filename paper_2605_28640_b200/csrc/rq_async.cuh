@@ -37,7 +37,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
 // Poll limit of a barrier wait.  One poll may itself suspend the thread for a
 // hardware-defined short time, so the limit is reached only after a time that
 // is orders of magnitude beyond any copy's latency.
-constexpr int kMbarPollLimit = 1 << 22;
+constexpr int kMbarPollLimit = 1 << 20;
+// upper bound (ns) of the time one poll may keep the thread suspended while the phase is pending
+constexpr uint32_t kMbarSuspendNs = 2000;
 
 // Wait for the phase with the given parity to complete.  Returns false if the
 // poll limit ran out first.
@@ -48,10 +50,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kMbarSuspendNs)
             : "memory");
         if (done) return true;
     }

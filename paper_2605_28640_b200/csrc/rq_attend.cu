@@ -60,6 +60,8 @@ struct AttendGeom {
     static constexpr int NI = TR / RPI;            // warp-wide reads per tile and tensor
     static constexpr int TILE_BYTES = TR * D * (int)sizeof(T);
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
+    static constexpr int SH = (LPR == 32 ? 5 : LPR == 16 ? 4 : LPR == 8 ? 3 : 2) - (NI == 16 ? 4 : NI == 8 ? 3 : NI == 4 ? 2 : 1);   // log2(LPR / NI)
+    static_assert(SH >= 0 && (NI << SH) == LPR, "a row's score must end up in at least one lane");
     static constexpr int NW = kAttendWarps;
     static constexpr int DEPTH_RAW = kAttendRingBytes / (NW * STAGE_BYTES);
     static constexpr int DEPTH = DEPTH_RAW < 1 ? 1 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
@@ -296,11 +298,15 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     uint32_t phase = 0;                              // one parity bit per stage
     bool dead = false;                               // a wait ran out: stop streaming, finish cleanly
 
-    // sum the row groups of the warp (they share m_run); lanes < LPR end up with the channel sums
+    // sum the warp's softmax denominators and the row groups' accumulators (all share m_run);
+    // lanes < LPR end up with the channel sums
     auto merge_rows = [&]() {
+        // every row's weight was added by the 2^SH lanes that hold the row: sum over the warp
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) l_run += __shfl_xor_sync(FULL, l_run, off);
+        l_run *= 1.0f / (float)(1 << G::SH);
 #pragma unroll
         for (int off = LPR; off < 32; off <<= 1) {
-            l_run += __shfl_xor_sync(FULL, l_run, off);
 #pragma unroll
             for (int c = 0; c < CH; ++c) acc[c] += __shfl_xor_sync(FULL, acc[c], off);
         }
@@ -369,8 +375,10 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
         if (valid > 0 && !dead) {
             const T *ks = reinterpret_cast<const T *>(myring + (size_t)stage * G::STAGE_BYTES);
             const T *vs = ks + TR * D;
+            // K: partial dot products of NI row groups, then a reduction over the LPR lanes of a
+            // row in which every step also halves the values a lane carries: afterwards a lane
+            // holds the complete score of ONE row (row group cgp >> SH, shared by 2^SH lanes)
             float s[NI];
-            float m_new = m_run;
 #pragma unroll
             for (int n = 0; n < NI; ++n) {
                 float kf[CH];
@@ -378,23 +386,42 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
                 float d = 0.0f;
 #pragma unroll
                 for (int c = 0; c < CH; ++c) d = fmaf(qf[c], kf[c], d);
-#pragma unroll
-                for (int off = LPR / 2; off > 0; off >>= 1) d += __shfl_xor_sync(FULL, d, off);
-                const int row = n * RPI + rsub;
-                s[n] = row < valid ? d : -CUDART_INF_F;
-                m_new = fmaxf(m_new, s[n]);
+                s[n] = d;
             }
+            int nv = NI;
 #pragma unroll
-            for (int off = LPR; off < 32; off <<= 1) m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, off));
+            for (int off = LPR / 2; off > 0; off >>= 1) {
+                if (nv > 1) {
+                    const int half = nv / 2;
+                    const bool hi = (lane & off) != 0;
+#pragma unroll
+                    for (int i = 0; i < NI / 2; ++i) {
+                        if (i < half) {
+                            const float send = hi ? s[i] : s[i + half];
+                            const float keep = hi ? s[i + half] : s[i];
+                            s[i] = keep + __shfl_xor_sync(FULL, send, off);
+                        }
+                    }
+                    nv = half;
+                } else {
+                    s[0] += __shfl_xor_sync(FULL, s[0], off);
+                }
+            }
+            const int row = ((cgp >> G::SH) & (NI - 1)) * RPI + rsub;
+            const float sc = row < valid ? s[0] : -CUDART_INF_F;
+            float m_new = fmaxf(m_run, sc);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, off));
             const float alpha = exp2f(m_run - m_new);    // 0 on the first tile (m_run = -inf)
+            const float p_row = exp2f(sc - m_new);       // 0 for a masked row
             m_run = m_new;
-            l_run *= alpha;
+            l_run = fmaf(l_run, alpha, p_row);           // per lane; 2^SH lanes repeat a row
 #pragma unroll
             for (int c = 0; c < CH; ++c) acc[c] *= alpha;
+            // V: row group n's weight comes from the lane that holds it
 #pragma unroll
             for (int n = 0; n < NI; ++n) {
-                const float p = exp2f(s[n] - m_new);     // 0 for masked rows
-                l_run += p;
+                const float p = __shfl_sync(FULL, p_row, rsub * LPR + (n << G::SH));
                 float vf[CH];
                 unpack16<T>(lds16(vs + (n * 32 + lane) * CH), vf);
 #pragma unroll
