@@ -74,7 +74,7 @@ struct AttendGeom {
 
 // Combine n partials of a head (one warp): o = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s.
 // Lane -> (channel group g = lane % 8 of D/8 channels, subset j = lane / 8): a lane sweeps the
-// partials s = j, j+4, ... with a running maximum, three records per round trip (their loads are
+// partials s = j, j+4, ... with a running maximum, four records per round trip (their loads are
 // all issued before the first is used); the four subsets are merged with two shuffle steps.
 // A record is [m, l, -, -, acc[D]]; an empty one has m = -inf and zeros.
 template <typename T, int D>
@@ -82,7 +82,7 @@ __device__ __forceinline__ void combine_head(const float *src, int n, T *o_row, 
 {
     constexpr int CPL = D / 8;                     // channels per lane
     constexpr int NV = CPL / 4;                    // 16-byte vectors per lane and record
-    constexpr int U = 3;                           // records in flight per lane
+    constexpr int U = 4;                           // records in flight per lane
     const int g = lane & 7, j = lane >> 3;
     float M = -CUDART_INF_F, L = 0.0f, A[CPL];
 #pragma unroll
@@ -313,16 +313,22 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     };
     // after a partial of head h has been written by this warp: count it, and combine if it was the last
     auto arrive = [&](int h, int count_word, int expect_ctas, int n_fixed) {
-        __threadfence();
+        // The partial was written by several lanes: the warp barrier orders those stores before
+        // lane 0's release; the same atomic acquires the partials of the arrivals before it.
         __syncwarp();
         int last = 0;
         if (lane == 0) {
-            const int now = atomicAdd(ctr.done + h * kCtrStride, count_word) + count_word;
+            int old;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;"
+                         : "=r"(old)
+                         : "l"(ctr.done + h * kCtrStride), "r"(count_word)
+                         : "memory");
+            const int now = old + count_word;
             last = (now & kDoneTileMask) == per_head && (now >> kDoneTileBits) == expect_ctas;
         }
         last = __shfl_sync(FULL, last, 0);
         if (last) {
-            __threadfence();
+            __syncwarp();
             const int n = n_fixed >= 0 ? n_fixed : min(ld_volatile(ctr.nslot + h * kCtrStride), slots_per_head);
             combine_head<T, D>(partial + (int64_t)h * slots_per_head * (D + 4), n, o + (int64_t)h * D, lane);
         }
