@@ -36,9 +36,11 @@ if ROOT not in sys.path:
 METRIC = "sparse decode us/step at 128K ctx, 1/16 budget"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu
-# captures (profiles/): kernel -> bytes for the default workload, or None.
-NCU_TRAFFIC = {"score": None, "attend": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
+# (profiles/*_kernel_64k_b1.md: 64 MiB launches, scaled by two to the 128 MiB launches of the
+# default workload, traffic being proportional to the pages processed): kernel -> bytes, or None
+# when the kernel has changed since the capture.
+NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.40e6), "attend": 2 * (67.24e6 + 0.93e6)}
 
 
 def measured_peak():
