@@ -151,11 +151,12 @@ RQ_API int rq_decode_step(rq_cache *cache, const void *q, const void *k_t, const
                    const void *g_t, int32_t budget_pages, float scale, void *o,
                    int32_t *sel_idx_out, void *stream);
 
-/* The same step for callers whose tensors live in HOST memory (pinned memory
- * makes the copies asynchronous): q, k_t, v_t, g_t are copied to the device,
- * the step runs, o (and sel_idx_out if not NULL) are copied back to host
- * memory, all on `stream`.  The outputs are valid after the stream is
- * synchronised.  Bytes moved per call: 4 inputs + 1 output of B*H*D elements
+/* The same step for callers whose tensors live in HOST memory: q, k_t, v_t, g_t are brought
+ * to the device, the step runs, o (and sel_idx_out if not NULL) are copied back to host
+ * memory, all on `stream`.  Pinned (page-locked or registered), 16-byte aligned inputs are read
+ * by one small gather kernel straight from host memory; other inputs go through four
+ * asynchronous copies (synchronous for pageable memory, as usual).  The outputs are valid after
+ * the stream is synchronised.  Bytes moved per call: 4 inputs + 1 output of B*H*D elements
  * (+ the index list). */
 RQ_API int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_host,
                         const void *v_t_host, const void *g_t_host,

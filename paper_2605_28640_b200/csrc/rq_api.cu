@@ -158,6 +158,34 @@ static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, con
     return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s, ev);
 }
 
+// Gather of the four per-step input tensors from pinned host memory (read over the bus by the
+// device) into the staging area: nv 16-byte vectors each for q, k_t, v_t and ng for g_t.
+__global__ void stage_in_kernel(const uint4 *q, const uint4 *k, const uint4 *v, const uint4 *g, uint4 *dq,
+                                uint4 *dk, uint4 *dv, uint4 *dg, int nv, int ng)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nv) { dq[i] = q[i]; return; }
+    i -= nv;
+    if (i < nv) { dk[i] = k[i]; return; }
+    i -= nv;
+    if (i < nv) { dv[i] = v[i]; return; }
+    i -= nv;
+    if (i < ng) dg[i] = g[i];
+}
+
+// Device address of a host buffer if it is pinned (or registered) and 16-byte aligned.
+static bool device_view(const void *host, const void **dev)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer || ((uintptr_t)at.devicePointer & 15)) return false;
+    *dev = at.devicePointer;
+    return true;
+}
+
 }  // namespace rq
 
 using namespace rq;
@@ -301,11 +329,25 @@ int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_hos
     char *stg = (char *)cache->workspace + w.staging;
     void *dq = stg, *dk = stg + slot, *dv = stg + 2 * slot, *dg = stg + 3 * slot, *dout = stg + 4 * slot;
     const size_t eb = n * elem_size(c.dtype), gb = n * elem_size(c.gate_dtype);
-    if (cudaMemcpyAsync(dq, q_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dk, k_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dv, v_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dg, g_t_host, gb, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    // Pinned host buffers are readable from the device: one small kernel gathers all four into
+    // the staging area (one launch instead of four copies).  Anything else goes through copies.
+    const void *src[4] = {q_host, k_t_host, v_t_host, g_t_host};
+    const void *dsrc[4];
+    bool direct = true;
+    for (int i = 0; i < 4 && direct; ++i) direct = device_view(src[i], &dsrc[i]);
+    if (direct) {
+        const int nv = (int)(eb / 16), ng = (int)(gb / 16);
+        const int total = 3 * nv + ng;
+        stage_in_kernel<<<(total + 255) / 256, 256, 0, s>>>((const uint4 *)dsrc[0], (const uint4 *)dsrc[1],
+                                                           (const uint4 *)dsrc[2], (const uint4 *)dsrc[3],
+                                                           (uint4 *)dq, (uint4 *)dk, (uint4 *)dv, (uint4 *)dg, nv, ng);
+        if (cudaGetLastError() != cudaSuccess) return RQ_ERR_CUDA;
+    } else if (cudaMemcpyAsync(dq, q_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+               cudaMemcpyAsync(dk, k_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+               cudaMemcpyAsync(dv, v_t_host, eb, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+               cudaMemcpyAsync(dg, g_t_host, gb, cudaMemcpyHostToDevice, s) != cudaSuccess) {
         return RQ_ERR_CUDA;
+    }
     int32_t *sel = (int32_t *)((char *)cache->workspace + w.sel);
     const int st = rq_decode_step(cache, dq, dk, dv, dg, budget_pages, scale, dout,
                                   sel_idx_out_host ? sel : nullptr, stream);

@@ -248,13 +248,14 @@ def test_decode_step_host_buffers():
     kt, vt, gt = wl.make_token(w, DEV)
     K = w.budget_pages()
     outs = []
-    for host in (False, True):
+    for host in (False, "pinned", "pageable"):       # pinned inputs are gathered by a kernel, pageable ones copied
         c = rq.Cache(w.B, w.H, w.D, w.S, w.T, w.dtype)
         rq.rq_build_cache(c.handle, k, v, g)
         if host:
-            hq, hk, hv, hg = (t.cpu().pin_memory() for t in (q, kt, vt, gt))
-            o = torch.empty(w.B, w.H, w.D, dtype=w.dtype).pin_memory()
-            idx = torch.empty(w.B, w.H, K, dtype=torch.int32).pin_memory()
+            pin = (lambda t: t.pin_memory()) if host == "pinned" else (lambda t: t)
+            hq, hk, hv, hg = (pin(t.cpu()) for t in (q, kt, vt, gt))
+            o = pin(torch.empty(w.B, w.H, w.D, dtype=w.dtype))
+            idx = pin(torch.empty(w.B, w.H, K, dtype=torch.int32))
             rq.rq_decode_step_host(c.handle, hq, hk, hv, hg, K, 0.0, o, idx)
         else:
             o = torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=DEV)
@@ -262,8 +263,8 @@ def test_decode_step_host_buffers():
             rq.rq_decode_step(c.handle, q, kt, vt, gt, K, 0.0, o, idx)
         torch.cuda.synchronize()
         outs.append((o.cpu(), idx.cpu(), c.state_view().cpu()))
-    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
-    assert torch.equal(outs[0][2], outs[1][2])
+    for other in outs[1:]:
+        assert torch.equal(outs[0][0], other[0]) and torch.equal(outs[0][1], other[1]) and torch.equal(outs[0][2], other[2])
 
 
 def test_capacity_errors_leave_cache_unchanged():
