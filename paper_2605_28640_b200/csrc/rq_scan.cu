@@ -10,8 +10,9 @@
 //
 // Work decomposition.  One CTA owns one (batch, head) pair and one chunk of
 // CT consecutive cache positions.  A thread owns CH channels (one 16-byte
-// vector of the storage type) and TS consecutive tokens whose k, v and g stay
-// in registers from the first to the last use.  Threads with the same
+// vector of the storage type) and TS consecutive tokens whose k, v and g are
+// fetched once, by asynchronous copies, into the thread's own slots of shared
+// memory and read from there for both of its passes.  Threads with the same
 // channels and consecutive token slices sit NCG lanes apart, so the carry
 // between the slices of a warp moves with warp shuffles; warps exchange their
 // totals through shared memory.
@@ -48,8 +49,42 @@ __device__ __forceinline__ void st_release(int32_t *p, int v)
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// asynchronous copy of BYTES (8 or 16) from global to shared memory
+template <int BYTES>
+__device__ __forceinline__ void cp_async(void *dst_smem, const void *src)
+{
+    static_assert(BYTES == 8 || BYTES == 16, "unsupported copy size");
+    if constexpr (BYTES == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// N consecutive elements of G from shared memory as floats (N * sizeof(G) in {8, 16, 32} bytes)
+template <typename G, int N>
+__device__ __forceinline__ void lds_n(const void *p, float *out)
+{
+    constexpr int BYTES = N * (int)sizeof(G);
+    if constexpr (BYTES == 16) {
+        unpack16<G>(lds16(p), out);
+    } else if constexpr (BYTES == 32) {
+        unpack16<G>(lds16(p), out);
+        unpack16<G>(lds16(static_cast<const char *>(p) + 16), out + N / 2);
+    } else {
+        static_assert(BYTES == 8, "unsupported vector width");
+        const uint2 r = *static_cast<const uint2 *>(p);
+        if constexpr (sizeof(G) == 2) {
+            out[0] = bf16lo(r.x); out[1] = bf16hi(r.x);
+            out[2] = bf16lo(r.y); out[3] = bf16hi(r.y);
+        } else {
+            out[0] = __uint_as_float(r.x); out[1] = __uint_as_float(r.y);
+        }
+    }
+}
+
 template <typename T, typename G, int D, int S>
-__global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
+__global__ void __launch_bounds__(NT, 3) scan_kernel(ScanArgs a, int64_t chunk0)
 {
     constexpr int CH = VecOf<T>::N;
     constexpr int NCG = D / CH;
@@ -81,24 +116,37 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
     const T *vp = static_cast<const T *>(a.v);
     const G *gp = static_cast<const G *>(a.g);
 
-    // ---- load this thread's TS tokens (identity map for positions outside the new range)
-    uint4 rk[TS], rv[TS];
-    float g[TS][CH];
+    // ---- fetch this thread's TS tokens into its own slots of shared memory with asynchronous
+    // copies (identity map for positions outside the new range): the data waits there, not in
+    // registers, so that three CTAs fit on an SM
+    constexpr int GB = CH * (int)sizeof(G);      // bytes of this thread's gates of one token
+    extern __shared__ __align__(16) unsigned char dsm[];
+    uint4 *kbuf = reinterpret_cast<uint4 *>(dsm);            // [TS][NT]
+    uint4 *vbuf = kbuf + TS * NT;                            // [TS][NT]
+    unsigned char *gbuf = reinterpret_cast<unsigned char *>(vbuf + TS * NT);   // [TS][NT][GB]
 #pragma unroll
     for (int i = 0; i < TS; ++i) {
         const int64_t pos = pos0 + i;
+        const int slot = i * NT + tid;
         if (pos >= a.len0 && pos < end) {
             const int64_t src = (int64_t)b * a.sb + (pos - a.len0) * a.st + (int64_t)h * a.sh + cg * CH;
-            rk[i] = ldg16(kp + src);
-            rv[i] = ldg16(vp + src);
-            load_n<G, CH>(gp + src, g[i]);
+            cp_async<16>(&kbuf[slot], kp + src);
+            cp_async<16>(&vbuf[slot], vp + src);
+            if constexpr (GB == 32) {
+                cp_async<16>(gbuf + (size_t)slot * GB, gp + src);
+                cp_async<16>(gbuf + (size_t)slot * GB + 16, reinterpret_cast<const char *>(gp + src) + 16);
+            } else {
+                cp_async<GB>(gbuf + (size_t)slot * GB, gp + src);
+            }
         } else {
-            rk[i] = make_uint4(0, 0, 0, 0);
-            rv[i] = make_uint4(0, 0, 0, 0);
+            kbuf[slot] = make_uint4(0, 0, 0, 0);
+            vbuf[slot] = make_uint4(0, 0, 0, 0);
+            constexpr uint32_t one = sizeof(G) == 2 ? 0x3f803f80u : 0x3f800000u;   // 1.0 in G, packed
 #pragma unroll
-            for (int c = 0; c < CH; ++c) g[i][c] = 1.0f;
+            for (int wd = 0; wd < GB / 4; ++wd) reinterpret_cast<uint32_t *>(gbuf + (size_t)slot * GB)[wd] = one;
         }
     }
+    cp_async_wait_all();                         // a thread only ever reads the slots it filled itself
 
     // ---- the slice's own map (A, Bk, Bv) from a zero state
     float A[CH], Bk[CH], Bv[CH];
@@ -107,14 +155,16 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
 #pragma unroll
     for (int i = 0; i < TS; ++i) {
         float kf[CH], vf[CH];
-        unpack16<T>(rk[i], kf);
-        unpack16<T>(rv[i], vf);
+        float gi[CH];
+        unpack16<T>(kbuf[i * NT + tid], kf);
+        unpack16<T>(vbuf[i * NT + tid], vf);
+        lds_n<G, CH>(gbuf + (size_t)(i * NT + tid) * GB, gi);
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
-            const float om = 1.0f - g[i][c];
-            Bk[c] = fmaf(g[i][c], Bk[c], om * kf[c]);
-            Bv[c] = fmaf(g[i][c], Bv[c], om * vf[c]);
-            A[c] *= g[i][c];
+            const float om = 1.0f - gi[c];
+            Bk[c] = fmaf(gi[c], Bk[c], om * kf[c]);
+            Bv[c] = fmaf(gi[c], Bv[c], om * vf[c]);
+            A[c] *= gi[c];
         }
     }
 
@@ -282,13 +332,15 @@ __global__ void __launch_bounds__(NT, 2) scan_kernel(ScanArgs a, int64_t chunk0)
         for (int i = 0; i < TS; ++i) {
             const int64_t pos = pos0 + i;
             float kf[CH], vf[CH];
-            unpack16<T>(rk[i], kf);
-            unpack16<T>(rv[i], vf);
+            float gi[CH];
+            unpack16<T>(kbuf[i * NT + tid], kf);
+            unpack16<T>(vbuf[i * NT + tid], vf);
+            lds_n<G, CH>(gbuf + (size_t)(i * NT + tid) * GB, gi);
 #pragma unroll
             for (int c = 0; c < CH; ++c) {
-                const float om = 1.0f - g[i][c];
-                sk[c] = fmaf(g[i][c], sk[c], om * kf[c]);
-                sv[c] = fmaf(g[i][c], sv[c], om * vf[c]);
+                const float om = 1.0f - gi[c];
+                sk[c] = fmaf(gi[c], sk[c], om * kf[c]);
+                sv[c] = fmaf(gi[c], sv[c], om * vf[c]);
             }
             const bool valid = pos >= a.len0 && pos < end;
             const bool fill = pos >= end && pos < tail_end;   // unused slots of the last page
@@ -375,7 +427,19 @@ cudaError_t run(const ScanArgs &a, cudaStream_t s)
     if (e != cudaSuccess) return e;
     e = cudaMemsetAsync(a.flags, 0, (size_t)a.B * a.H * a.chunks_cap * sizeof(int32_t), s);
     if (e != cudaSuccess) return e;
-    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, 0, s>>>(a, c0);
+    constexpr int TS = scan_ts(D, (int)sizeof(T));
+    constexpr int DSM = TS * NT * (32 + CH * (int)sizeof(G));    // k, v and g slots of every thread
+    static bool ready[64];
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!ready[dev]) {
+        e = cudaFuncSetAttribute(scan_kernel<T, G, D, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, DSM);
+        if (e != cudaSuccess) return e;
+        ready[dev] = true;
+    }
+    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, DSM, s>>>(a, c0);
     return cudaGetLastError();
 }
 
