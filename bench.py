@@ -109,6 +109,7 @@ def pick_workload(name):
              "cfg4-1/8": dataclasses.replace(wl.CONFIGS[4], budget_den=8),
              "cfg4-1/4": dataclasses.replace(wl.CONFIGS[4], budget_den=4),
              "half": dataclasses.replace(wl.METRIC, name="decode-64k-b1", T=65536),
+             "page64": dataclasses.replace(wl.METRIC, name="decode-128k-b1-page64", S=64),
              "small": dataclasses.replace(wl.CONFIGS[1], name="small-16k")}
     return table[name]
 

@@ -57,7 +57,9 @@ int rq::stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_c
     int64_t g = units / (2 * warps_per_cta);
     if (g > resident_ctas) g = resident_ctas;
     if (g > max_ctas) g = max_ctas;
-    if (g >= heads && heads > 0) g -= g % heads;
+    // whole CTAs per head when that leaves at most 15 % of the CTAs out; otherwise all CTAs run
+    // and their warps spread over the heads on their own (the kernels handle both)
+    if (g >= heads && heads > 0 && (g - g % heads) * 100 >= g * 85) g -= g % heads;
     if (g < 1) g = 1;
     return (int)g;
 }

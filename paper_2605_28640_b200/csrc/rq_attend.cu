@@ -6,13 +6,14 @@
 // block of decayed values (for 16-token pages a tile is the whole page and its
 // keys and values are adjacent in the cache).  A head's tiles are numbered in
 // the order of its index list and handed out one at a time through a per-head
-// ticket counter.  The grid is sized to what the GPU holds at once.  With at
-// least one CTA per head (the usual case) head h is served by the CTAs h,
-// h + BH, h + 2 BH, ...: they sit on SMs all over the chip, so every head's
+// ticket counter.  The grid is sized to what the GPU holds at once.  When it is
+// a whole number of CTAs per head (the usual case) head h is served by the CTAs
+// h, h + BH, h + 2 BH, ...: they sit on SMs all over the chip, so every head's
 // group is equally fast, and inside a group a warp that the memory system
 // serves more slowly simply pulls fewer tickets; everybody finishes together.
-// With fewer CTAs than heads every warp sweeps forward over the heads from its
-// own starting head.  The per-head counters are zero at launch: the selection
+// Otherwise (fewer CTAs than heads, or a head count that would leave many CTAs
+// out) the warps are spread evenly over the heads and every warp sweeps forward
+// from its starting head, helping the heads that still have tiles.  The per-head counters are zero at launch: the selection
 // kernel clears them (a memset does when this kernel is launched on its own).
 //
 // Data movement.  Each warp runs its own pipeline: lane 0 issues one bulk
@@ -180,8 +181,8 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     const T *kvbase = static_cast<const T *>(a.kv);
 
     // ------------------------------------------------------------ issue side
-    // fixed: at least one CTA per head; all warps of CTA c serve head c % BH and never change.
-    const bool fixed = NC >= BH;
+    // fixed: a whole number of CTAs per head; all warps of CTA c serve head c % BH and never change.
+    const bool fixed = NC >= BH && NC % BH == 0;
     const int h0 = fixed ? (int)(blockIdx.x % BH) : (int)((int64_t)wg * BH / TW);
     // Warps that start on head h.  Each owns DEPTH tickets by position, so its ring fills
     // without waiting for an atomic; the counter hands out the tickets after those.
@@ -684,7 +685,7 @@ extern "C" int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int
 #undef RQ_OCC
     if (e != cudaSuccess) return RQ_ERR_CUDA;
     const int grid = attend_grid((int64_t)BH * per_head, BH, occ * sms);
-    const int64_t slots = grid >= BH ? grid / BH : std::min<int64_t>((int64_t)grid * kAttendWarps, per_head);
+    const int64_t slots = (grid >= BH && grid % BH == 0) ? grid / BH : std::min<int64_t>((int64_t)grid * kAttendWarps, per_head);
     const size_t ctr_bytes = (size_t)BH * kCtrStride * sizeof(int32_t);
     const size_t need = 256 + ctr_bytes + (size_t)BH * slots * (a.D + 4) * sizeof(float);
     if (need > kStaticScratchBytes) return RQ_ERR_CAPACITY;

@@ -31,7 +31,7 @@ constexpr int kScoreWarps = 4;         // warps per scoring CTA, each with its o
 constexpr int kScoreRingBytes = 64 * 1024;   // shared-memory ring of one scoring CTA (all warps): three CTAs per SM
 constexpr int kAttendWarps = 4;        // warps per flash-decode CTA, each with its own copy pipeline
 constexpr int kAttendRingBytes = 64 * 1024;  // shared-memory ring of one flash-decode CTA (all warps): three CTAs per SM
-constexpr int kAttendMaxWarps = 1536;  // upper bound of the warps of a flash-decode grid
+constexpr int kAttendMaxWarps = 2048;  // upper bound of the warps of a flash-decode grid
 constexpr int kCtrStride = 64;         // int32 between the counters of two heads (256 bytes: different L2 lines)
 constexpr int kTopkThreads = 1024;     // threads of the selection CTA
 constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
@@ -98,8 +98,10 @@ cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx
                           int idx_stride, float scale, float *partial, const AttendCounters &ctr, void *o,
                           int sm_count, cudaStream_t s);
 // Grid of a streaming kernel for a number of work units spread evenly over `heads` heads: at
-// most what the device holds at once, at least two units per warp, and, once there is a CTA per
-// head, a whole number of CTAs per head (heads served by more CTAs than others would finish early).
+// most what the device holds at once, at least two units per warp, and a whole number of CTAs per
+// head if that keeps at least 85 % of the CTAs (heads served by more CTAs than others would
+// finish early); a grid that is not a multiple of the heads makes the kernels spread warps, not
+// CTAs, over the heads.
 int stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_cta, int max_ctas);
 // flash-decode grid for a number of tiles and the CTAs the device holds at once
 int attend_grid(int64_t tiles, int heads, int resident_ctas);

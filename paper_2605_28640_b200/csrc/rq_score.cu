@@ -13,8 +13,8 @@
 // Data movement is the flash-decode kernel's: the unit of work is 8 KiB of
 // consecutive records of one head, a head's units are handed out through a
 // per-head ticket counter (own tickets by position first), head h is served by
-// the CTAs h, h + BH, ... (or, with fewer CTAs than heads, warps sweep over
-// the heads), and every warp streams its units through its own ring of
+// the CTAs h, h + BH, ... (or, when the grid is not a whole number of CTAs
+// per head, warps spread over the heads and sweep forward), and every warp streams its units through its own ring of
 // shared-memory stages filled by bulk (TMA, 1-D) copies.  The ticket counters
 // are zero at launch; the selection kernel, which always runs next, clears
 // them.
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     const T *meta = static_cast<const T *>(a.meta);
 
     // ------------------------------------------------------------ issue side (as in the flash-decode kernel)
-    const bool fixed = NC >= BH;
+    const bool fixed = NC >= BH && NC % BH == 0;
     const int h0 = fixed ? (int)(blockIdx.x % BH) : (int)((int64_t)wg * BH / TW);
     auto first_warp = [&](int h) -> int { return (int)(((int64_t)h * TW + BH - 1) / BH); };   // sweeping mode
     auto owners = [&](int h) -> int {                // warps that start on head h; each owns DEPTH tickets
