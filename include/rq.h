@@ -24,9 +24,12 @@
  *   - Pointers are DEVICE pointers unless the name of the function ends in
  *     `_host` or the parameter is documented as host memory.
  *   - The caller owns every byte of device memory.  The library allocates no
- *     device memory and keeps no global state; `rq_sizes` tells the caller how
- *     much to allocate and `rq_cache_init` adopts the buffers.  Buffers must be
- *     256-byte aligned and must outlive the `rq_cache`.
+ *     device memory and keeps no state of a cache outside the caller's buffers
+ *     (it only remembers, per device, launch parameters it has looked up once);
+ *     `rq_sizes` tells the caller how much to allocate and `rq_cache_init`
+ *     adopts the buffers.  Buffers must be 256-byte aligned and must outlive
+ *     the `rq_cache`.  (rq_attend_pages_noalloc is the one call that uses a
+ *     fixed array inside the library instead of a workspace.)
  *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = default stream).
  *     Work is enqueued on it and the call returns without synchronising,
  *     except where stated.  Calls on one cache must be stream-ordered; two
