@@ -95,8 +95,12 @@ __global__ void __launch_bounds__(NT, 3) scan_kernel(ScanArgs a, int64_t chunk0)
     static_assert(CT % S == 0 && S % TS == 0, "chunk must hold whole pages of whole slices");
     static_assert(NCG <= 32 && 32 % NCG == 0, "a warp must hold whole slices");
 
-    __shared__ float wtot[NW][3][D];
-    __shared__ float mm[NSL][2][D];
+    // the warp totals are dead (several CTA barriers earlier) when the page bounds are reduced:
+    // both live in the same shared memory
+    constexpr int kScratchFloats = NW * 3 * D > NSL * 2 * D ? NW * 3 * D : NSL * 2 * D;
+    __shared__ float scratch[kScratchFloats];
+    float (*wtot)[3][D] = reinterpret_cast<float (*)[3][D]>(scratch);
+    float (*mm)[2][D] = reinterpret_cast<float (*)[2][D]>(scratch);
     __shared__ float sm_agg[3][D];               // the chunk's map
     __shared__ float sm_in[2][D];                // state entering the chunk
     __shared__ int sm_ticket;
