@@ -42,98 +42,11 @@
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
+#include "rq_stream.cuh"
 
 namespace rq {
 
 namespace {
-
-constexpr int kTileRows = 16;
-constexpr int kDoneTileBits = 20;                  // low bits of a head's done word count tiles
-constexpr int kDoneTileMask = (1 << kDoneTileBits) - 1;
-
-template <typename T, int D, int S>
-struct AttendGeom {
-    static constexpr int CH = VecOf<T>::N;         // elements per 16-byte vector
-    static constexpr int LPR = D / CH;             // lanes per row
-    static constexpr int RPI = 32 / LPR;           // rows per warp-wide read
-    static constexpr int TR = kTileRows;           // rows per tile
-    static constexpr int TPP = S / TR;             // tiles per page
-    static constexpr int NI = TR / RPI;            // warp-wide reads per tile and tensor
-    static constexpr int TILE_BYTES = TR * D * (int)sizeof(T);
-    static constexpr int STAGE_BYTES = 2 * TILE_BYTES;
-    static constexpr int SH = (LPR == 32 ? 5 : LPR == 16 ? 4 : LPR == 8 ? 3 : 2) - (NI == 16 ? 4 : NI == 8 ? 3 : NI == 4 ? 2 : 1);   // log2(LPR / NI)
-    static_assert(SH >= 0 && (NI << SH) == LPR, "a row's score must end up in at least one lane");
-    static constexpr int NW = kAttendWarps;
-    static constexpr int DEPTH_RAW = kAttendRingBytes / (NW * STAGE_BYTES);
-    static constexpr int DEPTH = DEPTH_RAW < 1 ? 1 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
-    static constexpr int RING_BYTES = NW * DEPTH * STAGE_BYTES;
-    // ring | barriers | (head, valid rows) per stage | per-warp m, l, tiles, head | per-warp acc
-    static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 8 + 4 * NW * 4 + NW * D * 4;
-    static_assert(LPR <= 32 && TR % RPI == 0 && S % TR == 0, "unsupported geometry");
-    static_assert(TILE_BYTES % 16 == 0, "bulk copies move multiples of 16 bytes");
-};
-
-// Combine n partials of a head (one warp): o = sum_s 2^(m_s-M) acc_s / sum_s 2^(m_s-M) l_s.
-// Lane -> (channel group g = lane % 8 of D/8 channels, subset j = lane / 8): a lane sweeps the
-// partials s = j, j+4, ... with a running maximum, four records per round trip (their loads are
-// all issued before the first is used); the four subsets are merged with two shuffle steps.
-// A record is [m, l, -, -, acc[D]]; an empty one has m = -inf and zeros.
-template <typename T, int D>
-__device__ __forceinline__ void combine_head(const float *src, int n, T *o_row, int lane)
-{
-    constexpr int CPL = D / 8;                     // channels per lane
-    constexpr int NV = CPL / 4;                    // 16-byte vectors per lane and record
-    constexpr int U = 4;                           // records in flight per lane
-    const int g = lane & 7, j = lane >> 3;
-    float M = -CUDART_INF_F, L = 0.0f, A[CPL];
-#pragma unroll
-    for (int c = 0; c < CPL; ++c) A[c] = 0.0f;
-    for (int s0 = j; s0 < n; s0 += 4 * U) {
-        float2 ml[U];
-        float4 v[U][NV];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int s = s0 + 4 * u;
-            const float *rec = src + (int64_t)(s < n ? s : s0) * (D + 4);
-            ml[u] = ld_cg_now(reinterpret_cast<const float2 *>(rec));
-            if (s >= n) ml[u].x = -CUDART_INF_F;
-#pragma unroll
-            for (int c = 0; c < NV; ++c) v[u][c] = ld_cg_now(reinterpret_cast<const float4 *>(rec + 4 + g * CPL) + c);
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            // branch-free; an empty partial or a record past the end gets weight 0
-            const float Mn = fmaxf(M, ml[u].x);
-            const float fo = M == -CUDART_INF_F ? 0.0f : exp2f(M - Mn);
-            const float fn = ml[u].x == -CUDART_INF_F ? 0.0f : exp2f(ml[u].x - Mn);
-            L = fmaf(L, fo, ml[u].y * fn);
-#pragma unroll
-            for (int c = 0; c < NV; ++c) {
-                A[4 * c + 0] = fmaf(A[4 * c + 0], fo, v[u][c].x * fn);
-                A[4 * c + 1] = fmaf(A[4 * c + 1], fo, v[u][c].y * fn);
-                A[4 * c + 2] = fmaf(A[4 * c + 2], fo, v[u][c].z * fn);
-                A[4 * c + 3] = fmaf(A[4 * c + 3], fo, v[u][c].w * fn);
-            }
-            M = Mn;
-        }
-    }
-#pragma unroll
-    for (int off = 8; off < 32; off <<= 1) {
-        const float Mo = __shfl_xor_sync(0xffffffffu, M, off);
-        const float Lo = __shfl_xor_sync(0xffffffffu, L, off);
-        const float Mn = fmaxf(M, Mo);
-        const float fa = M == -CUDART_INF_F ? 0.0f : exp2f(M - Mn), fb = Mo == -CUDART_INF_F ? 0.0f : exp2f(Mo - Mn);
-        L = L * fa + Lo * fb;
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) A[c] = A[c] * fa + __shfl_xor_sync(0xffffffffu, A[c], off) * fb;
-        M = Mn;
-    }
-    if (j == 0) {
-        const float inv = 1.0f / L;
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) store1<T>(o_row + g * CPL + c, A[c] * inv);
-    }
-}
 
 template <typename T, int D, int S>
 __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a, const T *q,
@@ -143,7 +56,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
                                                                    AttendCounters ctr, T *o)
 {
     using G = AttendGeom<T, D, S>;
-    constexpr int CH = G::CH, LPR = G::LPR, RPI = G::RPI, TR = G::TR, TPP = G::TPP, NI = G::NI;
+    constexpr int CH = G::CH, LPR = G::LPR, TR = G::TR, TPP = G::TPP;
     constexpr int NW = G::NW, DEPTH = G::DEPTH;
     constexpr unsigned FULL = 0xffffffffu;
 
@@ -158,7 +71,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     float *sm_acc = reinterpret_cast<float *>(sm_h + NW);            // [NW][D]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int rsub = lane / LPR, cgp = lane % LPR;
+    const int cgp = lane % LPR;
     const int BH = a.B * a.H;
     const int64_t P = (a.len + S - 1) / S;
     const int per_head = n_idx * TPP;                // tiles per head (host: < 2^20)
@@ -291,27 +204,15 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     int cur = -1;                                    // head of the running accumulation
     int tiles = 0;                                   // tiles of `cur` consumed by this warp
     int slot = 0;                                    // lane 0, sweeping only: this warp's partial slot in `cur`
-    float qf[CH], acc[CH];
+    AttendState<T> st;
 #pragma unroll
-    for (int c = 0; c < CH; ++c) { qf[c] = 0.0f; acc[c] = 0.0f; }
-    float m_run = -CUDART_INF_F, l_run = 0.0f;
+    for (int c = 0; c < CH; ++c) { st.qf[c] = 0.0f; st.acc[c] = 0.0f; }
+    st.m = -CUDART_INF_F;
+    st.l = 0.0f;
     int stage = 0;
     uint32_t phase = 0;                              // one parity bit per stage
     bool dead = false;                               // a wait ran out: stop streaming, finish cleanly
 
-    // sum the warp's softmax denominators and the row groups' accumulators (all share m_run);
-    // lanes < LPR end up with the channel sums
-    auto merge_rows = [&]() {
-        // every row's weight was added by the 2^SH lanes that hold the row: sum over the warp
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) l_run += __shfl_xor_sync(FULL, l_run, off);
-        l_run *= 1.0f / (float)(1 << G::SH);
-#pragma unroll
-        for (int off = LPR; off < 32; off <<= 1) {
-#pragma unroll
-            for (int c = 0; c < CH; ++c) acc[c] += __shfl_xor_sync(FULL, acc[c], off);
-        }
-    };
     // after a partial of head h has been written by this warp: count it, and combine if it was the last
     auto arrive = [&](int h, int count_word, int expect_ctas, int n_fixed) {
         // The partial was written by several lanes: the warp barrier orders those stores before
@@ -336,18 +237,18 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     };
     // sweeping mode: the warp writes its own partial for head h
     auto flush_warp = [&](int h) {
-        merge_rows();
+        attend_merge_rows<T, D, S>(st);
         const int s = __shfl_sync(FULL, slot, 0);
         if (s >= slots_per_head) {                   // cannot happen: a warp joins a head by holding one of its tiles
             if (lane == 0) atomicExch(a.status, RQ_ERR_CAPACITY);
             return;
         }
         float *dst = partial + ((int64_t)h * slots_per_head + s) * (D + 4);
-        if (lane == 0) *reinterpret_cast<float2 *>(dst) = make_float2(m_run, l_run);
+        if (lane == 0) *reinterpret_cast<float2 *>(dst) = make_float2(st.m, st.l);
         if (lane < LPR) {
 #pragma unroll
             for (int c = 0; c < CH; c += 4)
-                *reinterpret_cast<float4 *>(dst + 4 + cgp * CH + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+                *reinterpret_cast<float4 *>(dst + 4 + cgp * CH + c) = make_float4(st.acc[c], st.acc[c + 1], st.acc[c + 2], st.acc[c + 3]);
         }
         arrive(h, tiles, 0, -1);
     };
@@ -360,13 +261,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
             cur = inf.x;
             tiles = 0;
             if (!fixed && lane == 0) slot = atomicAdd(ctr.nslot + cur * kCtrStride, 1);
-#pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                qf[c] = load1<T>(q + (int64_t)cur * D + cgp * CH + c) * scale_log2;
-                acc[c] = 0.0f;
-            }
-            m_run = -CUDART_INF_F;
-            l_run = 0.0f;
+            attend_begin_head<T, D>(st, q, cur, scale_log2, lane);
         }
         const int valid = inf.y;
         if (valid > 0 && !dead) {
@@ -382,58 +277,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
         if (valid > 0 && !dead) {
             const T *ks = reinterpret_cast<const T *>(myring + (size_t)stage * G::STAGE_BYTES);
             const T *vs = ks + TR * D;
-            // K: partial dot products of NI row groups, then a reduction over the LPR lanes of a
-            // row in which every step also halves the values a lane carries: afterwards a lane
-            // holds the complete score of ONE row (row group cgp >> SH, shared by 2^SH lanes)
-            float s[NI];
-#pragma unroll
-            for (int n = 0; n < NI; ++n) {
-                float kf[CH];
-                unpack16<T>(lds16(ks + (n * 32 + lane) * CH), kf);
-                float d = 0.0f;
-#pragma unroll
-                for (int c = 0; c < CH; ++c) d = fmaf(qf[c], kf[c], d);
-                s[n] = d;
-            }
-            int nv = NI;
-#pragma unroll
-            for (int off = LPR / 2; off > 0; off >>= 1) {
-                if (nv > 1) {
-                    const int half = nv / 2;
-                    const bool hi = (lane & off) != 0;
-#pragma unroll
-                    for (int i = 0; i < NI / 2; ++i) {
-                        if (i < half) {
-                            const float send = hi ? s[i] : s[i + half];
-                            const float keep = hi ? s[i + half] : s[i];
-                            s[i] = keep + __shfl_xor_sync(FULL, send, off);
-                        }
-                    }
-                    nv = half;
-                } else {
-                    s[0] += __shfl_xor_sync(FULL, s[0], off);
-                }
-            }
-            const int row = ((cgp >> G::SH) & (NI - 1)) * RPI + rsub;
-            const float sc = row < valid ? s[0] : -CUDART_INF_F;
-            float m_new = fmaxf(m_run, sc);
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, off));
-            const float alpha = exp2f(m_run - m_new);    // 0 on the first tile (m_run = -inf)
-            const float p_row = exp2f(sc - m_new);       // 0 for a masked row
-            m_run = m_new;
-            l_run = fmaf(l_run, alpha, p_row);           // per lane; 2^SH lanes repeat a row
-#pragma unroll
-            for (int c = 0; c < CH; ++c) acc[c] *= alpha;
-            // V: row group n's weight comes from the lane that holds it
-#pragma unroll
-            for (int n = 0; n < NI; ++n) {
-                const float p = __shfl_sync(FULL, p_row, rsub * LPR + (n << G::SH));
-                float vf[CH];
-                unpack16<T>(lds16(vs + (n * 32 + lane) * CH), vf);
-#pragma unroll
-                for (int c = 0; c < CH; ++c) acc[c] = fmaf(p, vf[c], acc[c]);
-            }
+            attend_tile<T, D, S>(st, ks, vs, valid, lane);
         }
         ++tiles;
         __syncwarp();                                // every lane is done with the stage
@@ -449,12 +293,12 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     }
 
     // fixed mode: merge the CTA's warps (all on head h0) into one partial in slot blockIdx / BH
-    merge_rows();
-    if (dead || cur < 0) { m_run = -CUDART_INF_F; l_run = 0.0f; tiles = 0; }
-    if (lane == 0) { sm_m[warp] = m_run; sm_l[warp] = l_run; sm_t[warp] = tiles; sm_h[warp] = dead; }
+    attend_merge_rows<T, D, S>(st);
+    if (dead || cur < 0) { st.m = -CUDART_INF_F; st.l = 0.0f; tiles = 0; }
+    if (lane == 0) { sm_m[warp] = st.m; sm_l[warp] = st.l; sm_t[warp] = tiles; sm_h[warp] = dead; }
     if (lane < LPR) {
 #pragma unroll
-        for (int c = 0; c < CH; ++c) sm_acc[warp * D + cgp * CH + c] = (dead || cur < 0) ? 0.0f : acc[c];
+        for (int c = 0; c < CH; ++c) sm_acc[warp * D + cgp * CH + c] = (dead || cur < 0) ? 0.0f : st.acc[c];
     }
     __syncthreads();
     if (warp != 0) return;

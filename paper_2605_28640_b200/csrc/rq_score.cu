@@ -30,87 +30,11 @@
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
+#include "rq_stream.cuh"
 
 namespace rq {
 
 namespace {
-
-constexpr int kUnitBytes = 8192;
-
-template <typename T, int D>
-struct ScoreGeom {
-    static constexpr int CH = VecOf<T>::N;           // elements per 16-byte vector
-    static constexpr int REC_BYTES = 2 * D * (int)sizeof(T);
-    static constexpr int VPR = REC_BYTES / 16;       // 16-byte vectors per record
-    static constexpr int RU = kUnitBytes / REC_BYTES;   // records per unit
-    static constexpr int LPP = VPR > 32 ? 32 : VPR;  // lanes that share one record in a warp-wide read
-    static constexpr int VPL = VPR / LPP;            // vectors per lane and record (1 or 2)
-    static constexpr int PPW = 32 / LPP;             // records per warp-wide read
-    static constexpr int NR = RU / PPW;              // record groups per unit
-    static constexpr int NW = kScoreWarps;
-    static constexpr int DEPTH_RAW = kScoreRingBytes / (NW * kUnitBytes);
-    static constexpr int DEPTH = DEPTH_RAW < 1 ? 1 : (DEPTH_RAW > 8 ? 8 : DEPTH_RAW);
-    static constexpr int RING_BYTES = NW * DEPTH * kUnitBytes;
-    // ring | barriers | (head, first record, records) per stage | reduction scratch of the update
-    static constexpr int SMEM_BYTES = RING_BYTES + NW * DEPTH * 8 + NW * DEPTH * 16 + 64;
-    static_assert(VPL == 1 || VPL == 2, "unsupported record width");
-    static_assert(D <= NW * 32, "the update uses one thread per channel");
-};
-
-// One step of Eq. 1 for head h (thread d < D owns channel d): new state, cache row, bounds of
-// the newest page, and that page's score.  `len` is the length AFTER the append.
-template <typename T, int D>
-__device__ __forceinline__ void update_head(const DecodeArgs &a, int h, const T *q, const T *k_t, const T *v_t,
-                                            const void *g_t, float *scores, float *red)
-{
-    const int d = threadIdx.x;
-    const int S = a.S;
-    const int64_t pos = a.len - 1;
-    const int64_t page = pos / S;
-    const int slot = (int)(pos % S);
-    float term = 0.0f;
-    if (d < D) {
-        float *st = a.state + (int64_t)h * 2 * D;
-        const float g = a.gate_dtype == RQ_BF16 ? load1<bf16>(static_cast<const bf16 *>(g_t) + (int64_t)h * D + d)
-                                                : load1<float>(static_cast<const float *>(g_t) + (int64_t)h * D + d);
-        const float om = 1.0f - g;
-        const float sk = fmaf(g, st[d], om * load1<T>(k_t + (int64_t)h * D + d));
-        const float sv = fmaf(g, st[D + d], om * load1<T>(v_t + (int64_t)h * D + d));
-        st[d] = sk;
-        st[D + d] = sv;
-        T *pg = static_cast<T *>(a.kv) + (((int64_t)h * a.page_cap + page) * 2) * S * D;
-        store1<T>(pg + (int64_t)slot * D + d, sk);
-        store1<T>(pg + (int64_t)(S + slot) * D + d, sv);
-        const float r = round_storage<T>(sk);
-        T *m = static_cast<T *>(a.meta) + (((int64_t)h * a.page_cap + page) * 2) * D;
-        float mn = r, mx = r;
-        if (slot == 0) {
-            // a fresh page: clear its unused slots so that later reads are defined
-            for (int s2 = 1; s2 < S; ++s2) {
-                store1<T>(pg + (int64_t)s2 * D + d, 0.0f);
-                store1<T>(pg + (int64_t)(S + s2) * D + d, 0.0f);
-            }
-        } else {
-            mn = fminf(load1<T>(m + d), r);
-            mx = fmaxf(load1<T>(m + D + d), r);
-        }
-        store1<T>(m + d, mn);
-        store1<T>(m + D + d, mx);
-        const float qd = load1<T>(q + (int64_t)h * D + d);
-        term = fmaxf(qd * mn, qd * mx);
-    }
-    // score of the newest page: sum of the D terms
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) term += __shfl_xor_sync(0xffffffffu, term, off);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = term;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float s = 0.0f;
-        for (int w = 0; w < (D + 31) / 32; ++w) s += red[w];
-        scores[(int64_t)h * a.page_cap + page] = s;
-    }
-    __syncthreads();
-}
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, const T *q, const T *k_t,
@@ -118,7 +42,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
                                                                  int32_t *next, int do_update)
 {
     using G = ScoreGeom<T, D>;
-    constexpr int CH = G::CH, VPR = G::VPR, RU = G::RU, LPP = G::LPP, VPL = G::VPL, PPW = G::PPW, NR = G::NR;
+    constexpr int CH = G::CH, RU = G::RU, VPL = G::VPL;
     constexpr int NW = G::NW, DEPTH = G::DEPTH;
     constexpr unsigned FULL = 0xffffffffu;
 
@@ -129,7 +53,6 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     float *red = reinterpret_cast<float *>(infos + NW * DEPTH);
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int sub = lane / LPP, c = lane % LPP;
     const int BH = a.B * a.H;
     const int P = (int)((a.len + a.S - 1) / a.S);
     const int Ps = do_update ? P - 1 : P;            // records per head that are streamed
@@ -248,17 +171,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
         if (inf.x < 0) break;
         if (inf.x != cur) {
             cur = inf.x;
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-                const int vec = c + v * LPP;         // vector index inside the record
-                const bool is_max = vec >= VPR / 2;
-                const int ch0 = (vec % (VPR / 2)) * CH;
-#pragma unroll
-                for (int i = 0; i < CH; ++i) {
-                    const float x = load1<T>(q + (int64_t)cur * D + ch0 + i);
-                    qs[v][i] = is_max ? fmaxf(x, 0.0f) : fminf(x, 0.0f);
-                }
-            }
+            score_load_q<T, D>(q, cur, lane, qs);
         }
         if (!dead) {
             if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u)) {
@@ -271,49 +184,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
         }
         if (!dead) {
             const unsigned char *ub = myring + (size_t)stage * kUnitBytes;
-            float val[NR];
-#pragma unroll
-            for (int gi = 0; gi < NR; ++gi) {
-                const unsigned char *rec = ub + (size_t)(gi * PPW + sub) * G::REC_BYTES;
-                float s = 0.0f;
-#pragma unroll
-                for (int v = 0; v < VPL; ++v) {
-                    float m[CH];
-                    unpack16<T>(lds16(rec + (c + v * LPP) * 16), m);
-#pragma unroll
-                    for (int i = 0; i < CH; ++i) s = fmaf(qs[v][i], m[i], s);
-                }
-                val[gi] = s;
-            }
-            // sum over the LPP lanes of a record; while more than one value is left a step also
-            // halves the values a lane carries, so the whole reduction costs about NR shuffles
-            int n = NR;
-#pragma unroll
-            for (int off = LPP / 2; off > 0; off >>= 1) {
-                if (n > 1) {
-                    const int half = n / 2;
-                    const bool hi = (lane & off) != 0;
-#pragma unroll
-                    for (int i = 0; i < NR / 2; ++i) {
-                        if (i < half) {
-                            const float send = hi ? val[i] : val[i + half];
-                            const float keep = hi ? val[i + half] : val[i];
-                            val[i] = keep + __shfl_xor_sync(FULL, send, off);
-                        }
-                    }
-                    n = half;
-                } else {
-                    val[0] += __shfl_xor_sync(FULL, val[0], off);
-                }
-            }
-            // the lane now holds the sum of record group `gi` if its low lane bits are zero
-            constexpr int LOG_LPP = LPP == 32 ? 5 : (LPP == 16 ? 4 : (LPP == 8 ? 3 : 2));
-            constexpr int LOG_NR = NR == 32 ? 5 : (NR == 16 ? 4 : (NR == 8 ? 3 : (NR == 4 ? 2 : (NR == 2 ? 1 : 0))));
-            static_assert((1 << LOG_LPP) == LPP && (1 << LOG_NR) == NR && LOG_NR <= LOG_LPP, "unsupported reduction shape");
-            const int gi = (c >> (LOG_LPP - LOG_NR)) & (NR - 1);
-            const bool writer = (c & ((1 << (LOG_LPP - LOG_NR)) - 1)) == 0;
-            const int r = gi * PPW + sub;
-            if (writer && r < inf.z) scores[(int64_t)cur * a.page_cap + inf.y + r] = val[0];
+            score_unit<T, D>(ub, qs, inf.z, scores + (int64_t)cur * a.page_cap + inf.y, lane);
         }
         __syncwarp();
         if (dead) drained = true;
