@@ -1,32 +1,265 @@
 // Second kernel of a decode step: per (b,h) selection of the budget's pages from
 // the page scores (the TopK of Eq. 3), forced first/local pages inside the
-// budget (App. A.1), ties to the lower page index, output ascending.  The
-// routine itself is select_head in rq_select.cuh.
+// budget (App. A.1), ties to the lower page index, output ascending.
 #include <math_constants.h>
 
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
-#include "rq_select.cuh"
 
 namespace rq {
 
 namespace {
 
-// One CTA per (b,h) runs the selection routine; it also clears the ticket counters of the two
-// streaming kernels for its head.
-template <int NTH>
-__global__ void __launch_bounds__(NTH) topk_select_kernel(const float *scores, int64_t score_stride, int P, int K,
-                                                         int n_sink, int n_local, int32_t *idx, int idx_stride,
-                                                         int budget, int32_t *attend_ctr)
+// ---------------------------------------------------------------- top-k
+// One CTA per (b,h).  Scores become order-preserving 32-bit keys in shared
+// memory.  Forced pages (first / newest) are taken outright and count inside
+// the budget.  Among the rest, the k-th largest key is found by a
+// most-significant-digit radix select: the bits that all keys share are
+// skipped, then each pass histograms one 11-bit digit of the keys that still
+// match the prefix found so far and walks the bins from the top until the
+// remaining budget is used up; a pass whose chosen bin is wanted whole ends
+// the search early.  Pages with a larger key are taken; pages with an equal
+// key are taken in index order until the budget is full.  For the output,
+// warp w owns a contiguous range of pages and walks it row by row (row j:
+// pages base_w + 32 j + lane): warp ballots give every taken page its rank
+// inside the warp and a scan over the warp totals its rank in the head, so the
+// output is ascending and unique whatever the thread timing.
+//
+// Every CTA runs this code once on an SM whose instruction cache holds another
+// kernel's code, so the loops are kept rolled: fetching the instructions is a
+// visible part of the run time.
+constexpr uint32_t kKeyForced = 0xffffffffu;   // above every score key
+constexpr int kDigitBits = 11;
+constexpr int kBins = 1 << kDigitBits;
+constexpr int kCandMax = 1024;                 // candidates ranked directly; a fuller bucket goes through the key bits
+
+// the score a key was made from (inverse of order_key)
+__device__ __forceinline__ float key_value(uint32_t k)
 {
-    extern __shared__ __align__(16) unsigned char sel_smem[];
-    const int bh = blockIdx.x;
-    grid_dependency_wait();
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
+                                                            int P, int K, int n_sink, int n_local,
+                                                            int32_t *idx, int idx_stride, int budget,
+                                                            int32_t *attend_ctr)
+{
+    constexpr int NTH = kTopkThreads, NWP = NTH / 32;
+    constexpr unsigned FULL = 0xffffffffu;
+    static_assert(NWP == 32, "second-level reductions are one warp wide");
+    static_assert(kBins == 2 * NTH, "a thread owns two bins in the suffix scan");
+    constexpr int NH = 2;                            // histogram copies; warp w adds to copy w % NH
+    extern __shared__ __align__(16) uint32_t skey[]; // [P] keys of the head
+    __shared__ __align__(16) uint32_t hist[NH][kBins];   // read back as 8-byte pairs
+    __shared__ uint32_t red[NWP], red2[NWP];
+    __shared__ uint32_t s_digit, s_krem, s_cnt, s_ncand, s_tau;
+    __shared__ uint32_t cand[kCandMax];              // keys of the chosen bucket
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int32_t *out = idx + (int64_t)bh * idx_stride;
+    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
     grid_launch_dependents();
-    if (threadIdx.x < 4) attend_ctr[bh * kCtrStride + threadIdx.x] = 0;
-    select_head<NTH>(scores + (int64_t)bh * score_stride, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
-                     sel_smem);
+    if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
+
+    if (K >= P) {                                    // dense: every page, in order
+        for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
+        return;
+    }
+    const float *sc = scores + (int64_t)bh * score_stride;
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll 4
+    for (int p = tid; p < P; p += NTH) {
+        uint32_t kx = kKeyForced;
+        if (p >= n_sink && p < P - n_local) {
+            kx = order_key(__ldcg(sc + p));
+            kx = min(max(kx, 1u), 0xfffffffeu);      // stay clear of the reserved key
+            kmin = min(kmin, kx);
+            kmax = max(kmax, kx);
+        }
+        skey[p] = kx;
+    }
+    int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
+
+    // range of the score keys -> bits they all share
+    kmin = __reduce_min_sync(FULL, kmin);
+    kmax = __reduce_max_sync(FULL, kmax);
+    if (lane == 0) { red[warp] = kmin; red2[warp] = kmax; }
+    __syncthreads();
+    kmin = __reduce_min_sync(FULL, red[lane]);
+    kmax = __reduce_max_sync(FULL, red2[lane]);
+
+    // One histogram pass over the non-forced keys for which `in(key)` holds: bins by `bin(key)`,
+    // walked from the top until k_rem keys are covered.  Leaves the chosen bin in s_digit, the
+    // rank wanted inside it in s_krem and its population in s_cnt.
+    auto select_bin = [&](auto in, auto bin) {
+        __syncthreads();                             // earlier readers of hist / red / s_* are done
+#pragma unroll 1
+        for (int i = tid; i < NH * kBins; i += NTH) (&hist[0][0])[i] = 0u;
+        __syncthreads();
+#pragma unroll 2
+        for (int p = tid; p < P; p += NTH) {
+            const uint32_t kx = skey[p];
+            if (kx != kKeyForced && in(kx)) atomicAdd(&hist[warp % NH][bin(kx)], 1u);
+        }
+        __syncthreads();
+        // thread t owns bins 2t and 2t+1; suffix sums from the top bin down
+        uint32_t c0 = 0, c1 = 0;
+#pragma unroll
+        for (int w = 0; w < NH; ++w) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
+            c0 += v.x;
+            c1 += v.y;
+        }
+        uint32_t suf = c0 + c1;                      // inclusive suffix sum over the threads of the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, suf, off);
+            if (lane + off < 32) suf += t;
+        }
+        if (lane == 0) red[warp] = suf;              // warp totals
+        __syncthreads();
+        const uint32_t wtot = red[lane];
+        uint32_t wsuf = wtot;                        // suffix sum over the warps, every warp on its own
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+            if (lane + off < 32) wsuf += t;
+        }
+        const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+        const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
+        const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
+        const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
+        const uint32_t kr = (uint32_t)k_rem;
+        if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
+        if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
+        __syncthreads();
+    };
+    // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
+    // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
+    auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
+        if (lo_key == hi_key) return lo_key;
+        int hb = 31 - __clz(lo_key ^ hi_key);        // highest bit in which the keys differ
+        uint32_t t = hb == 31 ? 0u : (hi_key >> (hb + 1)) << (hb + 1);   // shared leading bits
+#pragma unroll 1
+        while (hb >= 0) {
+            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
+            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
+            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
+            select_bin([&](uint32_t kx) { return in(kx) && (kx & himask) == (t & himask); },
+                       [&](uint32_t kx) { return (kx >> lo) & dmask; });
+            t |= s_digit << lo;
+            k_rem = (int)s_krem;
+            // every key of the chosen bin is wanted: the bin's lowest possible key is a valid
+            // threshold and the remaining digits need not be resolved
+            if (s_cnt == s_krem) break;
+            hb = lo - 1;
+        }
+        return t;
+    };
+
+    uint32_t tau;                                    // k-th largest key among the non-forced pages
+    if (k_rem <= 0) {
+        tau = 0xfffffffeu + 1u;                      // nothing but forced pages fits: take none of the rest
+    } else if (kmin == kmax) {
+        tau = kmin;
+    } else {
+        // First pass on the score VALUES: 2048 equal-width buckets between the smallest and the
+        // largest score.  The map score -> bucket is monotone, so every key of a higher bucket is
+        // larger than every key of a lower one, and unlike a digit of the key bits the buckets
+        // resolve the bulk of the scores evenly whatever their sign and exponent.
+        const float v_lo = key_value(kmin);
+        const float scale = (float)(kBins - 1) / (key_value(kmax) - v_lo);
+        auto bucket = [&](uint32_t kx) -> uint32_t {
+            const float f = (key_value(kx) - v_lo) * scale;
+            return (uint32_t)min(max((int)f, 0), kBins - 1);
+        };
+        if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
+            tau = radix_select([](uint32_t) { return true; }, kmin, kmax);      // range too wide for a float
+        } else {
+            select_bin([](uint32_t) { return true; }, bucket);
+            const uint32_t b = s_digit, cnt = s_cnt;
+            k_rem = (int)s_krem;
+            // the candidates: keys of the chosen bucket, usually a handful
+            if (tid == 0) s_ncand = 0;
+            __syncthreads();
+            uint32_t cmin = 0xffffffffu, cmax = 0u;
+#pragma unroll 2
+            for (int p = tid; p < P; p += NTH) {
+                const uint32_t kx = skey[p];
+                if (kx != kKeyForced && bucket(kx) == b) {
+                    cmin = min(cmin, kx);
+                    cmax = max(cmax, kx);
+                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = kx;
+                }
+            }
+            __syncthreads();
+            if (cnt <= (uint32_t)kCandMax) {
+                // rank every candidate against all others; the wanted one has fewer than k_rem
+                // candidates above it and at least k_rem at or above it
+                if (tid < (int)cnt) {
+                    const uint32_t mine = cand[tid];
+                    uint32_t g = 0, ge = 0;
+#pragma unroll 4
+                    for (uint32_t j = 0; j < cnt; ++j) {
+                        const uint32_t o = cand[j];
+                        g += o > mine;
+                        ge += o >= mine;
+                    }
+                    if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) s_tau = mine;
+                }
+                __syncthreads();
+                tau = s_tau;
+            } else {
+                // an unusually full bucket (many equal scores): finish on the key bits
+                cmin = __reduce_min_sync(FULL, cmin);
+                cmax = __reduce_max_sync(FULL, cmax);
+                if (lane == 0) { red[warp] = cmin; red2[warp] = cmax; }
+                __syncthreads();
+                cmin = __reduce_min_sync(FULL, red[lane]);
+                cmax = __reduce_max_sync(FULL, red2[lane]);
+                tau = radix_select([&](uint32_t kx) { return bucket(kx) == b; }, cmin, cmax);
+            }
+        }
+    }
+
+    // rank of every taken page: ballots inside the warp, a scan over the warp totals across warps
+    const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp
+    const int base = warp * 32 * rows + lane;        // this lane's page in row 0
+    uint32_t wgt = 0, weq = 0;                       // this warp's counts of "greater" and "equal"
+#pragma unroll 1
+    for (int j = 0; j < rows; ++j) {
+        const int p = base + 32 * j;
+        const uint32_t kx = p < P ? skey[p] : 0u;    // 0 is below every key
+        wgt += __popc(__ballot_sync(FULL, kx > tau));
+        weq += __popc(__ballot_sync(FULL, kx == tau));
+    }
+    __syncthreads();
+    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
+    __syncthreads();
+    uint32_t g_inc = red[lane], e_inc = red2[lane];  // inclusive scans over the warps
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
+        if (lane >= off) { g_inc += tg; e_inc += te; }
+    }
+    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
+    const int r = K - n_gt;                          // how many equal keys to take
+    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
+    int eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll 1
+    for (int j = 0; j < rows; ++j) {
+        const int p = base + 32 * j;
+        const uint32_t kx = p < P ? skey[p] : 0u;
+        const bool is_gt = kx > tau, is_eq = kx == tau;
+        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
+        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
+        if (is_gt) out[gb + min(eb, r)] = p;
+        else if (is_eq && eb < r) out[gb + eb] = p;
+        gt_run += __popc(bg);
+        eq_run += __popc(be);
+    }
+    for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
 }  // namespace
@@ -50,15 +283,15 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
-        e = cudaFuncSetAttribute(topk_select_kernel<kTopkThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)select_smem_bytes(kTopkThreads * kTopkMaxPerThread));
+        e = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kTopkThreads * kTopkMaxPerThread * (int)sizeof(uint32_t));
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)BH);
     cfg.blockDim = dim3(kTopkThreads);
-    cfg.dynamicSmemBytes = select_smem_bytes(P);
+    cfg.dynamicSmemBytes = (size_t)P * sizeof(uint32_t);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -66,8 +299,7 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int64_t stride = a.page_cap;
-    return cudaLaunchKernelEx(&cfg, topk_select_kernel<kTopkThreads>, scores, stride, P, K, ns, nl, idx, idx_stride,
-                              budget, attend_ctr);
+    return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr);
 }
 
 }  // namespace rq
