@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     const int TW = NC * NW;                          // warps in the grid
     const int wg = blockIdx.x * NW + warp;
 
+    const uint64_t stream_policy = l2_evict_first_policy();
     uint64_t *mybars = bars + warp * DEPTH;
     int2 *myinfo = infos + warp * DEPTH;
     unsigned char *myring = ring + (size_t)warp * DEPTH * G::STAGE_BYTES;
@@ -158,8 +159,8 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
             const T *kb = kvbase + (((int64_t)h * a.page_cap + pg) * 2) * S * D + tile * TR * D;
             unsigned char *dst = myring + (size_t)stage * G::STAGE_BYTES;
             mbar_arrive_expect_tx(&mybars[stage], G::STAGE_BYTES);
-            bulk_g2s(dst, kb, G::TILE_BYTES, &mybars[stage]);
-            bulk_g2s(dst + G::TILE_BYTES, kb + (int64_t)S * D, G::TILE_BYTES, &mybars[stage]);
+            bulk_g2s_hint(dst, kb, G::TILE_BYTES, &mybars[stage], stream_policy);
+            bulk_g2s_hint(dst + G::TILE_BYTES, kb + (int64_t)S * D, G::TILE_BYTES, &mybars[stage], stream_policy);
         }
     };
     // put the next tile into a stage (or the end mark); called by the whole warp

@@ -60,6 +60,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     const int NC = gridDim.x, TW = NC * NW;
     const int wg = blockIdx.x * NW + warp;
 
+    const uint64_t stream_policy = l2_evict_first_policy();
     uint64_t *mybars = bars + warp * DEPTH;
     int4 *myinfo = infos + warp * DEPTH;
     unsigned char *myring = ring + (size_t)warp * DEPTH * kUnitBytes;
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
         myinfo[stage] = make_int4(h, first, n, 0);
         const T *src = meta + ((int64_t)h * a.page_cap + first) * 2 * D;
         mbar_arrive_expect_tx(&mybars[stage], n * G::REC_BYTES);
-        bulk_g2s(myring + (size_t)stage * kUnitBytes, src, n * G::REC_BYTES, &mybars[stage]);
+        bulk_g2s_hint(myring + (size_t)stage * kUnitBytes, src, n * G::REC_BYTES, &mybars[stage], stream_policy);
     };
     auto refill = [&](int stage) {                   // whole warp
         while (n_own > 0) {

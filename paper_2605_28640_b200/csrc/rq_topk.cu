@@ -262,6 +262,244 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
+
+// ---------------------------------------------------------------- top-k, keys in registers
+// The same selection for heads of at most ROWS * 1024 pages: a thread keeps the keys of its ROWS
+// pages (row j: page base_w + 32 j + lane, so a warp owns a contiguous range and reads whole
+// 128-byte lines) and their bucket numbers in registers; the passes over the keys then need no
+// shared-memory traffic and no address arithmetic, which is what the one SM that selects a head
+// spends its issue slots on.  The histogram is cleared before the wait for the scoring kernel.
+template <int ROWS>
+__global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *scores, int64_t score_stride, int P,
+                                                                int K, int n_sink, int n_local, int32_t *idx,
+                                                                int idx_stride, int budget, int32_t *attend_ctr)
+{
+    constexpr int NTH = kTopkThreads, NWP = NTH / 32;
+    constexpr unsigned FULL = 0xffffffffu;
+    constexpr uint32_t kAbsent = 0u;                 // below every key: a row beyond the head's pages
+    constexpr int NH = 2;                            // histogram copies; warp w adds to copy w % NH
+    static_assert(ROWS % 2 == 0, "bucket numbers are kept in pairs");
+    static_assert(NWP == 32 && kBins == 2 * NTH, "one warp wide second-level reductions; two bins per thread");
+    __shared__ __align__(16) uint32_t hist[NH][kBins];
+    __shared__ uint32_t red[NWP], red2[NWP];
+    __shared__ uint32_t s_digit, s_krem, s_cnt, s_ncand, s_tau;
+    __shared__ uint32_t cand[kCandMax];
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int32_t *out = idx + (int64_t)bh * idx_stride;
+    const float *sc = scores + (int64_t)bh * score_stride;
+    const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp (<= ROWS)
+    const int base = warp * 32 * rows + lane;        // this lane's page in row 0
+
+    static_assert(NH * kBins == 4 * NTH, "a thread clears four bins");
+    auto clear_hist = [&]() { reinterpret_cast<uint4 *>(&hist[0][0])[tid] = make_uint4(0u, 0u, 0u, 0u); };
+    clear_hist();
+    if (tid == 0) s_ncand = 0;
+    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
+    grid_launch_dependents();
+    if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
+    if (K >= P) {                                    // dense: every page, in order
+        for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
+        return;
+    }
+
+    float v[ROWS];
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+        const int p = base + 32 * j;
+        v[j] = (j < rows && p < P) ? __ldcg(sc + p) : 0.0f;
+    }
+    uint32_t key[ROWS];
+    uint32_t kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+        const int p = base + 32 * j;
+        uint32_t kx = kAbsent;
+        if (j < rows && p < P) {
+            kx = kKeyForced;
+            if (p >= n_sink && p < P - n_local) {
+                kx = min(max(order_key(v[j]), 1u), 0xfffffffeu);   // stay clear of the reserved keys
+                kmin = min(kmin, kx);
+                kmax = max(kmax, kx);
+            }
+        }
+        key[j] = kx;
+    }
+    int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
+    auto scored = [&](uint32_t kx) { return kx != kAbsent && kx != kKeyForced; };
+
+    auto block_minmax = [&](uint32_t &lo, uint32_t &hi) {
+        lo = __reduce_min_sync(FULL, lo);
+        hi = __reduce_max_sync(FULL, hi);
+        __syncthreads();                             // earlier readers of red / red2 are done
+        if (lane == 0) { red[warp] = lo; red2[warp] = hi; }
+        __syncthreads();
+        lo = __reduce_min_sync(FULL, red[lane]);
+        hi = __reduce_max_sync(FULL, red2[lane]);
+    };
+    block_minmax(kmin, kmax);                        // its barriers also publish the cleared histogram
+
+    // After a histogram pass: walk the bins from the top until k_rem keys are covered.  Leaves the
+    // chosen bin in s_digit, the rank wanted inside it in s_krem and its population in s_cnt.
+    auto pick_bin = [&]() {
+        __syncthreads();
+        uint32_t c0 = 0, c1 = 0;                     // thread t owns bins 2t and 2t+1
+#pragma unroll
+        for (int w = 0; w < NH; ++w) {
+            const uint2 h2 = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
+            c0 += h2.x;
+            c1 += h2.y;
+        }
+        uint32_t suf = c0 + c1;                      // inclusive suffix sum over the threads of the warp
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, suf, off);
+            if (lane + off < 32) suf += t;
+        }
+        if (lane == 0) red[warp] = suf;              // warp totals
+        __syncthreads();
+        const uint32_t wtot = red[lane];
+        uint32_t wsuf = wtot;                        // suffix sum over the warps, every warp on its own
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+            if (lane + off < 32) wsuf += t;
+        }
+        const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+        const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
+        const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
+        const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
+        const uint32_t kr = (uint32_t)k_rem;
+        if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
+        if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
+        __syncthreads();
+    };
+    // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
+    // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
+    auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
+        if (lo_key == hi_key) return lo_key;
+        int hb = 31 - __clz(lo_key ^ hi_key);        // highest bit in which the keys differ
+        uint32_t t = hb == 31 ? 0u : (hi_key >> (hb + 1)) << (hb + 1);   // shared leading bits
+#pragma unroll 1
+        while (hb >= 0) {
+            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
+            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
+            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
+            __syncthreads();                         // earlier readers of the histogram are done
+            clear_hist();
+            __syncthreads();
+#pragma unroll
+            for (int j = 0; j < ROWS; ++j) {
+                const uint32_t kx = key[j];
+                if (scored(kx) && in(kx, j) && (kx & himask) == (t & himask))
+                    atomicAdd(&hist[warp % NH][(kx >> lo) & dmask], 1u);
+            }
+            pick_bin();
+            t |= s_digit << lo;
+            k_rem = (int)s_krem;
+            if (s_cnt == s_krem) break;              // the whole bin is wanted: its lowest possible key is a threshold
+            hb = lo - 1;
+        }
+        return t;
+    };
+
+    uint32_t tau;                                    // k-th largest key among the non-forced pages
+    if (k_rem <= 0) {
+        tau = 0xfffffffeu + 1u;                      // nothing but forced pages fits: take none of the rest
+    } else if (kmin == kmax) {
+        tau = kmin;
+    } else {
+        // 2048 equal-width buckets of the score VALUE between the smallest and the largest score
+        // (monotone in the key), as in the kernel above
+        const float v_lo = key_value(kmin);
+        const float scale = (float)(kBins - 1) / (key_value(kmax) - v_lo);
+        if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
+            tau = radix_select([](uint32_t, int) { return true; }, kmin, kmax);      // range too wide for a float
+        } else {
+            uint32_t bk2[ROWS / 2];                  // bucket of every key of this thread, two to a word
+            auto bk = [&](int j) -> uint32_t { return (bk2[j / 2] >> (16 * (j & 1))) & 0xffffu; };
+#pragma unroll
+            for (int j = 0; j < ROWS; ++j) {
+                const uint32_t kx = key[j];
+                const float f = (key_value(kx) - v_lo) * scale;
+                const uint32_t bj = scored(kx) ? (uint32_t)min(max((int)f, 0), kBins - 1) : 0xffffu;
+                if (scored(kx)) atomicAdd(&hist[warp % NH][bj], 1u);
+                bk2[j / 2] = (j & 1) ? (bk2[j / 2] | (bj << 16)) : bj;
+            }
+            pick_bin();
+            const uint32_t b = s_digit, cnt = s_cnt;
+            k_rem = (int)s_krem;
+            uint32_t cmin = 0xffffffffu, cmax = 0u;
+#pragma unroll
+            for (int j = 0; j < ROWS; ++j) {
+                if (bk(j) == b) {                    // a candidate: usually a handful in the whole head
+                    cmin = min(cmin, key[j]);
+                    cmax = max(cmax, key[j]);
+                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = key[j];
+                }
+            }
+            __syncthreads();
+            if (cnt <= (uint32_t)kCandMax) {
+                // rank every candidate against all others; the wanted one has fewer than k_rem
+                // candidates above it and at least k_rem at or above it
+                if (tid < (int)cnt) {
+                    const uint32_t mine = cand[tid];
+                    uint32_t g = 0, ge = 0;
+#pragma unroll 4
+                    for (uint32_t j = 0; j < cnt; ++j) {
+                        const uint32_t o = cand[j];
+                        g += o > mine;
+                        ge += o >= mine;
+                    }
+                    if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) s_tau = mine;
+                }
+                __syncthreads();
+                tau = s_tau;
+            } else {
+                block_minmax(cmin, cmax);            // an unusually full bucket (many equal scores): finish on the key bits
+                tau = radix_select([&](uint32_t, int j) { return bk(j) == b; }, cmin, cmax);
+            }
+        }
+    }
+
+    // rank of every taken page: ballots inside the warp, a scan over the warp totals across warps
+    uint32_t wgt = 0, weq = 0;                       // this warp's counts of "greater" and "equal"
+    uint32_t mg = 0, me = 0;                         // bit j: this lane's key of row j is greater / equal
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+        const bool is_gt = key[j] > tau, is_eq = key[j] == tau;   // absent rows hold key 0: neither
+        mg |= (uint32_t)is_gt << j;
+        me |= (uint32_t)is_eq << j;
+    }
+    wgt = __reduce_add_sync(FULL, (uint32_t)__popc(mg));
+    weq = __reduce_add_sync(FULL, (uint32_t)__popc(me));
+    __syncthreads();
+    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
+    __syncthreads();
+    uint32_t g_inc = red[lane], e_inc = red2[lane];  // inclusive scans over the warps
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
+        if (lane >= off) { g_inc += tg; e_inc += te; }
+    }
+    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
+    const int r = K - n_gt;                          // how many equal keys to take
+    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
+    int eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+    for (int j = 0; j < ROWS; ++j) {
+        const bool is_gt = (mg >> j) & 1u, is_eq = (me >> j) & 1u;
+        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
+        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
+        const int p = base + 32 * j;
+        if (is_gt) out[gb + min(eb, r)] = p;
+        else if (is_eq && eb < r) out[gb + eb] = p;
+        gt_run += __popc(bg);
+        eq_run += __popc(be);
+    }
+    for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
+}
+
 }  // namespace
 
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
@@ -299,6 +537,15 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int64_t stride = a.page_cap;
+    const int rows = (P + kTopkThreads - 1) / kTopkThreads;
+    if (rows <= 16) {                                // the keys of a head fit in registers
+        using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *);
+        static const Kernel by_rows[8] = {topk_reg_kernel<2>,  topk_reg_kernel<4>,  topk_reg_kernel<6>,  topk_reg_kernel<8>,
+                                          topk_reg_kernel<10>, topk_reg_kernel<12>, topk_reg_kernel<14>, topk_reg_kernel<16>};
+        cfg.dynamicSmemBytes = 0;
+        return cudaLaunchKernelEx(&cfg, by_rows[(rows - 1) / 2], scores, stride, P, K, ns, nl, idx, idx_stride, budget,
+                                  attend_ctr);
+    }
     return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr);
 }
 
