@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/*_kernel_64k_b1.md: 64 MiB launches, scaled by two to the 128 MiB launches of the
 # default workload, traffic being proportional to the pages processed): kernel -> bytes, or None
 # when the kernel has changed since the capture.
-NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.40e6), "attend": 2 * (67.24e6 + 0.93e6)}
+NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.57e6), "attend": 2 * (67.24e6 + 1.05e6)}
 
 
 def measured_peak():
