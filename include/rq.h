@@ -158,8 +158,9 @@ RQ_API int rq_decode_step(rq_cache *cache, const void *q, const void *k_t, const
  * to the device, the step runs, o (and sel_idx_out if not NULL) are copied back to host
  * memory, all on `stream`.  Pinned (page-locked or registered), 16-byte aligned inputs are read
  * by one small gather kernel straight from host memory; other inputs go through four
- * asynchronous copies (synchronous for pageable memory, as usual).  The outputs are valid after
- * the stream is synchronised.  Bytes moved per call: 4 inputs + 1 output of B*H*D elements
+ * asynchronous copies (synchronous for pageable memory, as usual).  A pinned, 16-byte aligned o
+ * is written by the attention kernel itself; any other o is filled by a copy from a staging
+ * buffer.  The outputs are valid after the stream is synchronised.  Bytes moved per call: 4 inputs + 1 output of B*H*D elements
  * (+ the index list). */
 RQ_API int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_host,
                         const void *v_t_host, const void *g_t_host,

@@ -351,10 +351,14 @@ int rq_decode_step_host(rq_cache *cache, const void *q_host, const void *k_t_hos
         return RQ_ERR_CUDA;
     }
     int32_t *sel = (int32_t *)((char *)cache->workspace + w.sel);
-    const int st = rq_decode_step(cache, dq, dk, dv, dg, budget_pages, scale, dout,
+    // A pinned output buffer is writable from the device: the kernel that produces the output
+    // writes it there itself, which saves the copy operation behind it.
+    const void *o_view = nullptr;
+    const bool o_direct = device_view(o_host, &o_view);
+    const int st = rq_decode_step(cache, dq, dk, dv, dg, budget_pages, scale, o_direct ? const_cast<void *>(o_view) : dout,
                                   sel_idx_out_host ? sel : nullptr, stream);
     if (st != RQ_OK) return st;
-    if (cudaMemcpyAsync(o_host, dout, eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (!o_direct && cudaMemcpyAsync(o_host, dout, eb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return RQ_ERR_CUDA;
     if (sel_idx_out_host) {
         const size_t ib = (size_t)c.batch * c.heads * budget_pages * sizeof(int32_t);
         if (cudaMemcpyAsync(sel_idx_out_host, sel, ib, cudaMemcpyDeviceToHost, s) != cudaSuccess)
