@@ -33,8 +33,6 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     WorkspaceLayout w;
     const size_t BH = (size_t)c.batch * c.heads;
     const size_t pc = (size_t)((c.capacity_tokens + c.page_size - 1) / c.page_size);
-    const int ct = scan_chunk_tokens(c.head_dim, c.dtype);
-    w.scan_chunks_cap = (c.capacity_tokens + ct - 1) / ct + 1;
     size_t off = 0;
     w.status = off;  off += align256(64 * sizeof(int32_t));
     w.tickets = off; off += align256(BH * (size_t)kCtrStride * sizeof(int32_t));
@@ -42,9 +40,6 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
     const size_t slots = (size_t)attend_slots_per_head((int64_t)c.max_budget_pages * (c.page_size / 16));
     w.partial = off; off += align256(BH * slots * (size_t)(c.head_dim + 4) * sizeof(float));
-    w.agg = off;     off += align256(BH * (size_t)w.scan_chunks_cap * 3 * c.head_dim * sizeof(float));
-    w.inc = off;     off += align256(BH * (size_t)w.scan_chunks_cap * 2 * c.head_dim * sizeof(float));
-    w.flags = off;   off += align256((BH * (size_t)w.scan_chunks_cap + 64) * sizeof(int32_t));
     w.staging = off; off += align256(5 * BH * (size_t)c.head_dim * 4);
     w.total = off;
     return w;
@@ -262,14 +257,9 @@ int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
     a.k = k; a.v = v; a.g = g;
     a.sb = stride_b; a.st = stride_t; a.sh = stride_h;
     a.kv = cache->kv; a.meta = cache->meta; a.state = (float *)cache->state;
-    a.agg = (float *)((char *)cache->workspace + w.agg);
-    a.inc = (float *)((char *)cache->workspace + w.inc);
-    a.flags = (int32_t *)((char *)cache->workspace + w.flags);
-    a.ticket = a.flags + (size_t)c.batch * c.heads * w.scan_chunks_cap;
-    a.status = (int32_t *)((char *)cache->workspace + w.status);
     a.B = c.batch; a.H = c.heads; a.D = c.head_dim; a.S = c.page_size;
     a.dtype = c.dtype; a.gate_dtype = c.gate_dtype;
-    a.len0 = cache->len; a.T = T; a.page_cap = cache->page_capacity; a.chunks_cap = w.scan_chunks_cap;
+    a.len0 = cache->len; a.T = T; a.page_cap = cache->page_capacity;
     if (launch_scan(a, (cudaStream_t)stream) != cudaSuccess) return RQ_ERR_CUDA;
     cache->len += T;
     return RQ_OK;

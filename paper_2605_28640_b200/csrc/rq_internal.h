@@ -9,22 +9,10 @@
 namespace rq {
 
 // ---- geometry of the prefill scan (must agree between sizing and launch) ----
-constexpr int kScanThreads = 256;  // threads per CTA
+constexpr int kScanThreads = 512;  // threads per CTA
 
-// tokens a scan thread keeps in registers; chosen so that a chunk
-// (threads / channel-groups * tokens) is a whole number of 64-token pages too
-__host__ __device__ constexpr int scan_ts(int head_dim, int elem_bytes)
-{
-    return (kScanThreads / (head_dim / (16 / elem_bytes))) * 4 >= 64 ? 4 : 8;
-}
-
-// tokens covered by one scan CTA for a (head_dim, dtype) pair
-inline int scan_chunk_tokens(int head_dim, int dtype)
-{
-    int eb = dtype == RQ_BF16 ? 2 : 4;
-    int ncg = head_dim / (16 / eb);        // channel groups of one 16-byte vector
-    return (kScanThreads / ncg) * scan_ts(head_dim, eb);
-}
+constexpr int kScanChannels = 32;   // channels of one prefill CTA (a lane per channel)
+constexpr int kScanRunTokens = 8;   // consecutive positions that one warp of a prefill CTA owns in a tile
 
 // ---- decode-side geometry ----
 constexpr int kScoreWarps = 4;         // warps per scoring CTA, each with its own copy pipeline
@@ -44,12 +32,8 @@ struct WorkspaceLayout {
     size_t scores;    // float [BH][page_capacity]
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
-    size_t agg;       // float [BH][scan chunks][3][D] prefill chunk maps
-    size_t inc;       // float [BH][scan chunks][2][D] prefill chunk end states
-    size_t flags;     // int32 [BH][scan chunks] + ticket counter
     size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
     size_t total;
-    int64_t scan_chunks_cap;
 };
 
 WorkspaceLayout workspace_layout(const rq_config &c);
@@ -60,13 +44,8 @@ struct ScanArgs {
     int64_t sb, st, sh;     // element strides of k, v, g
     void *kv, *meta;
     float *state;
-    float *agg;             // [BH][chunks_cap][3][D] chunk maps
-    float *inc;             // [BH][chunks_cap][2][D] state at the end of a chunk
-    int32_t *flags;         // [BH][chunks_cap] 0 = nothing, 1 = map published, 2 = end state published
-    int32_t *ticket;        // next (chunk, head) to hand out
-    int32_t *status;
     int B, H, D, S, dtype, gate_dtype;
-    int64_t len0, T, page_cap, chunks_cap;
+    int64_t len0, T, page_cap;
 };
 cudaError_t launch_scan(const ScanArgs &a, cudaStream_t s);
 

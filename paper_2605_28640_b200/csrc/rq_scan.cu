@@ -1,37 +1,29 @@
-// Prefill: single-pass chained scan of the gated decay recurrence (Eq. 1)
-// fused with the paged cache write and the per-page min/max of the stored keys
-// (Appendix A.1, "Sparse inference settings").  Every input byte is read once.
+// Prefill: the gated decay recurrence (Eq. 1) over a whole sequence, fused with
+// the paged cache write and the per-page min/max of the stored keys
+// (Appendix A.1, "Sparse inference settings").  One launch, every input byte
+// read once, every output byte written once, no scratch in global memory.
 //
-// The recurrence x~_t = g_t x~_{t-1} + (1-g_t) x_t is a first-order linear
-// recurrence, so a run of tokens acts on the incoming state as the affine map
-// s -> A s + B with A = prod g and B = the run's own state from zero.  Maps
-// compose as (A2,B2)o(A1,B1) = (A2 A1, A2 B1 + B2), which is associative, so
-// time can be cut into pieces that are reduced independently.
+// The recurrence x~_t = g_t x~_{t-1} + (1-g_t) x_t runs along time and is
+// independent per (batch, head, channel).  Work decomposition: one CTA owns
+// one (batch, head) pair and 32 neighbouring channels (a lane per channel) and
+// walks the whole sequence, so the state never leaves the CTA: there is no
+// look-back between CTAs, no flag and no wait.  Measured on B200, 128 CTAs that
+// each stream 64-byte row segments 8 KiB apart reach the same bandwidth as a
+// plain copy, so nothing is lost by giving a CTA a quarter of a head's row.
 //
-// Work decomposition.  One CTA owns one (batch, head) pair and one chunk of
-// CT consecutive cache positions.  A thread owns CH channels (one 16-byte
-// vector of the storage type) and TS consecutive tokens whose k, v and g are
-// fetched once, by asynchronous copies, into the thread's own slots of shared
-// memory and read from there for both of its passes.  Threads with the same
-// channels and consecutive token slices sit NCG lanes apart, so the carry
-// between the slices of a warp moves with warp shuffles; warps exchange their
-// totals through shared memory.
-//
-// Chaining.  A CTA takes its (chunk, head) from a ticket counter, chunk-major
-// with the heads varying fastest, so every chunk before its own was taken
-// earlier by a CTA that is running or done, and CTAs that run together read
-// one contiguous stretch of the [B][T][H][D] inputs.  It loads its tokens,
-// reduces them to the chunk's map, publishes the map (flag 1), then looks back
-// over the records of the chunks before it, composing their maps until it
-// meets one that already knows the state at its own end (flag 2); that gives
-// the state entering the chunk.  Which chunks are composed is fixed by the
-// chunk's number (back to the last multiple of eight), not by timing, so the
-// result is the same bits on every run.  It publishes its own end state (flag 2)
-// before the heavy part, the token-by-token application with rounding, page
-// writes and page bounds, so later chunks never wait for that.  Waits on a
-// flag are bounded: when the limit runs out the kernel records
-// RQ_ERR_TIMEOUT in the status word and carries on with a zero carry instead
-// of spinning.
+// Inside a CTA time is cut into tiles of 128 positions that move through a
+// ring of shared-memory stages filled by asynchronous copies (several tiles
+// ahead of the arithmetic).  A warp owns 16 consecutive positions of the tile.
+// A run of tokens acts on the incoming state as the affine map s -> A s + B
+// with A = prod g and B = the run's own state from zero, and maps compose as
+// (A2,B2)o(A1,B1) = (A2 A1, A2 B1 + B2).  Per tile: every thread reduces its
+// run to a map (pass 1); after a barrier it composes the maps of the warps
+// before it onto the state that entered the tile, and the last warp leaves the
+// state for the next tile; then it applies the recurrence token by token,
+// rounds to the storage type, writes the rounded rows back into the stage and
+// tracks min/max of the rounded keys (pass 2); after a barrier the stage goes
+// out to the cache in 16-byte pieces.  The order of all floating-point
+// operations is fixed, so the result is the same bits on every run.
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
@@ -41,401 +33,246 @@ namespace rq {
 namespace {
 
 constexpr int NT = kScanThreads;
-constexpr int kLookWindow = 8;                  // chunks examined per look-back round
-constexpr int kFlagPollLimit = 1 << 20;         // polls of one flag before giving up
+constexpr int NW = NT / 32;
+constexpr int CG = kScanChannels;               // channels of one CTA: a lane per channel
+constexpr int RT = kScanRunTokens;              // consecutive positions of one warp in a tile
+constexpr int TT = NW * RT;                     // positions of one tile
 
-__device__ __forceinline__ void st_release(int32_t *p, int v)
+// asynchronous copy of 16 bytes from global to shared memory
+__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
 {
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// asynchronous copy of BYTES (8 or 16) from global to shared memory
-template <int BYTES>
-__device__ __forceinline__ void cp_async(void *dst_smem, const void *src)
-{
-    static_assert(BYTES == 8 || BYTES == 16, "unsupported copy size");
-    if constexpr (BYTES == 16)
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
-    else
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__device__ __forceinline__ float elem_to_float(bf16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float elem_to_float(float x) { return x; }
+template <typename T> __device__ __forceinline__ T float_to_elem(float x);
+template <> __device__ __forceinline__ bf16 float_to_elem<bf16>(float x) { return __float2bfloat16_rn(x); }
+template <> __device__ __forceinline__ float float_to_elem<float>(float x) { return x; }
 
-// N consecutive elements of G from shared memory as floats (N * sizeof(G) in {8, 16, 32} bytes)
-template <typename G, int N>
-__device__ __forceinline__ void lds_n(const void *p, float *out)
+// bytes of one ring stage: the k, v and g segments of a tile
+template <typename T, typename G> __host__ __device__ constexpr int scan_stage_bytes() { return TT * CG * (2 * (int)sizeof(T) + (int)sizeof(G)); }
+// stages of the ring: as many as fit in 192 KiB, at most six
+template <typename T, typename G> __host__ __device__ constexpr int scan_stages()
 {
-    constexpr int BYTES = N * (int)sizeof(G);
-    if constexpr (BYTES == 16) {
-        unpack16<G>(lds16(p), out);
-    } else if constexpr (BYTES == 32) {
-        unpack16<G>(lds16(p), out);
-        unpack16<G>(lds16(static_cast<const char *>(p) + 16), out + N / 2);
-    } else {
-        static_assert(BYTES == 8, "unsupported vector width");
-        const uint2 r = *static_cast<const uint2 *>(p);
-        if constexpr (sizeof(G) == 2) {
-            out[0] = bf16lo(r.x); out[1] = bf16hi(r.x);
-            out[2] = bf16lo(r.y); out[3] = bf16hi(r.y);
-        } else {
-            out[0] = __uint_as_float(r.x); out[1] = __uint_as_float(r.y);
-        }
-    }
+    return 192 * 1024 / scan_stage_bytes<T, G>() < 6 ? 192 * 1024 / scan_stage_bytes<T, G>() : 6;
 }
 
 template <typename T, typename G, int D, int S>
-__global__ void __launch_bounds__(NT, 3) scan_kernel(ScanArgs a, int64_t chunk0)
+__global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int ntiles)
 {
-    constexpr int CH = VecOf<T>::N;
-    constexpr int NCG = D / CH;
-    constexpr int NSL = NT / NCG;
-    constexpr int TS = scan_ts(D, (int)sizeof(T));
-    constexpr int CT = NSL * TS;
-    constexpr int NW = NT / 32;
-    static_assert(CT % S == 0 && S % TS == 0, "chunk must hold whole pages of whole slices");
-    static_assert(NCG <= 32 && 32 % NCG == 0, "a warp must hold whole slices");
+    constexpr int NST = scan_stages<T, G>();
+    constexpr int STAGE = scan_stage_bytes<T, G>();
+    constexpr int EPC_T = 16 / (int)sizeof(T), EPC_G = 16 / (int)sizeof(G);   // elements per 16-byte piece
+    constexpr int CPR_T = CG / EPC_T, CPR_G = CG / EPC_G;                      // pieces per row segment
+    constexpr int NCH_T = TT * CPR_T, NCH_G = TT * CPR_G;                      // pieces per tile
+    constexpr int WPP = S / RT;                                                // warps that share a page
+    static_assert(D % CG == 0, "a head is a whole number of channel groups");
+    static_assert(S % RT == 0 && TT % S == 0 && NW % WPP == 0, "a page is a whole number of warp runs inside one tile");
+    static_assert(NCH_T % NT == 0 && NCH_G % NT == 0, "every thread moves the same number of pieces");
+    static_assert(NST >= 2, "the ring needs two stages");
 
-    // the warp totals are dead (several CTA barriers earlier) when the page bounds are reduced:
-    // both live in the same shared memory
-    constexpr int kScratchFloats = NW * 3 * D > NSL * 2 * D ? NW * 3 * D : NSL * 2 * D;
-    __shared__ float scratch[kScratchFloats];
-    float (*wtot)[3][D] = reinterpret_cast<float (*)[3][D]>(scratch);
-    float (*mm)[2][D] = reinterpret_cast<float (*)[2][D]>(scratch);
-    __shared__ float sm_agg[3][D];               // the chunk's map
-    __shared__ float sm_in[2][D];                // state entering the chunk
-    __shared__ int sm_ticket;
+    extern __shared__ __align__(16) unsigned char dsm[];
+    __shared__ float wmap[NW][3][CG];            // the warps' maps of the current tile
+    __shared__ float carry[2][2][CG];            // state entering the tile (by tile parity): k, v
+    __shared__ float mm[NW][2][CG];              // min / max of the warps' runs (pages wider than a run)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int cg = tid % NCG, sl = tid / NCG;
-    const int BH = a.B * a.H;
-    if (tid == 0) sm_ticket = atomicAdd(a.ticket, 1);
-    __syncthreads();
-    const int rel = sm_ticket / BH;              // chunk number inside this call
-    const int bh = sm_ticket % BH, b = bh / a.H, h = bh % a.H;
-    const int64_t chunk = chunk0 + rel;
-    const int64_t pos0 = chunk * CT + (int64_t)sl * TS;
+    constexpr int GPH = D / CG;                  // channel groups per head
+    const int bh = blockIdx.x / GPH, c0 = (blockIdx.x % GPH) * CG;
+    const int b = bh / a.H, h = bh % a.H;
     const int64_t end = a.len0 + a.T;
+    const int64_t tail_end = (end + S - 1) / S * S;   // end of the last touched page
+    const int64_t in_base = (int64_t)b * a.sb + (int64_t)h * a.sh + c0;
+    const T *kp = static_cast<const T *>(a.k) + in_base;
+    const T *vp = static_cast<const T *>(a.v) + in_base;
+    const G *gp = static_cast<const G *>(a.g) + in_base;
 
-    const T *kp = static_cast<const T *>(a.k);
-    const T *vp = static_cast<const T *>(a.v);
-    const G *gp = static_cast<const G *>(a.g);
+    auto stage_k = [&](int st) { return reinterpret_cast<T *>(dsm + (size_t)st * STAGE); };
+    auto stage_v = [&](int st) { return reinterpret_cast<T *>(dsm + (size_t)st * STAGE) + TT * CG; };
+    auto stage_g = [&](int st) { return reinterpret_cast<G *>(dsm + (size_t)st * STAGE + 2 * TT * CG * sizeof(T)); };
 
-    // ---- fetch this thread's TS tokens into its own slots of shared memory with asynchronous
-    // copies (identity map for positions outside the new range): the data waits there, not in
-    // registers, so that three CTAs fit on an SM
-    constexpr int GB = CH * (int)sizeof(G);      // bytes of this thread's gates of one token
-    extern __shared__ __align__(16) unsigned char dsm[];
-    uint4 *kbuf = reinterpret_cast<uint4 *>(dsm);            // [TS][NT]
-    uint4 *vbuf = kbuf + TS * NT;                            // [TS][NT]
-    unsigned char *gbuf = reinterpret_cast<unsigned char *>(vbuf + TS * NT);   // [TS][NT][GB]
+    // start the copies of tile `rel` (positions outside the new range are left alone)
+    auto issue = [&](int rel, int st) {
+        const int64_t tile_start = (tile0 + rel) * TT;
+        const int lo = (int)max((int64_t)0, a.len0 - tile_start), hi = (int)min((int64_t)TT, end - tile_start);
+        const int64_t tok0 = tile_start - a.len0;        // input token of row 0
+        T *ks = stage_k(st), *vs = stage_v(st);
+        G *gs = stage_g(st);
 #pragma unroll
-    for (int i = 0; i < TS; ++i) {
-        const int64_t pos = pos0 + i;
-        const int slot = i * NT + tid;
-        if (pos >= a.len0 && pos < end) {
-            const int64_t src = (int64_t)b * a.sb + (pos - a.len0) * a.st + (int64_t)h * a.sh + cg * CH;
-            cp_async<16>(&kbuf[slot], kp + src);
-            cp_async<16>(&vbuf[slot], vp + src);
-            if constexpr (GB == 32) {
-                cp_async<16>(gbuf + (size_t)slot * GB, gp + src);
-                cp_async<16>(gbuf + (size_t)slot * GB + 16, reinterpret_cast<const char *>(gp + src) + 16);
-            } else {
-                cp_async<GB>(gbuf + (size_t)slot * GB, gp + src);
-            }
-        } else {
-            kbuf[slot] = make_uint4(0, 0, 0, 0);
-            vbuf[slot] = make_uint4(0, 0, 0, 0);
-            constexpr uint32_t one = sizeof(G) == 2 ? 0x3f803f80u : 0x3f800000u;   // 1.0 in G, packed
-#pragma unroll
-            for (int wd = 0; wd < GB / 4; ++wd) reinterpret_cast<uint32_t *>(gbuf + (size_t)slot * GB)[wd] = one;
-        }
-    }
-    cp_async_wait_all();                         // a thread only ever reads the slots it filled itself
-
-    // ---- the slice's own map (A, Bk, Bv) from a zero state
-    float A[CH], Bk[CH], Bv[CH];
-#pragma unroll
-    for (int c = 0; c < CH; ++c) { A[c] = 1.0f; Bk[c] = 0.0f; Bv[c] = 0.0f; }
-#pragma unroll
-    for (int i = 0; i < TS; ++i) {
-        float kf[CH], vf[CH];
-        float gi[CH];
-        unpack16<T>(kbuf[i * NT + tid], kf);
-        unpack16<T>(vbuf[i * NT + tid], vf);
-        lds_n<G, CH>(gbuf + (size_t)(i * NT + tid) * GB, gi);
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const float om = 1.0f - gi[c];
-            Bk[c] = fmaf(gi[c], Bk[c], om * kf[c]);
-            Bv[c] = fmaf(gi[c], Bv[c], om * vf[c]);
-            A[c] *= gi[c];
-        }
-    }
-
-    // ---- inclusive scan over the slices of this warp: carry by warp shuffle
-#pragma unroll
-    for (int off = NCG; off < 32; off <<= 1) {
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const float pa = __shfl_up_sync(0xffffffffu, A[c], off);
-            const float pk = __shfl_up_sync(0xffffffffu, Bk[c], off);
-            const float pv = __shfl_up_sync(0xffffffffu, Bv[c], off);
-            if (lane >= off) {
-                Bk[c] = fmaf(A[c], pk, Bk[c]);
-                Bv[c] = fmaf(A[c], pv, Bv[c]);
-                A[c] *= pa;
+        for (int i = 0; i < NCH_T / NT; ++i) {
+            const int ch = tid + i * NT, row = ch / CPR_T, cc = ch % CPR_T;
+            if (row >= lo && row < hi) {
+                const int64_t src = (tok0 + row) * a.st + cc * EPC_T;
+                cp_async16(ks + ch * EPC_T, kp + src);
+                cp_async16(vs + ch * EPC_T, vp + src);
             }
         }
-    }
-    if (lane >= 32 - NCG) {
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            wtot[warp][0][cg * CH + c] = A[c];
-            wtot[warp][1][cg * CH + c] = Bk[c];
-            wtot[warp][2][cg * CH + c] = Bv[c];
+        for (int i = 0; i < NCH_G / NT; ++i) {
+            const int ch = tid + i * NT, row = ch / CPR_G, cc = ch % CPR_G;
+            if (row >= lo && row < hi) cp_async16(gs + ch * EPC_G, gp + (tok0 + row) * a.st + cc * EPC_G);
         }
-    }
-    __syncthreads();
+    };
 
-    // ---- map of everything in the chunk before this warp
-    float Ap[CH], Pk[CH], Pv[CH];
-#pragma unroll
-    for (int c = 0; c < CH; ++c) { Ap[c] = 1.0f; Pk[c] = 0.0f; Pv[c] = 0.0f; }
-    for (int w = 0; w < warp; ++w) {
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            const float wa = wtot[w][0][cg * CH + c];
-            Pk[c] = fmaf(wa, Pk[c], wtot[w][1][cg * CH + c]);
-            Pv[c] = fmaf(wa, Pv[c], wtot[w][2][cg * CH + c]);
-            Ap[c] *= wa;
-        }
+    if (tid < CG) {                              // the state the sequence starts from
+        carry[0][0][tid] = a.state[(int64_t)bh * 2 * D + c0 + tid];
+        carry[0][1][tid] = a.state[(int64_t)bh * 2 * D + D + c0 + tid];
+    }
+#pragma unroll 1
+    for (int s = 0; s < NST - 1; ++s) {
+        if (s < ntiles) issue(s, s);
+        cp_async_commit();
     }
 
-    // ---- the chunk's map = (last warp's total) o (everything before the last warp)
-    if (warp == NW - 1 && lane >= 32 - NCG) {
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            sm_agg[0][cg * CH + c] = A[c] * Ap[c];
-            sm_agg[1][cg * CH + c] = fmaf(A[c], Pk[c], Bk[c]);
-            sm_agg[2][cg * CH + c] = fmaf(A[c], Pv[c], Bv[c]);
-        }
-    }
-    __syncthreads();
+    T *kv = static_cast<T *>(a.kv);
+    T *meta = static_cast<T *>(a.meta);
 
-    // ---- publish the map, find the state entering the chunk, publish the state leaving it
-    float *agg = a.agg + ((int64_t)bh * a.chunks_cap + rel) * 3 * D;
-    float *inc = a.inc + ((int64_t)bh * a.chunks_cap + rel) * 2 * D;
-    int32_t *flags = a.flags + (int64_t)bh * a.chunks_cap;
-    if (tid < D) {
-        const int d = tid;
-        const float ca = sm_agg[0][d], cbk = sm_agg[1][d], cbv = sm_agg[2][d];
-        float in_k, in_v;
-        if (rel == 0) {
-            in_k = a.state[(int64_t)bh * 2 * D + d];
-            in_v = a.state[(int64_t)bh * 2 * D + D + d];
-        } else {
-            agg[d] = ca;
-            agg[D + d] = cbk;
-            agg[2 * D + d] = cbv;
+#pragma unroll 1
+    for (int i = 0; i < ntiles; ++i) {
+        const int st = i % NST;
+        cp_async_wait<NST - 2>();                // this thread's pieces of tile i have landed ...
+        __syncthreads();                         // ... and everybody else's; the stage of tile i - 1 has gone out
+        if (i + NST - 1 < ntiles) issue(i + NST - 1, (i + NST - 1) % NST);
+        cp_async_commit();
+
+        T *ks = stage_k(st), *vs = stage_v(st);
+        const G *gs = stage_g(st);
+        const int row0 = warp * RT;
+        const int64_t tile_start = (tile0 + i) * TT;
+        const int64_t pos0 = tile_start + row0;
+        // rows of the tile that hold new tokens: [lo, hi); rows up to fill_hi pad the last page
+        const int lo = (int)max((int64_t)0, a.len0 - tile_start), hi = (int)min((int64_t)TT, end - tile_start);
+        const int fill_hi = (int)min((int64_t)TT, tail_end - tile_start);
+
+        // ---- pass 1: this thread's run as a map from a zero state (identity outside the new range)
+        float gg[RT], kk[RT], vv[RT];            // g, (1-g) k, (1-g) v
+        float A = 1.0f, Bk = 0.0f, Bv = 0.0f;
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+            const bool valid = row0 + r >= lo && row0 + r < hi;
+            const int e = (row0 + r) * CG + lane;
+            const float g = valid ? elem_to_float(gs[e]) : 1.0f;
+            const float om = 1.0f - g;
+            gg[r] = g;
+            kk[r] = valid ? om * elem_to_float(ks[e]) : 0.0f;
+            vv[r] = valid ? om * elem_to_float(vs[e]) : 0.0f;
+            A *= g;
+            Bk = fmaf(g, Bk, kk[r]);
+            Bv = fmaf(g, Bv, vv[r]);
         }
-        // the D publishing threads are whole warps (D is a multiple of 32); the barrier orders their
-        // stores before thread 0's release store of the flag
-        asm volatile("bar.sync 1, %0;" ::"n"(D));
-        if (rel != 0) {
-            if (d == 0) st_release(flags + rel, 1);
-            // Look back to the anchor: the last chunk before this one whose number is a multiple
-            // of kLookWindow.  The state entering this chunk is the anchor's end state pushed
-            // through the maps of the chunks in between, always in the same order, so the result
-            // does not depend on which chunk happened to finish first.
-            const int base = (rel - 1) / kLookWindow * kLookWindow;
-            const int n = rel - 1 - base;          // maps to compose: chunks base+1 .. rel-1
-            bool timed_out = false;
-            // all flags are read together (relaxed loads, one round trip), then only the ones that
-            // are not there yet are polled; the fence after the loop makes the reads acquire
-            int f[kLookWindow];                    // f[u], u < n: chunk rel-1-u; f[n]: the anchor
+        wmap[warp][0][lane] = A;
+        wmap[warp][1][lane] = Bk;
+        wmap[warp][2][lane] = Bv;
+        __syncthreads();
+
+        // ---- state entering this run: the tile's incoming state through the maps of the warps before
+        float sk = carry[i & 1][0][lane], sv = carry[i & 1][1][lane];
+        {
+            float wa[NW - 1], wk[NW - 1], wv[NW - 1];   // all loads first: only the multiply-adds form a chain
 #pragma unroll
-            for (int u = 0; u < kLookWindow; ++u) f[u] = u <= n ? ld_volatile(flags + (rel - 1 - u)) : 2;
+            for (int w = 0; w < NW - 1; ++w) {
+                wa[w] = wmap[w][0][lane];
+                wk[w] = wmap[w][1][lane];
+                wv[w] = wmap[w][2][lane];
+            }
 #pragma unroll
-            for (int u = 0; u < kLookWindow; ++u) {
-                const int need = u == n ? 2 : 1;
-                int polls = 0;
-                while (u <= n && f[u] < need && !timed_out) {
-                    if (++polls > kFlagPollLimit) timed_out = true;
-                    __nanosleep(32);
-                    f[u] = ld_volatile(flags + (rel - 1 - u));
+            for (int w = 0; w < NW - 1; ++w) {
+                if (w < warp) {
+                    sk = fmaf(wa[w], sk, wk[w]);
+                    sv = fmaf(wa[w], sv, wv[w]);
                 }
             }
-            __threadfence();
-            const float *pa = a.agg + ((int64_t)bh * a.chunks_cap + (rel - 1)) * 3 * D + d;
-            float ra[kLookWindow - 1], rbk[kLookWindow - 1], rbv[kLookWindow - 1];
-#pragma unroll
-            for (int u = 0; u < kLookWindow - 1; ++u) {
-                if (u < n && !timed_out) {
-                    ra[u] = __ldcg(pa - (int64_t)u * 3 * D);
-                    rbk[u] = __ldcg(pa - (int64_t)u * 3 * D + D);
-                    rbv[u] = __ldcg(pa - (int64_t)u * 3 * D + 2 * D);
-                }
-            }
-            float acc_a = 1.0f, acc_k = 0.0f, acc_v = 0.0f;     // map of the chunks base+1 .. rel-1
-#pragma unroll
-            for (int u = 0; u < kLookWindow - 1; ++u) {
-                if (u < n && !timed_out) {           // acc = acc o map(rel-1-u): the older map acts first
-                    acc_k = fmaf(acc_a, rbk[u], acc_k);
-                    acc_v = fmaf(acc_a, rbv[u], acc_v);
-                    acc_a *= ra[u];
-                }
-            }
-            in_k = 0.0f;
-            in_v = 0.0f;
-            if (!timed_out) {
-                const float *pi = a.inc + ((int64_t)bh * a.chunks_cap + base) * 2 * D + d;
-                in_k = fmaf(acc_a, __ldcg(pi), acc_k);
-                in_v = fmaf(acc_a, __ldcg(pi + D), acc_v);
-            }
-            if (timed_out) {
-                atomicExch(a.status, RQ_ERR_TIMEOUT);
-                in_k = 0.0f;
-                in_v = 0.0f;
-            }
         }
-        inc[d] = fmaf(ca, in_k, cbk);
-        inc[D + d] = fmaf(ca, in_v, cbv);
-        sm_in[0][d] = in_k;
-        sm_in[1][d] = in_v;
-        asm volatile("bar.sync 1, %0;" ::"n"(D));
-        if (d == 0) st_release(flags + rel, 2);
-    }
-    __syncthreads();
-
-    {
-        // ---- exclusive map inside the warp = inclusive map of the previous slice
-        float sk[CH], sv[CH];
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            float ea = __shfl_up_sync(0xffffffffu, A[c], NCG % 32);
-            float ek = __shfl_up_sync(0xffffffffu, Bk[c], NCG % 32);
-            float ev = __shfl_up_sync(0xffffffffu, Bv[c], NCG % 32);
-            if (NCG == 32 || lane < NCG) { ea = 1.0f; ek = 0.0f; ev = 0.0f; }
-            // state entering the chunk
-            const float ck = sm_in[0][cg * CH + c];
-            const float cv = sm_in[1][cg * CH + c];
-            // entering this warp, then entering this slice
-            const float wk = fmaf(Ap[c], ck, Pk[c]);
-            const float wv = fmaf(Ap[c], cv, Pv[c]);
-            sk[c] = fmaf(ea, wk, ek);
-            sv[c] = fmaf(ea, wv, ev);
+        if (warp == NW - 1) {                    // state entering the next tile
+            carry[(i + 1) & 1][0][lane] = fmaf(A, sk, Bk);
+            carry[(i + 1) & 1][1][lane] = fmaf(A, sv, Bv);
         }
 
-        // ---- apply the recurrence token by token, round, store, track bounds
-        T *kv = static_cast<T *>(a.kv);
-        float mn[CH], mx[CH];
+        // ---- pass 2: token by token, rounded rows back into the stage, bounds of the rounded keys
+        float mn = INFINITY, mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) { mn[c] = INFINITY; mx[c] = -INFINITY; }
-        const int64_t tail_end = (end + S - 1) / S * S;   // end of the last touched page
-#pragma unroll
-        for (int i = 0; i < TS; ++i) {
-            const int64_t pos = pos0 + i;
-            float kf[CH], vf[CH];
-            float gi[CH];
-            unpack16<T>(kbuf[i * NT + tid], kf);
-            unpack16<T>(vbuf[i * NT + tid], vf);
-            lds_n<G, CH>(gbuf + (size_t)(i * NT + tid) * GB, gi);
-#pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                const float om = 1.0f - gi[c];
-                sk[c] = fmaf(gi[c], sk[c], om * kf[c]);
-                sv[c] = fmaf(gi[c], sv[c], om * vf[c]);
-            }
-            const bool valid = pos >= a.len0 && pos < end;
-            const bool fill = pos >= end && pos < tail_end;   // unused slots of the last page
-            if (valid || fill) {
-                const int64_t page = pos / S;
-                const int slot = (int)(pos % S);
-                T *dst = kv + ((((int64_t)bh * a.page_cap + page) * 2) * S + slot) * D + cg * CH;
-                uint4 wk, wv;
-                if (valid) {
-                    wk = pack16<T>(sk);
-                    wv = pack16<T>(sv);
-                    float rk_[CH];
-                    unpack16<T>(wk, rk_);
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        mn[c] = fminf(mn[c], rk_[c]);
-                        mx[c] = fmaxf(mx[c], rk_[c]);
-                    }
-                } else {
-                    wk = make_uint4(0, 0, 0, 0);
-                    wv = wk;
-                }
-                *reinterpret_cast<uint4 *>(dst) = wk;
-                *reinterpret_cast<uint4 *>(dst + (int64_t)S * D) = wv;
+        for (int r = 0; r < RT; ++r) {
+            const int e = (row0 + r) * CG + lane;
+            if (row0 + r >= lo && row0 + r < hi) {
+                sk = fmaf(gg[r], sk, kk[r]);
+                sv = fmaf(gg[r], sv, vv[r]);
+                const T rk = float_to_elem<T>(sk);
+                ks[e] = rk;
+                vs[e] = float_to_elem<T>(sv);
+                const float f = elem_to_float(rk);
+                mn = fminf(mn, f);
+                mx = fmaxf(mx, f);
+            } else if (row0 + r >= hi && row0 + r < fill_hi) {   // unused slots of the last page
+                ks[e] = float_to_elem<T>(0.0f);
+                vs[e] = float_to_elem<T>(0.0f);
             }
         }
-        // the owner of the last new token leaves the fp32 state behind
-        if (end - 1 >= pos0 && end - 1 < pos0 + TS) {
-            float *st = a.state + (int64_t)bh * 2 * D;
-#pragma unroll
-            for (int c = 0; c < CH; ++c) {
-                st[cg * CH + c] = sk[c];
-                st[D + cg * CH + c] = sv[c];
-            }
-        }
-
-        // ---- page bounds: reduce the slices of each page through shared memory
-#pragma unroll
-        for (int c = 0; c < CH; ++c) {
-            mm[sl][0][cg * CH + c] = mn[c];
-            mm[sl][1][cg * CH + c] = mx[c];
+        if (WPP > 1) {
+            mm[warp][0][lane] = mn;
+            mm[warp][1][lane] = mx;
         }
         __syncthreads();
-        constexpr int SPP = S / TS;      // slices per page
-        constexpr int PPC = CT / S;      // pages per chunk
-        T *meta = static_cast<T *>(a.meta);
-        for (int idx = tid; idx < PPC * D; idx += NT) {
-            const int pg = idx / D, d = idx % D;
-            const int64_t page = chunk * PPC + pg;
-            const int64_t pstart = page * S;
-            if (pstart >= end || pstart + S <= a.len0) continue;   // no new token in this page
-            float lo = INFINITY, hi = -INFINITY;
+
+        // ---- page bounds: the first warp of a page writes them (merged with what the page held before)
+        if (warp % WPP == 0) {
+            const int64_t pstart = pos0;         // a multiple of S
+            if (pstart < end && pstart + S > a.len0) {
+                if (WPP > 1) {
 #pragma unroll
-            for (int s2 = 0; s2 < SPP; ++s2) {
-                lo = fminf(lo, mm[pg * SPP + s2][0][d]);
-                hi = fmaxf(hi, mm[pg * SPP + s2][1][d]);
+                    for (int w = 1; w < WPP; ++w) {
+                        mn = fminf(mn, mm[warp + w][0][lane]);
+                        mx = fmaxf(mx, mm[warp + w][1][lane]);
+                    }
+                }
+                T *m = meta + (((int64_t)bh * a.page_cap + pstart / S) * 2) * D + c0 + lane;
+                if (pstart < a.len0) {
+                    mn = fminf(mn, elem_to_float(m[0]));
+                    mx = fmaxf(mx, elem_to_float(m[D]));
+                }
+                m[0] = float_to_elem<T>(mn);
+                m[D] = float_to_elem<T>(mx);
             }
-            T *m = meta + (((int64_t)bh * a.page_cap + page) * 2) * D + d;
-            if (pstart < a.len0) {                                  // page already held tokens
-                lo = fminf(lo, load1<T>(m));
-                hi = fmaxf(hi, load1<T>(m + D));
-            }
-            store1<T>(m, lo);
-            store1<T>(m + D, hi);
         }
+
+        // ---- the stage's rows go out to their pages
+#pragma unroll
+        for (int j = 0; j < NCH_T / NT; ++j) {
+            const int ch = tid + j * NT, row = ch / CPR_T, cc = ch % CPR_T;
+            const int64_t pos = tile_start + row;
+            if (row >= lo && row < fill_hi) {
+                const int64_t page = pos / S;
+                const int slot = (int)(pos % S);
+                T *dst = kv + ((((int64_t)bh * a.page_cap + page) * 2) * S + slot) * D + c0 + cc * EPC_T;
+                __stcs(reinterpret_cast<uint4 *>(dst), *reinterpret_cast<const uint4 *>(ks + ch * EPC_T));
+                __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)S * D), *reinterpret_cast<const uint4 *>(vs + ch * EPC_T));
+            }
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    if (tid < CG) {                              // the state after the last token
+        a.state[(int64_t)bh * 2 * D + c0 + tid] = carry[ntiles & 1][0][tid];
+        a.state[(int64_t)bh * 2 * D + D + c0 + tid] = carry[ntiles & 1][1][tid];
     }
 }
 
 template <typename T, typename G, int D, int S>
 cudaError_t run(const ScanArgs &a, cudaStream_t s)
 {
-    constexpr int CH = VecOf<T>::N;
-    constexpr int CT = (NT / (D / CH)) * scan_ts(D, (int)sizeof(T));
     const int64_t end = a.len0 + a.T;
-    const int64_t c0 = a.len0 / CT;
-    const int64_t c1 = (end + CT - 1) / CT;
-    const int64_t nchunks = c1 - c0;
-    if (nchunks <= 0) return cudaSuccess;
-    if (nchunks > a.chunks_cap) return cudaErrorInvalidValue;
-    const int64_t ctas = nchunks * a.B * a.H;
+    const int64_t t0 = a.len0 / TT;
+    const int64_t t1 = (end + TT - 1) / TT;
+    if (t1 <= t0) return cudaSuccess;
+    if (t1 - t0 >= (int64_t)1 << 31) return cudaErrorInvalidValue;
+    const int64_t ctas = (int64_t)a.B * a.H * (D / CG);
     if (ctas >= (int64_t)1 << 31) return cudaErrorInvalidValue;
-    // the ticket counter and this call's flags start at zero
-    cudaError_t e = cudaMemsetAsync(a.ticket, 0, sizeof(int32_t), s);
-    if (e != cudaSuccess) return e;
-    e = cudaMemsetAsync(a.flags, 0, (size_t)a.B * a.H * a.chunks_cap * sizeof(int32_t), s);
-    if (e != cudaSuccess) return e;
-    constexpr int TS = scan_ts(D, (int)sizeof(T));
-    constexpr int DSM = TS * NT * (32 + CH * (int)sizeof(G));    // k, v and g slots of every thread
+    constexpr int DSM = scan_stages<T, G>() * scan_stage_bytes<T, G>();
     static bool ready[64];
     int dev = 0;
-    e = cudaGetDevice(&dev);
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
@@ -443,7 +280,7 @@ cudaError_t run(const ScanArgs &a, cudaStream_t s)
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
-    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, DSM, s>>>(a, c0);
+    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, DSM, s>>>(a, t0, (int)(t1 - t0));
     return cudaGetLastError();
 }
 

@@ -415,7 +415,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
         if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
             tau = radix_select([](uint32_t, int) { return true; }, kmin, kmax);      // range too wide for a float
         } else {
-            uint32_t bk2[ROWS / 2];                  // bucket of every key of this thread, two to a word
+            uint32_t bk2[ROWS / 2] = {};             // bucket of every key of this thread, two to a word
             auto bk = [&](int j) -> uint32_t { return (bk2[j / 2] >> (16 * (j & 1))) & 0xffffu; };
 #pragma unroll
             for (int j = 0; j < ROWS; ++j) {
