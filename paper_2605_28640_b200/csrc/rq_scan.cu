@@ -11,19 +11,25 @@
 // each stream 64-byte row segments 8 KiB apart reach the same bandwidth as a
 // plain copy, so nothing is lost by giving a CTA a quarter of a head's row.
 //
-// Inside a CTA time is cut into tiles of 128 positions that move through a
+// Inside a CTA time is cut into tiles of 256 positions that move through a
 // ring of shared-memory stages filled by asynchronous copies (several tiles
-// ahead of the arithmetic).  A warp owns 16 consecutive positions of the tile.
-// A run of tokens acts on the incoming state as the affine map s -> A s + B
-// with A = prod g and B = the run's own state from zero, and maps compose as
-// (A2,B2)o(A1,B1) = (A2 A1, A2 B1 + B2).  Per tile: every thread reduces its
-// run to a map (pass 1); after a barrier it composes the maps of the warps
-// before it onto the state that entered the tile, and the last warp leaves the
-// state for the next tile; then it applies the recurrence token by token,
-// rounds to the storage type, writes the rounded rows back into the stage and
-// tracks min/max of the rounded keys (pass 2); after a barrier the stage goes
-// out to the cache in 16-byte pieces.  The order of all floating-point
-// operations is fixed, so the result is the same bits on every run.
+// ahead of the arithmetic).  The kernel is bound by instruction issue, not by
+// memory, so the layout is chosen for few instructions per element: a lane
+// owns two neighbouring channels (one 4-byte access for a bf16 pair) and a
+// half-warp owns a run of 8 consecutive positions of the tile.  A run of tokens acts on the
+// incoming state as the affine map s -> A s + B with A = prod g and B = the
+// run's own state from zero, and maps compose as (A2,B2)o(A1,B1) = (A2 A1,
+// A2 B1 + B2).  Per tile: every thread reduces its run to a map (pass 1) and
+// the two runs of a warp are composed by shuffles; after a barrier the 16
+// warp maps of every channel are scanned by 16 lanes (warp w takes channels
+// 2w and 2w+1), which gives the state entering every warp and the state
+// entering the next tile; after a barrier every thread applies the recurrence
+// token by token, rounds to the storage type, writes the rounded rows back
+// into the stage and tracks min/max of the rounded keys (pass 2); after a
+// barrier the stage goes out to the cache in 16-byte pieces.  Tiles that lie
+// wholly inside the new tokens take a path without per-row range checks.  The
+// order of all floating-point operations is fixed, so the result is the same
+// bits on every run.
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
@@ -32,11 +38,16 @@ namespace rq {
 
 namespace {
 
+
 constexpr int NT = kScanThreads;
 constexpr int NW = NT / 32;
-constexpr int CG = kScanChannels;               // channels of one CTA: a lane per channel
-constexpr int RT = kScanRunTokens;              // consecutive positions of one warp in a tile
-constexpr int TT = NW * RT;                     // positions of one tile
+constexpr int CG = kScanChannels;               // channels of one CTA: two per lane of a half-warp
+constexpr int RT = kScanRunTokens;              // consecutive positions of one half-warp in a tile
+constexpr int TT = 2 * NW * RT;                 // positions of one tile
+constexpr int kMapStride = 3 * CG + 2;          // floats between two warps' maps: an even count, and lanes that read
+                                                // the same channel of 16 consecutive maps hit 16 different banks
+constexpr int kInStride = 2 * CG + 2;           // likewise for the states entering the warps
+static_assert(CG == 32 && NW == 16, "a half-warp holds a channel group two channels per lane; 16 warp maps are scanned by 16 lanes");
 
 // asynchronous copy of 16 bytes from global to shared memory
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
@@ -46,18 +57,40 @@ __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ float elem_to_float(bf16 x) { return __bfloat162float(x); }
-__device__ __forceinline__ float elem_to_float(float x) { return x; }
-template <typename T> __device__ __forceinline__ T float_to_elem(float x);
-template <> __device__ __forceinline__ bf16 float_to_elem<bf16>(float x) { return __float2bfloat16_rn(x); }
-template <> __device__ __forceinline__ float float_to_elem<float>(float x) { return x; }
+// two neighbouring elements from shared memory as floats
+__device__ __forceinline__ void load2(const bf16 *p, float &x, float &y)
+{
+    const uint32_t w = *reinterpret_cast<const uint32_t *>(p);
+    x = bf16lo(w);
+    y = bf16hi(w);
+}
+__device__ __forceinline__ void load2(const float *p, float &x, float &y)
+{
+    const float2 w = *reinterpret_cast<const float2 *>(p);
+    x = w.x;
+    y = w.y;
+}
+// round two floats to the storage type, store them side by side, return the stored values
+__device__ __forceinline__ void store2(bf16 *p, float &x, float &y)
+{
+    const uint32_t w = pack_bf16(x, y);
+    *reinterpret_cast<uint32_t *>(p) = w;
+    x = bf16lo(w);
+    y = bf16hi(w);
+}
+__device__ __forceinline__ void store2(float *p, float &x, float &y) { *reinterpret_cast<float2 *>(p) = make_float2(x, y); }
+
+template <bool B> struct BoolTag { static constexpr bool value = B; };
 
 // bytes of one ring stage: the k, v and g segments of a tile
-template <typename T, typename G> __host__ __device__ constexpr int scan_stage_bytes() { return TT * CG * (2 * (int)sizeof(T) + (int)sizeof(G)); }
-// stages of the ring: as many as fit in 192 KiB, at most six
+template <typename T, typename G> __host__ __device__ constexpr int scan_stage_bytes()
+{
+    return TT * CG * (2 * (int)sizeof(T) + (int)sizeof(G));
+}
+// stages of the ring: as many as fit in 192 KiB, at most four
 template <typename T, typename G> __host__ __device__ constexpr int scan_stages()
 {
-    return 192 * 1024 / scan_stage_bytes<T, G>() < 6 ? 192 * 1024 / scan_stage_bytes<T, G>() : 6;
+    return 192 * 1024 / scan_stage_bytes<T, G>() < 4 ? 192 * 1024 / scan_stage_bytes<T, G>() : 4;
 }
 
 template <typename T, typename G, int D, int S>
@@ -68,18 +101,22 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
     constexpr int EPC_T = 16 / (int)sizeof(T), EPC_G = 16 / (int)sizeof(G);   // elements per 16-byte piece
     constexpr int CPR_T = CG / EPC_T, CPR_G = CG / EPC_G;                      // pieces per row segment
     constexpr int NCH_T = TT * CPR_T, NCH_G = TT * CPR_G;                      // pieces per tile
-    constexpr int WPP = S / RT;                                                // warps that share a page
+    constexpr int WPP = S / (2 * RT);                                          // warps that share a page
+    constexpr unsigned FULLMASK = 0xffffffffu;
     static_assert(D % CG == 0, "a head is a whole number of channel groups");
-    static_assert(S % RT == 0 && TT % S == 0 && NW % WPP == 0, "a page is a whole number of warp runs inside one tile");
+    static_assert(S % (2 * RT) == 0 && TT % S == 0 && NW % WPP == 0, "a page is a whole number of warps inside one tile");
     static_assert(NCH_T % NT == 0 && NCH_G % NT == 0, "every thread moves the same number of pieces");
     static_assert(NST >= 2, "the ring needs two stages");
 
     extern __shared__ __align__(16) unsigned char dsm[];
-    __shared__ float wmap[NW][3][CG];            // the warps' maps of the current tile
-    __shared__ float carry[2][2][CG];            // state entering the tile (by tile parity): k, v
-    __shared__ float mm[NW][2][CG];              // min / max of the warps' runs (pages wider than a run)
+    __shared__ __align__(8) float wmap[NW * kMapStride];    // the warps' maps of the current tile: [warp][A, Bk, Bv][channel]
+    __shared__ __align__(8) float sin_[NW * kInStride];     // state entering every warp: [warp][k, v][channel]
+    __shared__ float carry[2][2][CG];                       // state entering the tile (by tile parity): k, v
+    __shared__ float mm[NW][2][CG];                         // min / max of the warps (pages wider than a warp's 16 positions)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int hl = lane & 15, half = lane >> 4;  // channel pair of this lane; which of the warp's two runs
+    const int ch2 = 2 * hl;                      // first of this lane's two channels inside the group
     constexpr int GPH = D / CG;                  // channel groups per head
     const int bh = blockIdx.x / GPH, c0 = (blockIdx.x % GPH) * CG;
     const int b = bh / a.H, h = bh % a.H;
@@ -130,110 +167,141 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
     T *kv = static_cast<T *>(a.kv);
     T *meta = static_cast<T *>(a.meta);
 
-#pragma unroll 1
-    for (int i = 0; i < ntiles; ++i) {
+    // one tile; FULL: every row of the tile is a new token, so no row needs a range check
+    auto tile = [&](auto full_tag, int i, int lo, int hi, int fill_hi) {
+        constexpr bool FULL = decltype(full_tag)::value;
         const int st = i % NST;
-        cp_async_wait<NST - 2>();                // this thread's pieces of tile i have landed ...
-        __syncthreads();                         // ... and everybody else's; the stage of tile i - 1 has gone out
-        if (i + NST - 1 < ntiles) issue(i + NST - 1, (i + NST - 1) % NST);
-        cp_async_commit();
-
         T *ks = stage_k(st), *vs = stage_v(st);
         const G *gs = stage_g(st);
-        const int row0 = warp * RT;
+        const int row0 = (2 * warp + half) * RT;
         const int64_t tile_start = (tile0 + i) * TT;
-        const int64_t pos0 = tile_start + row0;
-        // rows of the tile that hold new tokens: [lo, hi); rows up to fill_hi pad the last page
-        const int lo = (int)max((int64_t)0, a.len0 - tile_start), hi = (int)min((int64_t)TT, end - tile_start);
-        const int fill_hi = (int)min((int64_t)TT, tail_end - tile_start);
 
         // ---- pass 1: this thread's run as a map from a zero state (identity outside the new range)
-        float gg[RT], kk[RT], vv[RT];            // g, (1-g) k, (1-g) v
-        float A = 1.0f, Bk = 0.0f, Bv = 0.0f;
+        float g0[RT], g1[RT], k0[RT], k1[RT], v0[RT], v1[RT];    // g, (1-g) k, (1-g) v of the two channels
+        float A0 = 1.0f, A1 = 1.0f, Bk0 = 0.0f, Bk1 = 0.0f, Bv0 = 0.0f, Bv1 = 0.0f;
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
-            const bool valid = row0 + r >= lo && row0 + r < hi;
-            const int e = (row0 + r) * CG + lane;
-            const float g = valid ? elem_to_float(gs[e]) : 1.0f;
-            const float om = 1.0f - g;
-            gg[r] = g;
-            kk[r] = valid ? om * elem_to_float(ks[e]) : 0.0f;
-            vv[r] = valid ? om * elem_to_float(vs[e]) : 0.0f;
-            A *= g;
-            Bk = fmaf(g, Bk, kk[r]);
-            Bv = fmaf(g, Bv, vv[r]);
+            const int e = (row0 + r) * CG + ch2;
+            float ga, gb, ka, kb, va, vb;
+            load2(gs + e, ga, gb);
+            load2(ks + e, ka, kb);
+            load2(vs + e, va, vb);
+            if (!FULL && !(row0 + r >= lo && row0 + r < hi)) {
+                ga = 1.0f; gb = 1.0f;
+                ka = 0.0f; kb = 0.0f;
+                va = 0.0f; vb = 0.0f;
+            }
+            const float oa = 1.0f - ga, ob = 1.0f - gb;
+            g0[r] = ga; g1[r] = gb;
+            k0[r] = oa * ka; k1[r] = ob * kb;
+            v0[r] = oa * va; v1[r] = ob * vb;
+            A0 *= ga; A1 *= gb;
+            Bk0 = fmaf(ga, Bk0, k0[r]); Bk1 = fmaf(gb, Bk1, k1[r]);
+            Bv0 = fmaf(ga, Bv0, v0[r]); Bv1 = fmaf(gb, Bv1, v1[r]);
         }
-        wmap[warp][0][lane] = A;
-        wmap[warp][1][lane] = Bk;
-        wmap[warp][2][lane] = Bv;
+        // the map of the warp's first run, for the second run; the second run's lanes publish the warp's map
+        const float LA0 = __shfl_sync(FULLMASK, A0, hl), LA1 = __shfl_sync(FULLMASK, A1, hl);
+        const float LBk0 = __shfl_sync(FULLMASK, Bk0, hl), LBk1 = __shfl_sync(FULLMASK, Bk1, hl);
+        const float LBv0 = __shfl_sync(FULLMASK, Bv0, hl), LBv1 = __shfl_sync(FULLMASK, Bv1, hl);
+        if (half == 1) {
+            float *wm = wmap + warp * kMapStride + ch2;
+            *reinterpret_cast<float2 *>(wm) = make_float2(A0 * LA0, A1 * LA1);
+            *reinterpret_cast<float2 *>(wm + CG) = make_float2(fmaf(A0, LBk0, Bk0), fmaf(A1, LBk1, Bk1));
+            *reinterpret_cast<float2 *>(wm + 2 * CG) = make_float2(fmaf(A0, LBv0, Bv0), fmaf(A1, LBv1, Bv1));
+        }
         __syncthreads();
 
-        // ---- state entering this run: the tile's incoming state through the maps of the warps before
-        float sk = carry[i & 1][0][lane], sv = carry[i & 1][1][lane];
+        // ---- scan of the 16 warp maps of channels 2 warp and 2 warp + 1 (one per half-warp) by 16 lanes
         {
-            float wa[NW - 1], wk[NW - 1], wv[NW - 1];   // all loads first: only the multiply-adds form a chain
+            const int ci = 2 * warp + half, m = hl;          // channel inside the group, map (= warp) index
+            const float *wm = wmap + m * kMapStride + ci;
+            float sa = wm[0], sbk = wm[CG], sbv = wm[2 * CG];
 #pragma unroll
-            for (int w = 0; w < NW - 1; ++w) {
-                wa[w] = wmap[w][0][lane];
-                wk[w] = wmap[w][1][lane];
-                wv[w] = wmap[w][2][lane];
-            }
-#pragma unroll
-            for (int w = 0; w < NW - 1; ++w) {
-                if (w < warp) {
-                    sk = fmaf(wa[w], sk, wk[w]);
-                    sv = fmaf(wa[w], sv, wv[w]);
+            for (int off = 1; off < 16; off <<= 1) {
+                const float pa = __shfl_up_sync(FULLMASK, sa, off, 16);
+                const float pbk = __shfl_up_sync(FULLMASK, sbk, off, 16);
+                const float pbv = __shfl_up_sync(FULLMASK, sbv, off, 16);
+                if (m >= off) {
+                    sbk = fmaf(sa, pbk, sbk);
+                    sbv = fmaf(sa, pbv, sbv);
+                    sa *= pa;
                 }
             }
-        }
-        if (warp == NW - 1) {                    // state entering the next tile
-            carry[(i + 1) & 1][0][lane] = fmaf(A, sk, Bk);
-            carry[(i + 1) & 1][1][lane] = fmaf(A, sv, Bv);
-        }
-
-        // ---- pass 2: token by token, rounded rows back into the stage, bounds of the rounded keys
-        float mn = INFINITY, mx = -INFINITY;
-#pragma unroll
-        for (int r = 0; r < RT; ++r) {
-            const int e = (row0 + r) * CG + lane;
-            if (row0 + r >= lo && row0 + r < hi) {
-                sk = fmaf(gg[r], sk, kk[r]);
-                sv = fmaf(gg[r], sv, vv[r]);
-                const T rk = float_to_elem<T>(sk);
-                ks[e] = rk;
-                vs[e] = float_to_elem<T>(sv);
-                const float f = elem_to_float(rk);
-                mn = fminf(mn, f);
-                mx = fmaxf(mx, f);
-            } else if (row0 + r >= hi && row0 + r < fill_hi) {   // unused slots of the last page
-                ks[e] = float_to_elem<T>(0.0f);
-                vs[e] = float_to_elem<T>(0.0f);
+            float ea = __shfl_up_sync(FULLMASK, sa, 1, 16);  // maps of the warps before this one
+            float ebk = __shfl_up_sync(FULLMASK, sbk, 1, 16);
+            float ebv = __shfl_up_sync(FULLMASK, sbv, 1, 16);
+            if (m == 0) { ea = 1.0f; ebk = 0.0f; ebv = 0.0f; }
+            const float ck = carry[i & 1][0][ci], cv = carry[i & 1][1][ci];
+            sin_[m * kInStride + ci] = fmaf(ea, ck, ebk);
+            sin_[m * kInStride + CG + ci] = fmaf(ea, cv, ebv);
+            if (m == 15) {                                   // state entering the next tile
+                carry[(i + 1) & 1][0][ci] = fmaf(sa, ck, sbk);
+                carry[(i + 1) & 1][1][ci] = fmaf(sa, cv, sbv);
             }
         }
-        if (WPP > 1) {
-            mm[warp][0][lane] = mn;
-            mm[warp][1][lane] = mx;
+        __syncthreads();
+
+        // ---- pass 2: token by token, rounded rows back into the stage, bounds of the rounded keys
+        float sk0, sk1, sv0, sv1;
+        {
+            const float2 ek = *reinterpret_cast<const float2 *>(sin_ + warp * kInStride + ch2);
+            const float2 ev = *reinterpret_cast<const float2 *>(sin_ + warp * kInStride + CG + ch2);
+            sk0 = ek.x; sk1 = ek.y; sv0 = ev.x; sv1 = ev.y;
+            if (half == 1) {                                 // through the warp's first run
+                sk0 = fmaf(LA0, sk0, LBk0); sk1 = fmaf(LA1, sk1, LBk1);
+                sv0 = fmaf(LA0, sv0, LBv0); sv1 = fmaf(LA1, sv1, LBv1);
+            }
+        }
+        float mn0 = INFINITY, mn1 = INFINITY, mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int r = 0; r < RT; ++r) {
+            const int e = (row0 + r) * CG + ch2;
+            if (FULL || (row0 + r >= lo && row0 + r < hi)) {
+                sk0 = fmaf(g0[r], sk0, k0[r]); sk1 = fmaf(g1[r], sk1, k1[r]);
+                sv0 = fmaf(g0[r], sv0, v0[r]); sv1 = fmaf(g1[r], sv1, v1[r]);
+                float rk0 = sk0, rk1 = sk1, rv0 = sv0, rv1 = sv1;
+                store2(ks + e, rk0, rk1);
+                store2(vs + e, rv0, rv1);
+                mn0 = fminf(mn0, rk0); mx0 = fmaxf(mx0, rk0);
+                mn1 = fminf(mn1, rk1); mx1 = fmaxf(mx1, rk1);
+            } else if (row0 + r >= hi && row0 + r < fill_hi) {   // unused slots of the last page
+                float z0 = 0.0f, z1 = 0.0f;
+                store2(ks + e, z0, z1);
+                store2(vs + e, z0, z1);
+            }
+        }
+        // the warp's two runs together (16 positions)
+        mn0 = fminf(mn0, __shfl_xor_sync(FULLMASK, mn0, 16)); mn1 = fminf(mn1, __shfl_xor_sync(FULLMASK, mn1, 16));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(FULLMASK, mx0, 16)); mx1 = fmaxf(mx1, __shfl_xor_sync(FULLMASK, mx1, 16));
+        if (WPP > 1 && half == 0) {
+            *reinterpret_cast<float2 *>(&mm[warp][0][ch2]) = make_float2(mn0, mn1);
+            *reinterpret_cast<float2 *>(&mm[warp][1][ch2]) = make_float2(mx0, mx1);
         }
         __syncthreads();
 
         // ---- page bounds: the first warp of a page writes them (merged with what the page held before)
-        if (warp % WPP == 0) {
-            const int64_t pstart = pos0;         // a multiple of S
+        if (warp % WPP == 0 && half == 0) {
+            const int64_t pstart = tile_start + 2 * warp * RT;   // a multiple of S
             if (pstart < end && pstart + S > a.len0) {
                 if (WPP > 1) {
 #pragma unroll
                     for (int w = 1; w < WPP; ++w) {
-                        mn = fminf(mn, mm[warp + w][0][lane]);
-                        mx = fmaxf(mx, mm[warp + w][1][lane]);
+                        const float2 lo2 = *reinterpret_cast<const float2 *>(&mm[warp + w][0][ch2]);
+                        const float2 hi2 = *reinterpret_cast<const float2 *>(&mm[warp + w][1][ch2]);
+                        mn0 = fminf(mn0, lo2.x); mn1 = fminf(mn1, lo2.y);
+                        mx0 = fmaxf(mx0, hi2.x); mx1 = fmaxf(mx1, hi2.y);
                     }
                 }
-                T *m = meta + (((int64_t)bh * a.page_cap + pstart / S) * 2) * D + c0 + lane;
+                T *mrow = meta + (((int64_t)bh * a.page_cap + pstart / S) * 2) * D + c0 + ch2;
                 if (pstart < a.len0) {
-                    mn = fminf(mn, elem_to_float(m[0]));
-                    mx = fmaxf(mx, elem_to_float(m[D]));
+                    float o0, o1;
+                    load2(mrow, o0, o1);
+                    mn0 = fminf(mn0, o0); mn1 = fminf(mn1, o1);
+                    load2(mrow + D, o0, o1);
+                    mx0 = fmaxf(mx0, o0); mx1 = fmaxf(mx1, o1);
                 }
-                m[0] = float_to_elem<T>(mn);
-                m[D] = float_to_elem<T>(mx);
+                store2(mrow, mn0, mn1);
+                store2(mrow + D, mx0, mx1);
             }
         }
 
@@ -242,7 +310,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
         for (int j = 0; j < NCH_T / NT; ++j) {
             const int ch = tid + j * NT, row = ch / CPR_T, cc = ch % CPR_T;
             const int64_t pos = tile_start + row;
-            if (row >= lo && row < fill_hi) {
+            if (FULL || (row >= lo && row < fill_hi)) {
                 const int64_t page = pos / S;
                 const int slot = (int)(pos % S);
                 T *dst = kv + ((((int64_t)bh * a.page_cap + page) * 2) * S + slot) * D + c0 + cc * EPC_T;
@@ -250,6 +318,20 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
                 __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)S * D), *reinterpret_cast<const uint4 *>(vs + ch * EPC_T));
             }
         }
+    };
+
+#pragma unroll 1
+    for (int i = 0; i < ntiles; ++i) {
+        cp_async_wait<NST - 2>();                // this thread's pieces of tile i have landed ...
+        __syncthreads();                         // ... and everybody else's; the stage of tile i - 1 has gone out
+        if (i + NST - 1 < ntiles) issue(i + NST - 1, (i + NST - 1) % NST);
+        cp_async_commit();
+        // rows of the tile that hold new tokens: [lo, hi); rows up to fill_hi pad the last page
+        const int64_t tile_start = (tile0 + i) * TT;
+        const int lo = (int)max((int64_t)0, a.len0 - tile_start), hi = (int)min((int64_t)TT, end - tile_start);
+        const int fill_hi = (int)min((int64_t)TT, tail_end - tile_start);
+        if (lo == 0 && hi == TT) tile(BoolTag<true>(), i, lo, hi, fill_hi);
+        else tile(BoolTag<false>(), i, lo, hi, fill_hi);
     }
     cp_async_wait<0>();
     __syncthreads();
