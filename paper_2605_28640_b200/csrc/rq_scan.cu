@@ -47,7 +47,8 @@ constexpr int TT = 2 * NW * RT;                 // positions of one tile
 constexpr int kMapStride = 3 * CG + 2;          // floats between two warps' maps: an even count, and lanes that read
                                                 // the same channel of 16 consecutive maps hit 16 different banks
 constexpr int kInStride = 2 * CG + 2;           // likewise for the states entering the warps
-static_assert(CG == 32 && NW == 16, "a half-warp holds a channel group two channels per lane; 16 warp maps are scanned by 16 lanes");
+constexpr int LPC = NW;                         // lanes that scan the warp maps of one channel
+static_assert(CG == 32 && (NW == 16 || NW == 32), "a half-warp holds a channel group two channels per lane; the warp maps of a channel are scanned by 16 or 32 lanes");
 
 // asynchronous copy of 16 bytes from global to shared memory
 __device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
@@ -79,6 +80,15 @@ __device__ __forceinline__ void store2(bf16 *p, float &x, float &y)
     y = bf16hi(w);
 }
 __device__ __forceinline__ void store2(float *p, float &x, float &y) { *reinterpret_cast<float2 *>(p) = make_float2(x, y); }
+
+// Where a row's segment sits in its tile.  With 2-byte elements a segment is 64 bytes, two rows to
+// a 128-byte line, and the two half-warps of a warp read rows 8 apart, which would be the same 16
+// banks: rows whose bit 3 is set swap places with their neighbour, so the two rows land in
+// different halves of their lines.
+template <typename X> __device__ __forceinline__ int row_slot(int row)
+{
+    return sizeof(X) == 2 ? row ^ ((row >> 3) & 1) : row;
+}
 
 template <bool B> struct BoolTag { static constexpr bool value = B; };
 
@@ -143,14 +153,16 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
             const int ch = tid + i * NT, row = ch / CPR_T, cc = ch % CPR_T;
             if (row >= lo && row < hi) {
                 const int64_t src = (tok0 + row) * a.st + cc * EPC_T;
-                cp_async16(ks + ch * EPC_T, kp + src);
-                cp_async16(vs + ch * EPC_T, vp + src);
+                const int dst = row_slot<T>(row) * CG + cc * EPC_T;
+                cp_async16(ks + dst, kp + src);
+                cp_async16(vs + dst, vp + src);
             }
         }
 #pragma unroll
         for (int i = 0; i < NCH_G / NT; ++i) {
             const int ch = tid + i * NT, row = ch / CPR_G, cc = ch % CPR_G;
-            if (row >= lo && row < hi) cp_async16(gs + ch * EPC_G, gp + (tok0 + row) * a.st + cc * EPC_G);
+            if (row >= lo && row < hi)
+                cp_async16(gs + row_slot<G>(row) * CG + cc * EPC_G, gp + (tok0 + row) * a.st + cc * EPC_G);
         }
     };
 
@@ -181,9 +193,9 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
         float A0 = 1.0f, A1 = 1.0f, Bk0 = 0.0f, Bk1 = 0.0f, Bv0 = 0.0f, Bv1 = 0.0f;
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
-            const int e = (row0 + r) * CG + ch2;
+            const int e = row_slot<T>(row0 + r) * CG + ch2;
             float ga, gb, ka, kb, va, vb;
-            load2(gs + e, ga, gb);
+            load2(gs + row_slot<G>(row0 + r) * CG + ch2, ga, gb);
             load2(ks + e, ka, kb);
             load2(vs + e, va, vb);
             if (!FULL && !(row0 + r >= lo && row0 + r < hi)) {
@@ -213,28 +225,28 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
 
         // ---- scan of the 16 warp maps of channels 2 warp and 2 warp + 1 (one per half-warp) by 16 lanes
         {
-            const int ci = 2 * warp + half, m = hl;          // channel inside the group, map (= warp) index
+            const int ci = warp * (32 / LPC) + lane / LPC, m = lane % LPC;   // channel inside the group, map (= warp) index
             const float *wm = wmap + m * kMapStride + ci;
             float sa = wm[0], sbk = wm[CG], sbv = wm[2 * CG];
 #pragma unroll
-            for (int off = 1; off < 16; off <<= 1) {
-                const float pa = __shfl_up_sync(FULLMASK, sa, off, 16);
-                const float pbk = __shfl_up_sync(FULLMASK, sbk, off, 16);
-                const float pbv = __shfl_up_sync(FULLMASK, sbv, off, 16);
+            for (int off = 1; off < LPC; off <<= 1) {
+                const float pa = __shfl_up_sync(FULLMASK, sa, off, LPC);
+                const float pbk = __shfl_up_sync(FULLMASK, sbk, off, LPC);
+                const float pbv = __shfl_up_sync(FULLMASK, sbv, off, LPC);
                 if (m >= off) {
                     sbk = fmaf(sa, pbk, sbk);
                     sbv = fmaf(sa, pbv, sbv);
                     sa *= pa;
                 }
             }
-            float ea = __shfl_up_sync(FULLMASK, sa, 1, 16);  // maps of the warps before this one
-            float ebk = __shfl_up_sync(FULLMASK, sbk, 1, 16);
-            float ebv = __shfl_up_sync(FULLMASK, sbv, 1, 16);
+            float ea = __shfl_up_sync(FULLMASK, sa, 1, LPC);  // maps of the warps before this one
+            float ebk = __shfl_up_sync(FULLMASK, sbk, 1, LPC);
+            float ebv = __shfl_up_sync(FULLMASK, sbv, 1, LPC);
             if (m == 0) { ea = 1.0f; ebk = 0.0f; ebv = 0.0f; }
             const float ck = carry[i & 1][0][ci], cv = carry[i & 1][1][ci];
             sin_[m * kInStride + ci] = fmaf(ea, ck, ebk);
             sin_[m * kInStride + CG + ci] = fmaf(ea, cv, ebv);
-            if (m == 15) {                                   // state entering the next tile
+            if (m == LPC - 1) {                              // state entering the next tile
                 carry[(i + 1) & 1][0][ci] = fmaf(sa, ck, sbk);
                 carry[(i + 1) & 1][1][ci] = fmaf(sa, cv, sbv);
             }
@@ -255,7 +267,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
         float mn0 = INFINITY, mn1 = INFINITY, mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
-            const int e = (row0 + r) * CG + ch2;
+            const int e = row_slot<T>(row0 + r) * CG + ch2;
             if (FULL || (row0 + r >= lo && row0 + r < hi)) {
                 sk0 = fmaf(g0[r], sk0, k0[r]); sk1 = fmaf(g1[r], sk1, k1[r]);
                 sv0 = fmaf(g0[r], sv0, v0[r]); sv1 = fmaf(g1[r], sv1, v1[r]);
@@ -314,8 +326,9 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
                 const int64_t page = pos / S;
                 const int slot = (int)(pos % S);
                 T *dst = kv + ((((int64_t)bh * a.page_cap + page) * 2) * S + slot) * D + c0 + cc * EPC_T;
-                __stcs(reinterpret_cast<uint4 *>(dst), *reinterpret_cast<const uint4 *>(ks + ch * EPC_T));
-                __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)S * D), *reinterpret_cast<const uint4 *>(vs + ch * EPC_T));
+                const int src = row_slot<T>(row) * CG + cc * EPC_T;
+                __stcs(reinterpret_cast<uint4 *>(dst), *reinterpret_cast<const uint4 *>(ks + src));
+                __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)S * D), *reinterpret_cast<const uint4 *>(vs + src));
             }
         }
     };
