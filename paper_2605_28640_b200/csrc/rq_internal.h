@@ -8,7 +8,7 @@
 
 namespace rq {
 
-// ---- geometry of the prefill scan (must agree between sizing and launch) ----
+// ---- geometry of the prefill kernel ----
 constexpr int kScanThreads = 512;  // threads per CTA
 
 constexpr int kScanChannels = 32;   // channels of one prefill CTA (a lane per channel)
