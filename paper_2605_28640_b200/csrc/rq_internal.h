@@ -11,8 +11,8 @@ namespace rq {
 // ---- geometry of the prefill kernel ----
 constexpr int kScanThreads = 512;  // threads per CTA
 
-constexpr int kScanChannels = 32;   // channels of one prefill CTA (a lane per channel)
-constexpr int kScanRunTokens = 8;   // consecutive positions that one warp of a prefill CTA owns in a tile
+constexpr int kScanChannels = 32;   // channels of one prefill CTA (two per lane of a half-warp)
+constexpr int kScanRunTokens = 8;   // consecutive positions that one half-warp of a prefill CTA owns in a tile
 
 // ---- decode-side geometry ----
 constexpr int kScoreWarps = 4;         // warps per scoring CTA, each with its own copy pipeline
