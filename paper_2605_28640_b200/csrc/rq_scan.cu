@@ -25,8 +25,8 @@
 // 2w and 2w+1), which gives the state entering every warp and the state
 // entering the next tile; after a barrier every thread applies the recurrence
 // token by token, rounds to the storage type, writes the rounded rows back
-// into the stage and tracks min/max of the rounded keys (pass 2); after a
-// barrier the stage goes out to the cache in 16-byte pieces.  Tiles that lie
+// into the stage and tracks min/max of the rounded keys (pass 2); then every
+// warp sends its own rows out to the cache in 16-byte pieces.  Tiles that lie
 // wholly inside the new tokens take a path without per-row range checks.  The
 // order of all floating-point operations is fixed, so the result is the same
 // bits on every run.
@@ -289,7 +289,8 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
             *reinterpret_cast<float2 *>(&mm[warp][0][ch2]) = make_float2(mn0, mn1);
             *reinterpret_cast<float2 *>(&mm[warp][1][ch2]) = make_float2(mx0, mx1);
         }
-        __syncthreads();
+        if (WPP > 1) __syncthreads();            // pages wider than a warp's rows: the bounds cross warps
+        else __syncwarp();                       // the rows below were written by other lanes of this warp
 
         // ---- page bounds: the first warp of a page writes them (merged with what the page held before)
         if (warp % WPP == 0 && half == 0) {
@@ -317,10 +318,12 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
             }
         }
 
-        // ---- the stage's rows go out to their pages
+        // ---- the warp's own rows go out to their pages (no other warp touches them: no CTA barrier)
+        constexpr int WROWS = 2 * RT;            // rows of a warp
+        static_assert((WROWS * CPR_T) % 32 == 0, "every lane moves the same number of pieces");
 #pragma unroll
-        for (int j = 0; j < NCH_T / NT; ++j) {
-            const int ch = tid + j * NT, row = ch / CPR_T, cc = ch % CPR_T;
+        for (int j = 0; j < WROWS * CPR_T / 32; ++j) {
+            const int ch = lane + j * 32, row = warp * WROWS + ch / CPR_T, cc = ch % CPR_T;
             const int64_t pos = tile_start + row;
             if (FULL || (row >= lo && row < fill_hi)) {
                 const int64_t page = pos / S;
@@ -336,7 +339,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
 #pragma unroll 1
     for (int i = 0; i < ntiles; ++i) {
         cp_async_wait<NST - 2>();                // this thread's pieces of tile i have landed ...
-        __syncthreads();                         // ... and everybody else's; the stage of tile i - 1 has gone out
+        __syncthreads();                         // ... and everybody else's; every warp has sent its rows of tile i - 1
         if (i + NST - 1 < ntiles) issue(i + NST - 1, (i + NST - 1) % NST);
         cp_async_commit();
         // rows of the tile that hold new tokens: [lo, hi); rows up to fill_hi pad the last page
