@@ -115,3 +115,17 @@ def test_config4_needles_128k(den):
     hit = sum(len(set(planted[b, h].tolist()) & set(sel[b, h].tolist())) for b in range(w.B) for h in range(w.H))
     recall = hit / (w.B * w.H * w.needles)
     assert recall >= 0.9, f"recall of planted pages {recall:.3f}"
+
+
+@pytest.mark.parametrize("T", [16384 * 16 + 40, 32768 * 16 - 9])
+def test_long_context_selection_paths(T):
+    """Heads of more than 16384 pages are selected with the keys in shared memory instead of registers;
+    32768 pages is the largest head the selection supports.  One head pair of a narrow model keeps the
+    oracle's work small."""
+    w = wl.Workload("long", B=1, H=2, D=64, T=T, budget_num=1, budget_den=32, seed=77)
+    heads = [(0, 0), (0, 1)]
+    cache, ohs = build(w, T - 1, T + 4, heads, maxK=w.budget_pages(T) + 1)
+    stats = {}
+    decode_and_check(w, cache, ohs, 0, w.budget_pages(T), stats, check_cache=False)
+    assert stats["heads"] == 2
+    assert stats.get("near_tie_mismatch", 0) <= stats.get("near_tie", 0)
