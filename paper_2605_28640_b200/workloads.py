@@ -39,6 +39,7 @@ class Workload:
     steps: int = 1         # consecutive decode steps
     resets: bool = False
     needles: int = 0
+    gate_zero: bool = False   # g = 0 everywhere: the cache holds k and v themselves (Eq. 2's paired baseline)
 
     @property
     def gdtype(self):
@@ -83,7 +84,7 @@ def make_token(w: Workload, device, step=0):
     k = torch.randn(w.B, w.H, w.D, generator=_gen(device, w.seed, 11 + 4 * step), device=device)
     v = torch.randn(w.B, w.H, w.D, generator=_gen(device, w.seed, 12 + 4 * step), device=device)
     x = torch.randn(w.B, w.H, w.D, generator=_gen(device, w.seed, 13 + 4 * step), device=device)
-    g = torch.sigmoid(4.12 + 0.5 * x)
+    g = torch.zeros_like(x) if w.gate_zero else torch.sigmoid(4.12 + 0.5 * x)
     return k.to(w.dtype), v.to(w.dtype), g.to(w.gdtype)
 
 
@@ -131,6 +132,8 @@ def make_prefill(w: Workload, device, T=None, q_for_needles=None):
         if w.resets:
             hit = (torch.rand(T, generator=reset_gen) < 0.01).to(device)
             gb[hit] = 0.5
+        if w.gate_zero:
+            gb.zero_()
         g[b] = gb.to(w.gdtype)
         del gb
     return k, v, g
