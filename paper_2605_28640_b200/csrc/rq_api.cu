@@ -112,7 +112,7 @@ static int select_into(const rq_cache *c, int64_t len, const void *q, const void
     int32_t *ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
     if (launch_score(a, q, k_t, v_t, g_t, scores, ctr + 3, do_update, sm_count(), s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 1, s);
-    if (launch_topk(a, scores, budget, idx, idx_stride, ctr, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (launch_topk(a, scores, budget, idx, idx_stride, ctr, do_update, s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 2, s);
     return RQ_OK;
 }

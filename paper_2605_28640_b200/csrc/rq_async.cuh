@@ -92,6 +92,13 @@ __device__ __forceinline__ void bulk_g2s_hint(void *dst_smem, const void *src_gm
         : "memory");
 }
 
+// Start bringing `bytes` (a multiple of 16, from a 16-byte aligned address) of global memory into L2;
+// nothing waits for it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src_gmem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
+}
+
 // Programmatic dependent launch: wait until the kernels this one depends on
 // have completed and their writes are visible (no-op without the attribute).
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

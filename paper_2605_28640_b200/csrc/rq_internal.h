@@ -22,6 +22,7 @@ constexpr int kAttendRingBytes = 64 * 1024;  // shared-memory ring of one flash-
 constexpr int kAttendMaxWarps = 2048;  // upper bound of the warps of a flash-decode grid
 constexpr int kCtrStride = 64;         // int32 between the counters of two heads (256 bytes: different L2 lines)
 constexpr int kTopkThreads = 1024;     // threads of the selection CTA
+constexpr int64_t kTopkPrefetchBytes = 16ll << 20;   // selected pages the selection kernel sends towards L2, all heads together
 constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
 constexpr int kTargetSMs = 148;        // B200
 
@@ -64,8 +65,9 @@ struct DecodeArgs {
 cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
                          float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s);
 // attend_ctr: the ticket counters of the streaming kernels (cleared here, one head per CTA)
+// prefetch: the flash-decode kernel runs next, start moving the first selected pages into L2
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, int32_t *attend_ctr, cudaStream_t s);
+                        int idx_stride, int32_t *attend_ctr, int prefetch, cudaStream_t s);
 // per-head counters of the flash-decode kernel, kCtrStride int32 apart from head to head; all
 // zero at launch
 struct AttendCounters {

@@ -43,7 +43,8 @@ __device__ __forceinline__ float key_value(uint32_t k)
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
                                                             int P, int K, int n_sink, int n_local,
                                                             int32_t *idx, int idx_stride, int budget,
-                                                            int32_t *attend_ctr)
+                                                            int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
+                                                            int n_prefetch)
 {
     constexpr int NTH = kTopkThreads, NWP = NTH / 32;
     constexpr unsigned FULL = 0xffffffffu;
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
     __shared__ uint32_t cand[kCandMax];              // keys of the chosen bucket
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
+    const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
     grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
     grid_launch_dependents();
     if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
@@ -254,8 +256,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         const bool is_gt = kx > tau, is_eq = kx == tau;
         const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
         const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
-        if (is_gt) out[gb + min(eb, r)] = p;
-        else if (is_eq && eb < r) out[gb + eb] = p;
+        // the pages the flash-decode kernel reads first are on their way into L2 before it starts
+        const int rank = is_gt ? gb + min(eb, r) : (is_eq && eb < r) ? gb + eb : -1;
+        if (rank >= 0) {
+            out[rank] = p;
+            if (rank < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
+        }
         gt_run += __popc(bg);
         eq_run += __popc(be);
     }
@@ -272,7 +278,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
 template <int ROWS>
 __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *scores, int64_t score_stride, int P,
                                                                 int K, int n_sink, int n_local, int32_t *idx,
-                                                                int idx_stride, int budget, int32_t *attend_ctr)
+                                                                int idx_stride, int budget, int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
+                                                            int n_prefetch)
 {
     constexpr int NTH = kTopkThreads, NWP = NTH / 32;
     constexpr unsigned FULL = 0xffffffffu;
@@ -286,6 +293,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
     __shared__ uint32_t cand[kCandMax];
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
+    const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
     const float *sc = scores + (int64_t)bh * score_stride;
     const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp (<= ROWS)
     const int base = warp * 32 * rows + lane;        // this lane's page in row 0
@@ -492,8 +500,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
         const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
         const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
         const int p = base + 32 * j;
-        if (is_gt) out[gb + min(eb, r)] = p;
-        else if (is_eq && eb < r) out[gb + eb] = p;
+        // the pages the flash-decode kernel reads first are on their way into L2 before it starts
+        const int rank = is_gt ? gb + min(eb, r) : (is_eq && eb < r) ? gb + eb : -1;
+        if (rank >= 0) {
+            out[rank] = p;
+            if (rank < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
+        }
         gt_run += __popc(bg);
         eq_run += __popc(be);
     }
@@ -503,7 +515,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
 }  // namespace
 
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, int32_t *attend_ctr, cudaStream_t s)
+                        int idx_stride, int32_t *attend_ctr, int prefetch, cudaStream_t s)
 {
     const int P = (int)((a.len + a.S - 1) / a.S);
     const int K = budget < P ? budget : P;
@@ -537,16 +549,26 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     const int64_t stride = a.page_cap;
+    // pages per head whose keys and values the selection starts moving into L2 for the kernel after it
+    // (the first ones of the list, which that kernel's warps read first): up to kTopkPrefetchBytes in all
+    const int es = a.dtype == RQ_BF16 ? 2 : 4;
+    const int page_bytes = 2 * a.S * a.D * es;
+    const int64_t kv_head_bytes = a.page_cap * (int64_t)page_bytes;
+    const char *kv = static_cast<const char *>(a.kv);
+    int n_prefetch = prefetch ? (int)(kTopkPrefetchBytes / BH / page_bytes) : 0;
+    if (n_prefetch > K) n_prefetch = K;
     const int rows = (P + kTopkThreads - 1) / kTopkThreads;
     if (rows <= 16) {                                // the keys of a head fit in registers
-        using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *);
+        using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
+                                int, int);
         static const Kernel by_rows[8] = {topk_reg_kernel<2>,  topk_reg_kernel<4>,  topk_reg_kernel<6>,  topk_reg_kernel<8>,
                                           topk_reg_kernel<10>, topk_reg_kernel<12>, topk_reg_kernel<14>, topk_reg_kernel<16>};
         cfg.dynamicSmemBytes = 0;
         return cudaLaunchKernelEx(&cfg, by_rows[(rows - 1) / 2], scores, stride, P, K, ns, nl, idx, idx_stride, budget,
-                                  attend_ctr);
+                                  attend_ctr, kv, kv_head_bytes, page_bytes, n_prefetch);
     }
-    return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr);
+    return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv,
+                              kv_head_bytes, page_bytes, n_prefetch);
 }
 
 }  // namespace rq
