@@ -551,12 +551,13 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     const int64_t stride = a.page_cap;
     // pages per head whose keys and values the selection starts moving into L2 for the kernel after it
     // (the first ones of the list, which that kernel's warps read first): up to kTopkPrefetchBytes in all
+    // and an eighth of a head's list
     const int es = a.dtype == RQ_BF16 ? 2 : 4;
     const int page_bytes = 2 * a.S * a.D * es;
     const int64_t kv_head_bytes = a.page_cap * (int64_t)page_bytes;
     const char *kv = static_cast<const char *>(a.kv);
     int n_prefetch = prefetch ? (int)(kTopkPrefetchBytes / BH / page_bytes) : 0;
-    if (n_prefetch > K) n_prefetch = K;
+    if (n_prefetch > K / 8) n_prefetch = K / 8;      // the head of the list only: the kernel waits for its prefetches
     const int rows = (P + kTopkThreads - 1) / kTopkThreads;
     if (rows <= 16) {                                // the keys of a head fit in registers
         using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
