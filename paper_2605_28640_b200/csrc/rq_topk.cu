@@ -34,6 +34,100 @@ constexpr int kDigitBits = 11;
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kCandMax = 1024;                 // candidates ranked directly; a fuller bucket goes through the key bits
 
+constexpr int kHistCopies = 2;                 // histogram copies; warp w adds to copy w % kHistCopies
+static_assert(kTopkThreads == 1024 && kBins == 2 * kTopkThreads, "32 warps; a thread owns two bins in the suffix scan");
+
+// shared-memory scratch of a selection CTA
+struct SelectScratch {
+    alignas(16) uint32_t hist[kHistCopies][kBins];   // read back as 8-byte pairs
+    uint32_t red[32], red2[32];                      // per-warp values of block-wide reductions
+    uint32_t digit, krem, cnt, ncand, tau;           // chosen bin, rank wanted inside it, its population; candidates; threshold
+    uint32_t cand[kCandMax];                         // keys of the chosen bucket
+};
+
+// After a histogram pass (all kHistCopies copies filled): walk the bins from the top until k_rem
+// keys are covered.  Leaves the chosen bin in sh.digit, the rank wanted inside it in sh.krem and
+// its population in sh.cnt.  Called by every thread of the CTA.
+__device__ __forceinline__ void pick_bin(SelectScratch &sh, int k_rem)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __syncthreads();                                 // the histogram is complete
+    uint32_t c0 = 0, c1 = 0;                         // thread t owns bins 2t and 2t+1
+#pragma unroll
+    for (int w = 0; w < kHistCopies; ++w) {
+        const uint2 h2 = *reinterpret_cast<const uint2 *>(&sh.hist[w][2 * tid]);
+        c0 += h2.x;
+        c1 += h2.y;
+    }
+    uint32_t suf = c0 + c1;                          // inclusive suffix sum over the threads of the warp
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_down_sync(FULL, suf, off);
+        if (lane + off < 32) suf += t;
+    }
+    if (lane == 0) sh.red[warp] = suf;               // warp totals
+    __syncthreads();
+    const uint32_t wtot = sh.red[lane];
+    uint32_t wsuf = wtot;                            // suffix sum over the warps, every warp on its own
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+        if (lane + off < 32) wsuf += t;
+    }
+    const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+    const uint32_t incl1 = above + suf - c0;         // keys in bins >= 2t+1
+    const uint32_t excl1 = incl1 - c1;               // keys in bins >  2t+1
+    const uint32_t incl0 = incl1 + c0;               // keys in bins >= 2t
+    const uint32_t kr = (uint32_t)k_rem;
+    if (incl1 >= kr && excl1 < kr) { sh.digit = 2u * tid + 1u; sh.krem = kr - excl1; sh.cnt = c1; }
+    if (incl0 >= kr && incl1 < kr) { sh.digit = 2u * tid; sh.krem = kr - incl1; sh.cnt = c0; }
+    __syncthreads();
+}
+
+// The k_rem-th largest of the cnt candidates in sh.cand (cnt <= kCandMax; they are complete): every
+// candidate is ranked against all others; the wanted one has fewer than k_rem candidates above it
+// and at least k_rem at or above it.  Called by every thread of the CTA.
+__device__ __forceinline__ uint32_t rank_candidates(SelectScratch &sh, uint32_t cnt, int k_rem)
+{
+    const int tid = threadIdx.x;
+    if (tid < (int)cnt) {
+        const uint32_t mine = sh.cand[tid];
+        uint32_t g = 0, ge = 0;
+#pragma unroll 4
+        for (uint32_t j = 0; j < cnt; ++j) {
+            const uint32_t o = sh.cand[j];
+            g += o > mine;
+            ge += o >= mine;
+        }
+        if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) sh.tau = mine;
+    }
+    __syncthreads();
+    return sh.tau;
+}
+
+// From every warp's counts of keys above (wgt) and equal to (weq) the threshold: how many equal keys
+// are taken in all (r) and how many pages of either kind are taken before this warp's.
+__device__ __forceinline__ void scan_warp_counts(SelectScratch &sh, uint32_t wgt, uint32_t weq, int K, int &r, int &gt_run,
+                                                 int &eq_run)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();                                 // earlier readers of red / red2 are done
+    if (lane == 0) { sh.red[warp] = wgt; sh.red2[warp] = weq; }
+    __syncthreads();
+    uint32_t g_inc = sh.red[lane], e_inc = sh.red2[lane];   // inclusive scans over the warps
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
+        if (lane >= off) { g_inc += tg; e_inc += te; }
+    }
+    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
+    r = K - n_gt;                                    // how many equal keys to take
+    gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
+    eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+}
+
 // the score a key was made from (inverse of order_key)
 __device__ __forceinline__ float key_value(uint32_t k)
 {
@@ -46,16 +140,14 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
                                                             int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
                                                             int n_prefetch)
 {
-    constexpr int NTH = kTopkThreads, NWP = NTH / 32;
+    constexpr int NTH = kTopkThreads;
     constexpr unsigned FULL = 0xffffffffu;
-    static_assert(NWP == 32, "second-level reductions are one warp wide");
-    static_assert(kBins == 2 * NTH, "a thread owns two bins in the suffix scan");
-    constexpr int NH = 2;                            // histogram copies; warp w adds to copy w % NH
+    constexpr int NH = kHistCopies;
     extern __shared__ __align__(16) uint32_t skey[]; // [P] keys of the head
-    __shared__ __align__(16) uint32_t hist[NH][kBins];   // read back as 8-byte pairs
-    __shared__ uint32_t red[NWP], red2[NWP];
-    __shared__ uint32_t s_digit, s_krem, s_cnt, s_ncand, s_tau;
-    __shared__ uint32_t cand[kCandMax];              // keys of the chosen bucket
+    __shared__ SelectScratch sh;
+    auto &hist = sh.hist;
+    uint32_t *red = sh.red, *red2 = sh.red2, *cand = sh.cand;
+    uint32_t &s_digit = sh.digit, &s_krem = sh.krem, &s_cnt = sh.cnt, &s_ncand = sh.ncand;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
     const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
@@ -103,38 +195,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
             const uint32_t kx = skey[p];
             if (kx != kKeyForced && in(kx)) atomicAdd(&hist[warp % NH][bin(kx)], 1u);
         }
-        __syncthreads();
-        // thread t owns bins 2t and 2t+1; suffix sums from the top bin down
-        uint32_t c0 = 0, c1 = 0;
-#pragma unroll
-        for (int w = 0; w < NH; ++w) {
-            const uint2 v = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
-            c0 += v.x;
-            c1 += v.y;
-        }
-        uint32_t suf = c0 + c1;                      // inclusive suffix sum over the threads of the warp
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t t = __shfl_down_sync(FULL, suf, off);
-            if (lane + off < 32) suf += t;
-        }
-        if (lane == 0) red[warp] = suf;              // warp totals
-        __syncthreads();
-        const uint32_t wtot = red[lane];
-        uint32_t wsuf = wtot;                        // suffix sum over the warps, every warp on its own
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
-            if (lane + off < 32) wsuf += t;
-        }
-        const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
-        const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
-        const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
-        const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
-        const uint32_t kr = (uint32_t)k_rem;
-        if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
-        if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
-        __syncthreads();
+        pick_bin(sh, k_rem);
     };
     // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
     // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
@@ -196,21 +257,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
             }
             __syncthreads();
             if (cnt <= (uint32_t)kCandMax) {
-                // rank every candidate against all others; the wanted one has fewer than k_rem
-                // candidates above it and at least k_rem at or above it
-                if (tid < (int)cnt) {
-                    const uint32_t mine = cand[tid];
-                    uint32_t g = 0, ge = 0;
-#pragma unroll 4
-                    for (uint32_t j = 0; j < cnt; ++j) {
-                        const uint32_t o = cand[j];
-                        g += o > mine;
-                        ge += o >= mine;
-                    }
-                    if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) s_tau = mine;
-                }
-                __syncthreads();
-                tau = s_tau;
+                tau = rank_candidates(sh, cnt, k_rem);
             } else {
                 // an unusually full bucket (many equal scores): finish on the key bits
                 cmin = __reduce_min_sync(FULL, cmin);
@@ -235,19 +282,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
         wgt += __popc(__ballot_sync(FULL, kx > tau));
         weq += __popc(__ballot_sync(FULL, kx == tau));
     }
-    __syncthreads();
-    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
-    __syncthreads();
-    uint32_t g_inc = red[lane], e_inc = red2[lane];  // inclusive scans over the warps
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
-        if (lane >= off) { g_inc += tg; e_inc += te; }
-    }
-    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
-    const int r = K - n_gt;                          // how many equal keys to take
-    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
-    int eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    int r, gt_run, eq_run;                           // equal keys to take; pages taken before this warp's
+    scan_warp_counts(sh, wgt, weq, K, r, gt_run, eq_run);
     const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll 1
     for (int j = 0; j < rows; ++j) {
@@ -281,16 +317,15 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
                                                                 int idx_stride, int budget, int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
                                                             int n_prefetch)
 {
-    constexpr int NTH = kTopkThreads, NWP = NTH / 32;
+    constexpr int NTH = kTopkThreads;
     constexpr unsigned FULL = 0xffffffffu;
     constexpr uint32_t kAbsent = 0u;                 // below every key: a row beyond the head's pages
-    constexpr int NH = 2;                            // histogram copies; warp w adds to copy w % NH
+    constexpr int NH = kHistCopies;
     static_assert(ROWS % 2 == 0, "bucket numbers are kept in pairs");
-    static_assert(NWP == 32 && kBins == 2 * NTH, "one warp wide second-level reductions; two bins per thread");
-    __shared__ __align__(16) uint32_t hist[NH][kBins];
-    __shared__ uint32_t red[NWP], red2[NWP];
-    __shared__ uint32_t s_digit, s_krem, s_cnt, s_ncand, s_tau;
-    __shared__ uint32_t cand[kCandMax];
+    __shared__ SelectScratch sh;
+    auto &hist = sh.hist;
+    uint32_t *red = sh.red, *red2 = sh.red2, *cand = sh.cand;
+    uint32_t &s_digit = sh.digit, &s_krem = sh.krem, &s_cnt = sh.cnt, &s_ncand = sh.ncand;
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t *out = idx + (int64_t)bh * idx_stride;
     const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
@@ -348,39 +383,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
 
     // After a histogram pass: walk the bins from the top until k_rem keys are covered.  Leaves the
     // chosen bin in s_digit, the rank wanted inside it in s_krem and its population in s_cnt.
-    auto pick_bin = [&]() {
-        __syncthreads();
-        uint32_t c0 = 0, c1 = 0;                     // thread t owns bins 2t and 2t+1
-#pragma unroll
-        for (int w = 0; w < NH; ++w) {
-            const uint2 h2 = *reinterpret_cast<const uint2 *>(&hist[w][2 * tid]);
-            c0 += h2.x;
-            c1 += h2.y;
-        }
-        uint32_t suf = c0 + c1;                      // inclusive suffix sum over the threads of the warp
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t t = __shfl_down_sync(FULL, suf, off);
-            if (lane + off < 32) suf += t;
-        }
-        if (lane == 0) red[warp] = suf;              // warp totals
-        __syncthreads();
-        const uint32_t wtot = red[lane];
-        uint32_t wsuf = wtot;                        // suffix sum over the warps, every warp on its own
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
-            if (lane + off < 32) wsuf += t;
-        }
-        const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
-        const uint32_t incl1 = above + suf - c0;     // keys in bins >= 2t+1
-        const uint32_t excl1 = incl1 - c1;           // keys in bins >  2t+1
-        const uint32_t incl0 = incl1 + c0;           // keys in bins >= 2t
-        const uint32_t kr = (uint32_t)k_rem;
-        if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
-        if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
-        __syncthreads();
-    };
+    auto pick_bin = [&]() { rq::pick_bin(sh, k_rem); };
     // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
     // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
     auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
@@ -447,21 +450,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
             }
             __syncthreads();
             if (cnt <= (uint32_t)kCandMax) {
-                // rank every candidate against all others; the wanted one has fewer than k_rem
-                // candidates above it and at least k_rem at or above it
-                if (tid < (int)cnt) {
-                    const uint32_t mine = cand[tid];
-                    uint32_t g = 0, ge = 0;
-#pragma unroll 4
-                    for (uint32_t j = 0; j < cnt; ++j) {
-                        const uint32_t o = cand[j];
-                        g += o > mine;
-                        ge += o >= mine;
-                    }
-                    if (g < (uint32_t)k_rem && ge >= (uint32_t)k_rem) s_tau = mine;
-                }
-                __syncthreads();
-                tau = s_tau;
+                tau = rank_candidates(sh, cnt, k_rem);
             } else {
                 block_minmax(cmin, cmax);            // an unusually full bucket (many equal scores): finish on the key bits
                 tau = radix_select([&](uint32_t, int j) { return bk(j) == b; }, cmin, cmax);
@@ -480,19 +469,8 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
     }
     wgt = __reduce_add_sync(FULL, (uint32_t)__popc(mg));
     weq = __reduce_add_sync(FULL, (uint32_t)__popc(me));
-    __syncthreads();
-    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
-    __syncthreads();
-    uint32_t g_inc = red[lane], e_inc = red2[lane];  // inclusive scans over the warps
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
-        if (lane >= off) { g_inc += tg; e_inc += te; }
-    }
-    const int n_gt = (int)__shfl_sync(FULL, g_inc, 31);
-    const int r = K - n_gt;                          // how many equal keys to take
-    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt);   // taken before this warp
-    int eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    int r, gt_run, eq_run;                           // equal keys to take; pages taken before this warp's
+    scan_warp_counts(sh, wgt, weq, K, r, gt_run, eq_run);
     const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
     for (int j = 0; j < ROWS; ++j) {
