@@ -110,7 +110,10 @@ def pick_workload(name):
              "cfg4-1/4": dataclasses.replace(wl.CONFIGS[4], budget_den=4),
              "half": dataclasses.replace(wl.METRIC, name="decode-64k-b1", T=65536),
              "page64": dataclasses.replace(wl.METRIC, name="decode-128k-b1-page64", S=64),
-             "small": dataclasses.replace(wl.CONFIGS[1], name="small-16k")}
+             "small": dataclasses.replace(wl.CONFIGS[1], name="small-16k"),
+             # the paper's own Quest settings (App. A.1): 4K context, block 64 with 16 kept pages; block 16 with 4
+             "paper4k": dataclasses.replace(wl.CONFIGS[1], name="quest-4k-block64-k16", T=4096, S=64, budget_den=4),
+             "paper4k-b16": dataclasses.replace(wl.CONFIGS[1], name="quest-4k-block16-k4", T=4096, S=16, budget_den=64)}
     return table[name]
 
 
