@@ -351,10 +351,12 @@ def main():
     ho = torch.empty(w.B, w.H, w.D, dtype=w.dtype).pin_memory()
     n_e2e = min(args.steps, 50)
 
+    stream = torch.cuda.current_stream()
+
     def e2e_step(i):
         kt, vt, gt = ht[i % 8]
-        rq.rq_decode_step_host(caches[i % ncopies].handle, hq[i % 8], kt, vt, gt, K, 0.0, ho)
-        torch.cuda.current_stream().synchronize()      # the caller reads the result before the next step
+        rq.rq_decode_step_host(caches[i % ncopies].handle, hq[i % 8], kt, vt, gt, K, 0.0, ho, stream=stream)
+        stream.synchronize()                           # the caller reads the result before the next step
 
     for i in range(3):
         e2e_step(i)
