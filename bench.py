@@ -291,9 +291,11 @@ def main():
     toks = [wl.make_token(w, dev, s) for s in range(pool)]
     outs = [torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=dev) for _ in range(4)]
 
+    stream = torch.cuda.current_stream()
+
     def step(i):
         kt, vt, gt = toks[i % pool]
-        rq.rq_decode_step(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[i % 4])
+        rq.rq_decode_step(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[i % 4], stream=stream)
 
     for i in range(args.warmup):
         step(i)
@@ -350,8 +352,6 @@ def main():
     ht = [tuple(x.cpu().pin_memory() for x in tk) for tk in toks[:8]]
     ho = torch.empty(w.B, w.H, w.D, dtype=w.dtype).pin_memory()
     n_e2e = min(args.steps, 50)
-
-    stream = torch.cuda.current_stream()
 
     def e2e_step(i):
         kt, vt, gt = ht[i % 8]
