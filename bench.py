@@ -329,7 +329,7 @@ def main():
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms_per_step = t.item() / args.steps
-    n_launches = args.steps * rq.binding.RQ_PROFILE_SLOTS
+    n_launches = args.steps * rq.rq_decode_step_launches(caches[0].handle)
 
     # ---- per-kernel times (separate pass, same rotation): events between the kernels of a step
     prof = {}

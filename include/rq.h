@@ -234,6 +234,12 @@ RQ_API int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int64_t
 /* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
 RQ_API int64_t rq_cache_len(const rq_cache *cache);
 
+/* Kernel launches the next rq_decode_step on this cache will enqueue [no counterpart in the paper:
+ * bookkeeping for benchmarks]: three (update + scoring, selection, attention), or two when the
+ * context is short enough (at most 256 pages per head, at least 16 heads) for one CTA per head to
+ * do the first two kernels' work in one launch.  Host bookkeeping; no CUDA call.  -1 for NULL. */
+RQ_API int rq_decode_step_launches(const rq_cache *cache);
+
 /* Synchronises `stream`, reads the device status word into *status_out (host
  * memory; RQ_OK if no kernel reported anything) and clears it.
  * Returns RQ_OK, INVALID_ARG or CUDA. */

@@ -49,6 +49,7 @@ SIGNATURES = {
     "rq_attend_pages": (C.c_int, [_cachep, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_attend_pages_noalloc": (C.c_int, [_cfgp, _vp, _i64, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
+    "rq_decode_step_launches": (C.c_int, [_cachep]),
     "rq_device_status": (C.c_int, [_cachep, C.POINTER(C.c_int32), _vp]),
     "rq_status_string": (C.c_char_p, [C.c_int]),
     "rq_version": (C.c_int, []),
@@ -165,6 +166,10 @@ def rq_attend_pages_noalloc(cfg: rq_config, kv, length, q, idx, n_idx, scale, o,
 
 def rq_cache_len(cache: rq_cache) -> int:
     return lib().rq_cache_len(C.byref(cache))
+
+
+def rq_decode_step_launches(cache: rq_cache) -> int:
+    return lib().rq_decode_step_launches(C.byref(cache))
 
 
 def rq_device_status(cache: rq_cache, stream=None) -> int:

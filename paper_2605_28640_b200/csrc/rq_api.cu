@@ -110,6 +110,16 @@ static int select_into(const rq_cache *c, int64_t len, const void *q, const void
 {
     DecodeArgs a = decode_args(c, len);
     int32_t *ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
+    const int64_t P = (len + c->cfg.page_size - 1) / c->cfg.page_size;
+    if (P <= kSmallStepPages && c->cfg.batch * c->cfg.heads >= kSmallStepMinHeads) {
+        // a short context: one launch instead of two (the per-kernel marks then show the whole under "score")
+        if (launch_score_select(a, q, k_t, v_t, g_t, scores, do_update, budget, idx, idx_stride, ctr, do_update, s) !=
+            cudaSuccess)
+            return RQ_ERR_CUDA;
+        mark(ev, 1, s);
+        mark(ev, 2, s);
+        return RQ_OK;
+    }
     if (launch_score(a, q, k_t, v_t, g_t, scores, ctr + 3, do_update, sm_count(), s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 1, s);
     if (launch_topk(a, scores, budget, idx, idx_stride, ctr, do_update, s) != cudaSuccess) return RQ_ERR_CUDA;
@@ -396,6 +406,14 @@ int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t 
 }
 
 int64_t rq_cache_len(const rq_cache *cache) { return cache ? cache->len : -1; }
+
+int rq_decode_step_launches(const rq_cache *cache)
+{
+    if (!cache) return -1;
+    const rq_config &c = cache->cfg;
+    const int64_t P = (cache->len + 1 + c.page_size - 1) / c.page_size;     // after the step's append
+    return P <= kSmallStepPages && c.batch * c.heads >= kSmallStepMinHeads ? 2 : 3;
+}
 
 int rq_device_status(rq_cache *cache, int32_t *status_out, void *stream)
 {

@@ -23,6 +23,8 @@ constexpr int kAttendMaxWarps = 2048;  // upper bound of the warps of a flash-de
 constexpr int kCtrStride = 64;         // int32 between the counters of two heads (256 bytes: different L2 lines)
 constexpr int kTopkThreads = 1024;     // threads of the selection CTA
 constexpr int64_t kTopkPrefetchBytes = 16ll << 20;   // selected pages the selection kernel sends towards L2, all heads together
+constexpr int kSmallStepPages = 256;   // heads of up to this many pages are scored and selected by one CTA in one launch ...
+constexpr int kSmallStepMinHeads = 16; // ... when there are at least this many heads to spread over the SMs
 constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
 constexpr int kTargetSMs = 148;        // B200
 
@@ -65,6 +67,11 @@ struct DecodeArgs {
 cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
                          float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s);
 // attend_ctr: the ticket counters of the streaming kernels (cleared here, one head per CTA)
+// Short contexts: the work of launch_score and launch_topk in one launch, one CTA per head (at most
+// kSmallStepPages pages per head).
+cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                                float *scores, int do_update, int budget, int32_t *idx, int idx_stride,
+                                int32_t *attend_ctr, int prefetch, cudaStream_t s);
 // prefetch: the flash-decode kernel runs next, start moving the first selected pages into L2
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
                         int idx_stride, int32_t *attend_ctr, int prefetch, cudaStream_t s);

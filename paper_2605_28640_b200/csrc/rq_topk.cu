@@ -6,6 +6,7 @@
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
+#include "rq_stream.cuh"
 
 namespace rq {
 
@@ -311,35 +312,32 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores,
 // 128-byte lines) and their bucket numbers in registers; the passes over the keys then need no
 // shared-memory traffic and no address arithmetic, which is what the one SM that selects a head
 // spends its issue slots on.  The histogram is cleared before the wait for the scoring kernel.
+// clears what select_rows expects to find clear; a CTA barrier must lie between the two
+__device__ __forceinline__ void select_prepare(SelectScratch &sh)
+{
+    reinterpret_cast<uint4 *>(&sh.hist[0][0])[threadIdx.x] = make_uint4(0u, 0u, 0u, 0u);
+    if (threadIdx.x == 0) sh.ncand = 0;
+}
+
+// The selection proper for one head by the whole CTA (1024 threads): scores sc[0 .. P) -> out[0 .. budget).
+// The histogram and the candidate counter of `sh` are clear on entry (select_prepare).
 template <int ROWS>
-__global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *scores, int64_t score_stride, int P,
-                                                                int K, int n_sink, int n_local, int32_t *idx,
-                                                                int idx_stride, int budget, int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
-                                                            int n_prefetch)
+__device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, int P, int K, int n_sink, int n_local,
+                                            int32_t *out, int budget, const char *kvh, int page_bytes, int n_prefetch)
 {
     constexpr int NTH = kTopkThreads;
     constexpr unsigned FULL = 0xffffffffu;
     constexpr uint32_t kAbsent = 0u;                 // below every key: a row beyond the head's pages
     constexpr int NH = kHistCopies;
     static_assert(ROWS % 2 == 0, "bucket numbers are kept in pairs");
-    __shared__ SelectScratch sh;
     auto &hist = sh.hist;
     uint32_t *red = sh.red, *red2 = sh.red2, *cand = sh.cand;
     uint32_t &s_digit = sh.digit, &s_krem = sh.krem, &s_cnt = sh.cnt, &s_ncand = sh.ncand;
-    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int32_t *out = idx + (int64_t)bh * idx_stride;
-    const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
-    const float *sc = scores + (int64_t)bh * score_stride;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp (<= ROWS)
     const int base = warp * 32 * rows + lane;        // this lane's page in row 0
-
     static_assert(NH * kBins == 4 * NTH, "a thread clears four bins");
     auto clear_hist = [&]() { reinterpret_cast<uint4 *>(&hist[0][0])[tid] = make_uint4(0u, 0u, 0u, 0u); };
-    clear_hist();
-    if (tid == 0) s_ncand = 0;
-    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
-    grid_launch_dependents();
-    if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
     if (K >= P) {                                    // dense: every page, in order
         for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
         return;
@@ -490,6 +488,89 @@ __global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *sco
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
+
+template <int ROWS>
+__global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *scores, int64_t score_stride, int P,
+                                                                int K, int n_sink, int n_local, int32_t *idx,
+                                                                int idx_stride, int budget, int32_t *attend_ctr,
+                                                                const char *kv, int64_t kv_head_bytes, int page_bytes,
+                                                                int n_prefetch)
+{
+    __shared__ SelectScratch sh;
+    const int bh = blockIdx.x;
+    select_prepare(sh);
+    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
+    grid_launch_dependents();
+    if (threadIdx.x < 4) attend_ctr[bh * kCtrStride + threadIdx.x] = 0;   // this head's ticket counters of the streaming kernels
+    select_rows<ROWS>(sh, scores + (int64_t)bh * score_stride, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
+                      kv + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch);
+}
+
+
+// ---------------------------------------------------------------- short contexts: append, score and select in one launch
+// When a head has so few pages that a step is three launch latencies rather than memory traffic, one
+// CTA per head does the first two kernels' work back to back: the single-token update (Eq. 1), the
+// score of every page (Eq. 3; a record per group of lanes, read straight from global memory) and the
+// selection, with the scores passing through the scores buffer.  The flash-decode kernel follows as usual.
+template <typename T, int D, int ROWS>
+__global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a, const T *q, const T *k_t, const T *v_t,
+                                                                    const void *g_t, float *scores, int do_update, int K,
+                                                                    int n_sink, int n_local, int32_t *idx, int idx_stride,
+                                                                    int budget, int32_t *attend_ctr, int64_t kv_head_bytes,
+                                                                    int page_bytes, int n_prefetch)
+{
+    using G = ScoreGeom<T, D>;
+    constexpr unsigned FULL = 0xffffffffu;
+    __shared__ SelectScratch sh;
+    __shared__ float red[32];
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int P = (int)((a.len + a.S - 1) / a.S);
+    select_prepare(sh);
+    grid_dependency_wait();          // earlier kernels may still read what the update rewrites
+    grid_launch_dependents();
+    if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the flash-decode kernel
+    if (do_update) update_head<T, D>(a, bh, q, k_t, v_t, g_t, scores, red);   // also scores the newest page
+
+    const int Ps = do_update ? P - 1 : P;            // pages whose records are read here
+    float qs[G::VPL][G::CH];
+    score_load_q<T, D>(q, bh, lane, qs);
+    const unsigned char *meta = static_cast<const unsigned char *>(a.meta) + (int64_t)bh * a.page_cap * G::REC_BYTES;
+    float *sc = scores + (int64_t)bh * a.page_cap;
+    const int sub = lane / G::LPP, c = lane % G::LPP;
+    constexpr int U = 4;                             // records a lane group has in flight
+    constexpr int STEP = (kTopkThreads / 32) * G::PPW;   // records the CTA covers with one warp-wide read per warp
+    // (the loop bound is the same for every lane of a warp: the shuffles below need all of them)
+    for (int rb = warp * G::PPW; rb < Ps; rb += U * STEP) {
+        const int r0 = rb + sub;
+        uint4 raw[U][G::VPL];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int rec = r0 + u * STEP;
+#pragma unroll
+            for (int v = 0; v < G::VPL; ++v)
+                raw[u][v] = rec < Ps ? ldcs16(meta + (int64_t)rec * G::REC_BYTES + (c + v * G::LPP) * 16) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int rec = r0 + u * STEP;
+            float s = 0.0f;
+#pragma unroll
+            for (int v = 0; v < G::VPL; ++v) {
+                float m[G::CH];
+                unpack16<T>(raw[u][v], m);
+#pragma unroll
+                for (int i = 0; i < G::CH; ++i) s = fmaf(qs[v][i], m[i], s);
+            }
+#pragma unroll
+            for (int off = G::LPP / 2; off > 0; off >>= 1) s += __shfl_xor_sync(FULL, s, off);
+            if (c == 0 && rec < Ps) sc[rec] = s;
+        }
+    }
+    __syncthreads();                 // the head's scores are in the scores buffer
+    select_rows<ROWS>(sh, sc, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
+                      static_cast<const char *>(a.kv) + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch);
+}
+
 }  // namespace
 
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
@@ -548,6 +629,50 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     }
     return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv,
                               kv_head_bytes, page_bytes, n_prefetch);
+}
+
+cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
+                                float *scores, int do_update, int budget, int32_t *idx, int idx_stride,
+                                int32_t *attend_ctr, int prefetch, cudaStream_t s)
+{
+    const int P = (int)((a.len + a.S - 1) / a.S);
+    const int K = budget < P ? budget : P;
+    const int BH = a.B * a.H;
+    int ns = a.n_sink < K ? a.n_sink : K;
+    if (ns > P) ns = P;
+    int nl = a.n_local < K - ns ? a.n_local : K - ns;
+    if (nl > P - ns) nl = P - ns;
+    if (P > kSmallStepPages) return cudaErrorInvalidValue;
+    const int es = a.dtype == RQ_BF16 ? 2 : 4;
+    const int page_bytes = 2 * a.S * a.D * es;
+    const int64_t kv_head_bytes = a.page_cap * (int64_t)page_bytes;
+    int n_prefetch = prefetch ? (int)(kTopkPrefetchBytes / BH / page_bytes) : 0;
+    if (n_prefetch > K / 8) n_prefetch = K / 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)BH);
+    cfg.blockDim = dim3(kTopkThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    constexpr int ROWS = 2;
+    static_assert(kSmallStepPages <= ROWS * kTopkThreads, "the fused kernel keeps a head's keys in two rows");
+#define RQ_LAUNCH_SMALL(T, D)                                                                                          \
+    return cudaLaunchKernelEx(&cfg, score_select_kernel<T, D, ROWS>, a, (const T *)q, (const T *)k_t, (const T *)v_t,  \
+                              g_t, scores, do_update, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv_head_bytes,   \
+                              page_bytes, n_prefetch)
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128) RQ_LAUNCH_SMALL(bf16, 128);
+        if (a.D == 64) RQ_LAUNCH_SMALL(bf16, 64);
+    } else {
+        if (a.D == 128) RQ_LAUNCH_SMALL(float, 128);
+        if (a.D == 64) RQ_LAUNCH_SMALL(float, 64);
+    }
+#undef RQ_LAUNCH_SMALL
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace rq

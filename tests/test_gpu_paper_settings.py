@@ -86,3 +86,25 @@ def test_hit_rate_of_query_aware_and_random_selection():
     assert quest >= 0.9, quest
     # (K / P)^3 = 2.4e-4 per head: over 5 seeds x 16 heads a hit is already unlikely
     assert rand <= 0.05, rand
+
+
+@pytest.mark.parametrize("S,K,T", [(64, 16, 4096), (16, 4, 4096), (16, 9, 1000), (64, 3, 16384)])
+def test_short_context_single_launch_path(S, K, T):
+    """With at least 16 heads and at most 256 pages per head the update, the scoring and the selection
+    run as one launch (one CTA per head); same staged parity as the three-launch path, three steps
+    so that the token count crosses a page boundary, and the stage export must agree with it."""
+    w = wl.Workload("short", B=2, H=16, D=128, T=T, S=S, seed=500 + S + K)
+    heads = [(0, 0), (0, 7), (1, 3), (1, 15)]
+    stats = {}
+    run_case(w, T - 3, steps=3, heads=heads, budget=K, stats=stats)
+    assert stats["heads"] == 3 * len(heads)
+    assert stats.get("near_tie_mismatch", 0) <= stats.get("near_tie", 0)
+
+
+def test_short_context_path_other_shapes():
+    """fp32 I/O with 64 channels and fp32 gates on bf16 I/O through the single-launch path."""
+    for dtype, gdt, D in ((torch.float32, None, 64), (torch.bfloat16, torch.float32, 128), (torch.bfloat16, None, 64)):
+        w = wl.Workload("short-shapes", B=1, H=16, D=D, T=777, S=16, dtype=dtype, gate_dtype=gdt, budget_den=4, seed=600 + D)
+        stats = {}
+        run_case(w, w.T - 2, steps=2, heads=[(0, 0), (0, 9), (0, 15)], stats=stats)
+        assert stats["heads"] == 6
