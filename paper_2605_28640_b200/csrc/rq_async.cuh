@@ -1,6 +1,6 @@
 // Asynchronous-copy helpers for sm_100a: shared-memory transaction barriers
 // (mbarrier) and 1-D bulk copies global -> shared issued through the TMA unit
-// (cp.async.bulk, no tensor map, no multicast).  Every wait is bounded: it
+// (cp.async.bulk, no tensor map, every copy for this CTA alone).  Every wait is bounded: it
 // gives up after a fixed number of polls and reports that to the caller, so no
 // kernel can spin forever on a barrier that never completes.
 #pragma once
