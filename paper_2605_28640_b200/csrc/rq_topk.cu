@@ -13,30 +13,36 @@ namespace rq {
 namespace {
 
 // ---------------------------------------------------------------- top-k
-// One CTA per (b,h).  Scores become order-preserving 32-bit keys in shared
-// memory.  Forced pages (first / newest) are taken outright and count inside
-// the budget.  Among the rest, the k-th largest key is found by a
-// most-significant-digit radix select: the bits that all keys share are
-// skipped, then each pass histograms one 11-bit digit of the keys that still
-// match the prefix found so far and walks the bins from the top until the
-// remaining budget is used up; a pass whose chosen bin is wanted whole ends
-// the search early.  Pages with a larger key are taken; pages with an equal
-// key are taken in index order until the budget is full.  For the output,
-// warp w owns a contiguous range of pages and walks it row by row (row j:
-// pages base_w + 32 j + lane): warp ballots give every taken page its rank
-// inside the warp and a scan over the warp totals its rank in the head, so the
-// output is ascending and unique whatever the thread timing.
+// One CTA of 1024 threads per (b,h).  Scores become order-preserving 32-bit keys.  Forced pages
+// (first / newest) are taken outright and count inside the budget.  Among the rest the k-th
+// largest key (the threshold) is found in two steps: one histogram pass over 2048 equal-width
+// buckets of the score VALUE between the head's smallest and largest score (the map score ->
+// bucket is monotone, so bucket order is key order, and the bulk of the scores is resolved evenly
+// whatever their sign and exponent), then the keys of the bucket that holds the threshold are
+// ranked against each other directly.  A bucket with more than 1024 keys (many equal scores), or a
+// score range too narrow or too wide for a float bucket width, is finished by
+// most-significant-digit radix passes on the key bits instead: the bits all keys share are
+// skipped, each pass histograms one 11-bit digit of the keys that still match the prefix found so
+// far, and a pass whose chosen bin is wanted whole ends the search.  Pages with a key above the
+// threshold are taken; pages with a key equal to it are taken in index order until the budget is
+// full.  For the output, warp w owns a contiguous range of pages and walks it row by row (row j:
+// pages base_w + 32 j + lane): warp ballots give every taken page its rank inside the warp and a
+// scan over the warp totals its rank in the head, so the list is ascending and unique whatever
+// the thread timing.
 //
-// Every CTA runs this code once on an SM whose instruction cache holds another
-// kernel's code, so the loops are kept rolled: fetching the instructions is a
-// visible part of the run time.
+// A thread keeps the keys of its ROWS pages (and their bucket numbers) in registers when a head
+// has at most 10240 pages: the passes over the keys then need no shared-memory traffic and no
+// address arithmetic, which is what the one SM that selects a head spends its issue slots on.
+// Larger heads (up to 32768 pages) keep the keys in shared memory; the code is the same.
 constexpr uint32_t kKeyForced = 0xffffffffu;   // above every score key
+constexpr uint32_t kKeyAbsent = 0u;            // below every score key: a row beyond the head's pages
 constexpr int kDigitBits = 11;
 constexpr int kBins = 1 << kDigitBits;
 constexpr int kCandMax = 1024;                 // candidates ranked directly; a fuller bucket goes through the key bits
 
 constexpr int kHistCopies = 2;                 // histogram copies; warp w adds to copy w % kHistCopies
 static_assert(kTopkThreads == 1024 && kBins == 2 * kTopkThreads, "32 warps; a thread owns two bins in the suffix scan");
+static_assert(kHistCopies * kBins == 4 * kTopkThreads, "a thread clears four bins");
 
 // shared-memory scratch of a selection CTA
 struct SelectScratch {
@@ -135,183 +141,6 @@ __device__ __forceinline__ float key_value(uint32_t k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride,
-                                                            int P, int K, int n_sink, int n_local,
-                                                            int32_t *idx, int idx_stride, int budget,
-                                                            int32_t *attend_ctr, const char *kv, int64_t kv_head_bytes, int page_bytes,
-                                                            int n_prefetch)
-{
-    constexpr int NTH = kTopkThreads;
-    constexpr unsigned FULL = 0xffffffffu;
-    constexpr int NH = kHistCopies;
-    extern __shared__ __align__(16) uint32_t skey[]; // [P] keys of the head
-    __shared__ SelectScratch sh;
-    auto &hist = sh.hist;
-    uint32_t *red = sh.red, *red2 = sh.red2, *cand = sh.cand;
-    uint32_t &s_digit = sh.digit, &s_krem = sh.krem, &s_cnt = sh.cnt, &s_ncand = sh.ncand;
-    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int32_t *out = idx + (int64_t)bh * idx_stride;
-    const char *kvh = kv + (int64_t)bh * kv_head_bytes;   // this head's pages
-    grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
-    grid_launch_dependents();
-    if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the streaming kernels
-
-    if (K >= P) {                                    // dense: every page, in order
-        for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
-        return;
-    }
-    const float *sc = scores + (int64_t)bh * score_stride;
-    uint32_t kmin = 0xffffffffu, kmax = 0u;
-#pragma unroll 4
-    for (int p = tid; p < P; p += NTH) {
-        uint32_t kx = kKeyForced;
-        if (p >= n_sink && p < P - n_local) {
-            kx = order_key(__ldcg(sc + p));
-            kx = min(max(kx, 1u), 0xfffffffeu);      // stay clear of the reserved key
-            kmin = min(kmin, kx);
-            kmax = max(kmax, kx);
-        }
-        skey[p] = kx;
-    }
-    int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
-
-    // range of the score keys -> bits they all share
-    kmin = __reduce_min_sync(FULL, kmin);
-    kmax = __reduce_max_sync(FULL, kmax);
-    if (lane == 0) { red[warp] = kmin; red2[warp] = kmax; }
-    __syncthreads();
-    kmin = __reduce_min_sync(FULL, red[lane]);
-    kmax = __reduce_max_sync(FULL, red2[lane]);
-
-    // One histogram pass over the non-forced keys for which `in(key)` holds: bins by `bin(key)`,
-    // walked from the top until k_rem keys are covered.  Leaves the chosen bin in s_digit, the
-    // rank wanted inside it in s_krem and its population in s_cnt.
-    auto select_bin = [&](auto in, auto bin) {
-        __syncthreads();                             // earlier readers of hist / red / s_* are done
-#pragma unroll 1
-        for (int i = tid; i < NH * kBins; i += NTH) (&hist[0][0])[i] = 0u;
-        __syncthreads();
-#pragma unroll 2
-        for (int p = tid; p < P; p += NTH) {
-            const uint32_t kx = skey[p];
-            if (kx != kKeyForced && in(kx)) atomicAdd(&hist[warp % NH][bin(kx)], 1u);
-        }
-        pick_bin(sh, k_rem);
-    };
-    // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
-    // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
-    auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
-        if (lo_key == hi_key) return lo_key;
-        int hb = 31 - __clz(lo_key ^ hi_key);        // highest bit in which the keys differ
-        uint32_t t = hb == 31 ? 0u : (hi_key >> (hb + 1)) << (hb + 1);   // shared leading bits
-#pragma unroll 1
-        while (hb >= 0) {
-            const int lo = hb >= kDigitBits - 1 ? hb - (kDigitBits - 1) : 0;   // this pass decides bits hb .. lo
-            const uint32_t dmask = (1u << (hb - lo + 1)) - 1u;
-            const uint32_t himask = hb == 31 ? 0u : ~0u << (hb + 1);
-            select_bin([&](uint32_t kx) { return in(kx) && (kx & himask) == (t & himask); },
-                       [&](uint32_t kx) { return (kx >> lo) & dmask; });
-            t |= s_digit << lo;
-            k_rem = (int)s_krem;
-            // every key of the chosen bin is wanted: the bin's lowest possible key is a valid
-            // threshold and the remaining digits need not be resolved
-            if (s_cnt == s_krem) break;
-            hb = lo - 1;
-        }
-        return t;
-    };
-
-    uint32_t tau;                                    // k-th largest key among the non-forced pages
-    if (k_rem <= 0) {
-        tau = 0xfffffffeu + 1u;                      // nothing but forced pages fits: take none of the rest
-    } else if (kmin == kmax) {
-        tau = kmin;
-    } else {
-        // First pass on the score VALUES: 2048 equal-width buckets between the smallest and the
-        // largest score.  The map score -> bucket is monotone, so every key of a higher bucket is
-        // larger than every key of a lower one, and unlike a digit of the key bits the buckets
-        // resolve the bulk of the scores evenly whatever their sign and exponent.
-        const float v_lo = key_value(kmin);
-        const float scale = (float)(kBins - 1) / (key_value(kmax) - v_lo);
-        auto bucket = [&](uint32_t kx) -> uint32_t {
-            const float f = (key_value(kx) - v_lo) * scale;
-            return (uint32_t)min(max((int)f, 0), kBins - 1);
-        };
-        if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
-            tau = radix_select([](uint32_t) { return true; }, kmin, kmax);      // range too wide for a float
-        } else {
-            select_bin([](uint32_t) { return true; }, bucket);
-            const uint32_t b = s_digit, cnt = s_cnt;
-            k_rem = (int)s_krem;
-            // the candidates: keys of the chosen bucket, usually a handful
-            if (tid == 0) s_ncand = 0;
-            __syncthreads();
-            uint32_t cmin = 0xffffffffu, cmax = 0u;
-#pragma unroll 2
-            for (int p = tid; p < P; p += NTH) {
-                const uint32_t kx = skey[p];
-                if (kx != kKeyForced && bucket(kx) == b) {
-                    cmin = min(cmin, kx);
-                    cmax = max(cmax, kx);
-                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = kx;
-                }
-            }
-            __syncthreads();
-            if (cnt <= (uint32_t)kCandMax) {
-                tau = rank_candidates(sh, cnt, k_rem);
-            } else {
-                // an unusually full bucket (many equal scores): finish on the key bits
-                cmin = __reduce_min_sync(FULL, cmin);
-                cmax = __reduce_max_sync(FULL, cmax);
-                if (lane == 0) { red[warp] = cmin; red2[warp] = cmax; }
-                __syncthreads();
-                cmin = __reduce_min_sync(FULL, red[lane]);
-                cmax = __reduce_max_sync(FULL, red2[lane]);
-                tau = radix_select([&](uint32_t kx) { return bucket(kx) == b; }, cmin, cmax);
-            }
-        }
-    }
-
-    // rank of every taken page: ballots inside the warp, a scan over the warp totals across warps
-    const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp
-    const int base = warp * 32 * rows + lane;        // this lane's page in row 0
-    uint32_t wgt = 0, weq = 0;                       // this warp's counts of "greater" and "equal"
-#pragma unroll 1
-    for (int j = 0; j < rows; ++j) {
-        const int p = base + 32 * j;
-        const uint32_t kx = p < P ? skey[p] : 0u;    // 0 is below every key
-        wgt += __popc(__ballot_sync(FULL, kx > tau));
-        weq += __popc(__ballot_sync(FULL, kx == tau));
-    }
-    int r, gt_run, eq_run;                           // equal keys to take; pages taken before this warp's
-    scan_warp_counts(sh, wgt, weq, K, r, gt_run, eq_run);
-    const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll 1
-    for (int j = 0; j < rows; ++j) {
-        const int p = base + 32 * j;
-        const uint32_t kx = p < P ? skey[p] : 0u;
-        const bool is_gt = kx > tau, is_eq = kx == tau;
-        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
-        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
-        // the pages the flash-decode kernel reads first are on their way into L2 before it starts
-        const int rank = is_gt ? gb + min(eb, r) : (is_eq && eb < r) ? gb + eb : -1;
-        if (rank >= 0) {
-            out[rank] = p;
-            if (rank < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
-        }
-        gt_run += __popc(bg);
-        eq_run += __popc(be);
-    }
-    for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
-}
-
-
-// ---------------------------------------------------------------- top-k, keys in registers
-// The same selection for heads of at most ROWS * 1024 pages: a thread keeps the keys of its ROWS
-// pages (row j: page base_w + 32 j + lane, so a warp owns a contiguous range and reads whole
-// 128-byte lines) and their bucket numbers in registers; the passes over the keys then need no
-// shared-memory traffic and no address arithmetic, which is what the one SM that selects a head
-// spends its issue slots on.  The histogram is cleared before the wait for the scoring kernel.
 // clears what select_rows expects to find clear; a CTA barrier must lie between the two
 __device__ __forceinline__ void select_prepare(SelectScratch &sh)
 {
@@ -320,15 +149,18 @@ __device__ __forceinline__ void select_prepare(SelectScratch &sh)
 }
 
 // The selection proper for one head by the whole CTA (1024 threads): scores sc[0 .. P) -> out[0 .. budget).
-// The histogram and the candidate counter of `sh` are clear on entry (select_prepare).
-template <int ROWS>
-__device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, int P, int K, int n_sink, int n_local,
-                                            int32_t *out, int budget, const char *kvh, int page_bytes, int n_prefetch)
+// The histogram and the candidate counter of `sh` are clear on entry (select_prepare).  A thread's
+// row j is page base_w + 32 j + lane; with SMEM_KEYS its key lives in skey[j * 1024 + tid]
+// (skey: ROWS * 1024 words of shared memory), otherwise in a register.
+template <int ROWS, bool SMEM_KEYS>
+__device__ __forceinline__ void select_rows(SelectScratch &sh, uint32_t *skey, const float *sc, int P, int K, int n_sink,
+                                            int n_local, int32_t *out, int budget, const char *kvh, int page_bytes,
+                                            int n_prefetch)
 {
     constexpr int NTH = kTopkThreads;
     constexpr unsigned FULL = 0xffffffffu;
-    constexpr uint32_t kAbsent = 0u;                 // below every key: a row beyond the head's pages
     constexpr int NH = kHistCopies;
+    constexpr int RR = SMEM_KEYS ? 2 : ROWS;         // register rows (the shared-memory variant keeps none)
     static_assert(ROWS % 2 == 0, "bucket numbers are kept in pairs");
     auto &hist = sh.hist;
     uint32_t *red = sh.red, *red2 = sh.red2, *cand = sh.cand;
@@ -336,37 +168,48 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows = (P + NTH - 1) / NTH;            // rows of 32 pages per warp (<= ROWS)
     const int base = warp * 32 * rows + lane;        // this lane's page in row 0
-    static_assert(NH * kBins == 4 * NTH, "a thread clears four bins");
     auto clear_hist = [&]() { reinterpret_cast<uint4 *>(&hist[0][0])[tid] = make_uint4(0u, 0u, 0u, 0u); };
     if (K >= P) {                                    // dense: every page, in order
         for (int p = tid; p < budget; p += NTH) out[p] = p < P ? p : -1;
         return;
     }
 
-    float v[ROWS];
-#pragma unroll
-    for (int j = 0; j < ROWS; ++j) {
-        const int p = base + 32 * j;
-        v[j] = (j < rows && p < P) ? __ldcg(sc + p) : 0.0f;
-    }
-    uint32_t key[ROWS];
+    uint32_t key_r[RR] = {};                         // the keys of this thread's rows (register variant)
+    auto key = [&](int j) -> uint32_t {
+        if constexpr (SMEM_KEYS) return skey[j * NTH + tid];
+        else return key_r[j];
+    };
     uint32_t kmin = 0xffffffffu, kmax = 0u;
+    {
+        float v[RR];
+        if constexpr (!SMEM_KEYS) {                  // all loads first: one round trip
 #pragma unroll
-    for (int j = 0; j < ROWS; ++j) {
-        const int p = base + 32 * j;
-        uint32_t kx = kAbsent;
-        if (j < rows && p < P) {
-            kx = kKeyForced;
-            if (p >= n_sink && p < P - n_local) {
-                kx = min(max(order_key(v[j]), 1u), 0xfffffffeu);   // stay clear of the reserved keys
-                kmin = min(kmin, kx);
-                kmax = max(kmax, kx);
+            for (int j = 0; j < ROWS; ++j) {
+                const int p = base + 32 * j;
+                v[j] = (j < rows && p < P) ? __ldcg(sc + p) : 0.0f;
             }
         }
-        key[j] = kx;
+#pragma unroll (SMEM_KEYS ? 4 : ROWS)
+        for (int j = 0; j < ROWS; ++j) {
+            const int p = base + 32 * j;
+            uint32_t kx = kKeyAbsent;
+            if (j < rows && p < P) {
+                kx = kKeyForced;
+                if (p >= n_sink && p < P - n_local) {
+                    float x;
+                    if constexpr (SMEM_KEYS) x = __ldcg(sc + p);
+                    else x = v[j];
+                    kx = min(max(order_key(x), 1u), 0xfffffffeu);   // stay clear of the reserved keys
+                    kmin = min(kmin, kx);
+                    kmax = max(kmax, kx);
+                }
+            }
+            if constexpr (SMEM_KEYS) skey[j * NTH + tid] = kx;      // read back by this thread only
+            else key_r[j] = kx;
+        }
     }
     int k_rem = K - n_sink - n_local;                // budget left for pages that are not forced
-    auto scored = [&](uint32_t kx) { return kx != kAbsent && kx != kKeyForced; };
+    auto scored = [&](uint32_t kx) { return kx != kKeyAbsent && kx != kKeyForced; };
 
     auto block_minmax = [&](uint32_t &lo, uint32_t &hi) {
         lo = __reduce_min_sync(FULL, lo);
@@ -379,11 +222,10 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
     };
     block_minmax(kmin, kmax);                        // its barriers also publish the cleared histogram
 
-    // After a histogram pass: walk the bins from the top until k_rem keys are covered.  Leaves the
-    // chosen bin in s_digit, the rank wanted inside it in s_krem and its population in s_cnt.
-    auto pick_bin = [&]() { rq::pick_bin(sh, k_rem); };
-    // Most-significant-digit radix select on the key bits among the keys for which `in` holds and
-    // whose extreme keys are lo_key and hi_key: returns the k_rem-th largest of them.
+    // Most-significant-digit radix select on the key bits among the scored keys for which `in`
+    // holds, whose extreme keys are lo_key and hi_key: returns a threshold t such that exactly the
+    // wanted keys of that set are > t or (== t, in index order, as many as are still wanted), and
+    // no key outside the set that is below lo_key is >= t.
     auto radix_select = [&](auto in, uint32_t lo_key, uint32_t hi_key) -> uint32_t {
         if (lo_key == hi_key) return lo_key;
         int hb = 31 - __clz(lo_key ^ hi_key);        // highest bit in which the keys differ
@@ -396,16 +238,20 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
             __syncthreads();                         // earlier readers of the histogram are done
             clear_hist();
             __syncthreads();
-#pragma unroll
+#pragma unroll (SMEM_KEYS ? 2 : ROWS)
             for (int j = 0; j < ROWS; ++j) {
-                const uint32_t kx = key[j];
+                const uint32_t kx = key(j);
                 if (scored(kx) && in(kx, j) && (kx & himask) == (t & himask))
                     atomicAdd(&hist[warp % NH][(kx >> lo) & dmask], 1u);
             }
-            pick_bin();
+            pick_bin(sh, k_rem);
             t |= s_digit << lo;
             k_rem = (int)s_krem;
-            if (s_cnt == s_krem) break;              // the whole bin is wanted: its lowest possible key is a threshold
+            // The whole bin is wanted: any threshold at or below its smallest key takes it all.  The
+            // bin's lowest possible key, t, may lie below lo_key, where keys outside the set may
+            // sit, so the threshold is raised to lo_key (every key of the set is >= lo_key, and
+            // when t < lo_key the bin holds lo_key itself, whose copies are all wanted).
+            if (s_cnt == s_krem) return max(t, lo_key);
             hb = lo - 1;
         }
         return t;
@@ -417,33 +263,39 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
     } else if (kmin == kmax) {
         tau = kmin;
     } else {
-        // 2048 equal-width buckets of the score VALUE between the smallest and the largest score
-        // (monotone in the key), as in the kernel above
         const float v_lo = key_value(kmin);
         const float scale = (float)(kBins - 1) / (key_value(kmax) - v_lo);
+        auto bucket = [&](uint32_t kx) -> uint32_t {
+            const float f = (key_value(kx) - v_lo) * scale;
+            return (uint32_t)min(max((int)f, 0), kBins - 1);
+        };
         if (!(scale > 0.0f) || !(scale < CUDART_INF_F)) {
-            tau = radix_select([](uint32_t, int) { return true; }, kmin, kmax);      // range too wide for a float
+            // the range is too narrow or too wide for a float bucket width
+            tau = radix_select([](uint32_t, int) { return true; }, kmin, kmax);
         } else {
-            uint32_t bk2[ROWS / 2] = {};             // bucket of every key of this thread, two to a word
-            auto bk = [&](int j) -> uint32_t { return (bk2[j / 2] >> (16 * (j & 1))) & 0xffffu; };
-#pragma unroll
+            uint32_t bk2[RR / 2] = {};               // register variant: bucket of every key of this thread, two to a word
+            auto bk = [&](uint32_t kx, int j) -> uint32_t {
+                if constexpr (SMEM_KEYS) return bucket(kx);
+                else return (bk2[j / 2] >> (16 * (j & 1))) & 0xffffu;
+            };
+#pragma unroll (SMEM_KEYS ? 2 : ROWS)
             for (int j = 0; j < ROWS; ++j) {
-                const uint32_t kx = key[j];
-                const float f = (key_value(kx) - v_lo) * scale;
-                const uint32_t bj = scored(kx) ? (uint32_t)min(max((int)f, 0), kBins - 1) : 0xffffu;
+                const uint32_t kx = key(j);
+                const uint32_t bj = scored(kx) ? bucket(kx) : 0xffffu;
                 if (scored(kx)) atomicAdd(&hist[warp % NH][bj], 1u);
-                bk2[j / 2] = (j & 1) ? (bk2[j / 2] | (bj << 16)) : bj;
+                if constexpr (!SMEM_KEYS) bk2[j / 2] = (j & 1) ? (bk2[j / 2] | (bj << 16)) : bj;
             }
-            pick_bin();
+            pick_bin(sh, k_rem);
             const uint32_t b = s_digit, cnt = s_cnt;
             k_rem = (int)s_krem;
             uint32_t cmin = 0xffffffffu, cmax = 0u;
-#pragma unroll
+#pragma unroll (SMEM_KEYS ? 2 : ROWS)
             for (int j = 0; j < ROWS; ++j) {
-                if (bk(j) == b) {                    // a candidate: usually a handful in the whole head
-                    cmin = min(cmin, key[j]);
-                    cmax = max(cmax, key[j]);
-                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = key[j];
+                const uint32_t kx = key(j);
+                if (scored(kx) && bk(kx, j) == b) {  // a candidate: usually a handful in the whole head
+                    cmin = min(cmin, kx);
+                    cmax = max(cmax, kx);
+                    if (cnt <= (uint32_t)kCandMax) cand[atomicAdd(&s_ncand, 1u)] = kx;
                 }
             }
             __syncthreads();
@@ -451,26 +303,25 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
                 tau = rank_candidates(sh, cnt, k_rem);
             } else {
                 block_minmax(cmin, cmax);            // an unusually full bucket (many equal scores): finish on the key bits
-                tau = radix_select([&](uint32_t, int j) { return bk(j) == b; }, cmin, cmax);
+                tau = radix_select([&](uint32_t kx, int j) { return bk(kx, j) == b; }, cmin, cmax);
             }
         }
     }
 
     // rank of every taken page: ballots inside the warp, a scan over the warp totals across warps
-    uint32_t wgt = 0, weq = 0;                       // this warp's counts of "greater" and "equal"
     uint32_t mg = 0, me = 0;                         // bit j: this lane's key of row j is greater / equal
-#pragma unroll
+#pragma unroll (SMEM_KEYS ? 4 : ROWS)
     for (int j = 0; j < ROWS; ++j) {
-        const bool is_gt = key[j] > tau, is_eq = key[j] == tau;   // absent rows hold key 0: neither
-        mg |= (uint32_t)is_gt << j;
-        me |= (uint32_t)is_eq << j;
+        const uint32_t kx = key(j);                  // absent rows hold key 0: neither greater nor equal
+        mg |= (uint32_t)(kx > tau) << j;
+        me |= (uint32_t)(kx == tau) << j;
     }
-    wgt = __reduce_add_sync(FULL, (uint32_t)__popc(mg));
-    weq = __reduce_add_sync(FULL, (uint32_t)__popc(me));
+    const uint32_t wgt = __reduce_add_sync(FULL, (uint32_t)__popc(mg));   // this warp's counts
+    const uint32_t weq = __reduce_add_sync(FULL, (uint32_t)__popc(me));
     int r, gt_run, eq_run;                           // equal keys to take; pages taken before this warp's
     scan_warp_counts(sh, wgt, weq, K, r, gt_run, eq_run);
     const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll
+#pragma unroll (SMEM_KEYS ? 4 : ROWS)
     for (int j = 0; j < ROWS; ++j) {
         const bool is_gt = (mg >> j) & 1u, is_eq = (me >> j) & 1u;
         const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
@@ -488,22 +339,24 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, const float *sc, 
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
-
-template <int ROWS>
-__global__ void __launch_bounds__(kTopkThreads) topk_reg_kernel(const float *scores, int64_t score_stride, int P,
-                                                                int K, int n_sink, int n_local, int32_t *idx,
-                                                                int idx_stride, int budget, int32_t *attend_ctr,
-                                                                const char *kv, int64_t kv_head_bytes, int page_bytes,
-                                                                int n_prefetch)
+// The selection kernel: one CTA per head.  SMEM_KEYS: the keys of a head (ROWS * 1024 words) live
+// in dynamic shared memory.  The histogram is cleared before the wait for the scoring kernel.
+template <int ROWS, bool SMEM_KEYS>
+__global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride, int P, int K,
+                                                            int n_sink, int n_local, int32_t *idx, int idx_stride,
+                                                            int budget, int32_t *attend_ctr, const char *kv,
+                                                            int64_t kv_head_bytes, int page_bytes, int n_prefetch)
 {
+    extern __shared__ __align__(16) uint32_t skey[];
     __shared__ SelectScratch sh;
     const int bh = blockIdx.x;
     select_prepare(sh);
     grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
     grid_launch_dependents();
     if (threadIdx.x < 4) attend_ctr[bh * kCtrStride + threadIdx.x] = 0;   // this head's ticket counters of the streaming kernels
-    select_rows<ROWS>(sh, scores + (int64_t)bh * score_stride, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
-                      kv + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch);
+    select_rows<ROWS, SMEM_KEYS>(sh, skey, scores + (int64_t)bh * score_stride, P, K, n_sink, n_local,
+                                 idx + (int64_t)bh * idx_stride, budget, kv + (int64_t)bh * kv_head_bytes, page_bytes,
+                                 n_prefetch);
 }
 
 
@@ -567,8 +420,10 @@ __global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a
         }
     }
     __syncthreads();                 // the head's scores are in the scores buffer
-    select_rows<ROWS>(sh, sc, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
-                      static_cast<const char *>(a.kv) + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch);
+    // (a head has at most kSmallStepPages = 256 pages here, so no bucket can hold more than kCandMax keys:
+    // the radix passes are reached only through a degenerate score range)
+    select_rows<ROWS, false>(sh, nullptr, sc, P, K, n_sink, n_local, idx + (int64_t)bh * idx_stride, budget,
+                             static_cast<const char *>(a.kv) + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch);
 }
 
 }  // namespace
@@ -585,22 +440,25 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     int nl = a.n_local < K - ns ? a.n_local : K - ns;
     if (nl > P - ns) nl = P - ns;
     if (P > kTopkThreads * kTopkMaxPerThread) return cudaErrorInvalidValue;
-    // the keys of a head live in dynamic shared memory: allow the largest head once per device
+    // the keys of a large head live in dynamic shared memory: allow it once per device
+    constexpr int kMidRows = 16, kBigRows = kTopkMaxPerThread;
+    constexpr int kMidSmem = kMidRows * kTopkThreads * (int)sizeof(uint32_t);
+    constexpr int kBigSmem = kBigRows * kTopkThreads * (int)sizeof(uint32_t);
     static bool ready[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
-        e = cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 kTopkThreads * kTopkMaxPerThread * (int)sizeof(uint32_t));
+        e = cudaFuncSetAttribute(topk_kernel<kMidRows, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMidSmem);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(topk_kernel<kBigRows, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBigSmem);
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)BH);
     cfg.blockDim = dim3(kTopkThreads);
-    cfg.dynamicSmemBytes = (size_t)P * sizeof(uint32_t);
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -618,16 +476,22 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     int n_prefetch = prefetch ? (int)(kTopkPrefetchBytes / BH / page_bytes) : 0;
     if (n_prefetch > K / 8) n_prefetch = K / 8;      // the head of the list only: the kernel waits for its prefetches
     const int rows = (P + kTopkThreads - 1) / kTopkThreads;
-    if (rows <= 16) {                                // the keys of a head fit in registers
-        using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
-                                int, int);
-        static const Kernel by_rows[8] = {topk_reg_kernel<2>,  topk_reg_kernel<4>,  topk_reg_kernel<6>,  topk_reg_kernel<8>,
-                                          topk_reg_kernel<10>, topk_reg_kernel<12>, topk_reg_kernel<14>, topk_reg_kernel<16>};
+    using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
+                            int, int);
+    Kernel kern;
+    if (rows <= 10) {                                // the keys of a head fit in registers (more rows would spill)
+        static const Kernel by_rows[5] = {topk_kernel<2, false>, topk_kernel<4, false>, topk_kernel<6, false>,
+                                          topk_kernel<8, false>, topk_kernel<10, false>};
+        kern = by_rows[(rows - 1) / 2];
         cfg.dynamicSmemBytes = 0;
-        return cudaLaunchKernelEx(&cfg, by_rows[(rows - 1) / 2], scores, stride, P, K, ns, nl, idx, idx_stride, budget,
-                                  attend_ctr, kv, kv_head_bytes, page_bytes, n_prefetch);
+    } else if (rows <= kMidRows) {
+        kern = topk_kernel<kMidRows, true>;
+        cfg.dynamicSmemBytes = kMidSmem;
+    } else {
+        kern = topk_kernel<kBigRows, true>;
+        cfg.dynamicSmemBytes = kBigSmem;
     }
-    return cudaLaunchKernelEx(&cfg, topk_kernel, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv,
+    return cudaLaunchKernelEx(&cfg, kern, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv,
                               kv_head_bytes, page_bytes, n_prefetch);
 }
 
