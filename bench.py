@@ -37,10 +37,10 @@ METRIC = "sparse decode us/step at 128K ctx, 1/16 budget"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
-# (profiles/*_kernel_64k_b1.md: 64 MiB launches, scaled by two to the 128 MiB launches of the
+# (profiles/*_64k_b1.md: captured on the 64K-context case, scaled by two to the launches of the
 # default workload, traffic being proportional to the pages processed): kernel -> bytes, or None
 # when the kernel has changed since the capture.
-NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.57e6), "attend": 2 * (67.24e6 + 1.05e6)}
+NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.57e6), "attend": 2 * (67.24e6 + 1.05e6), "step": None}
 
 
 def measured_peak():
@@ -198,17 +198,86 @@ def run_reference(args, w):
     line = {"impl": "reference", "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": dict(workload_config(w, 1), l2="not applicable: CPU oracle on a sample of heads"),
+            "config": workload_config(w), "l2": "not applicable: CPU oracle on a sample of heads",
             "cpu_baseline": {"value": us, "unit": "us/step", "cores": threads, "kind": "oracle", "sample": sample},
             "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def workload_config(w, ncopies):
+def workload_config(w):
     return {"workload": w.name, "batch": w.B, "heads": w.H, "head_dim": w.D, "context": w.T,
             "page_size": w.S, "budget": f"{w.budget_num}/{w.budget_den}", "budget_pages": w.budget_pages(),
-            "io_dtype": str(w.dtype).replace("torch.", ""), "state_dtype": "float32",
-            "l2": f"inputs larger than L2: {ncopies} independent caches rotated, fresh q/k/v/g every step"}
+            "io_dtype": str(w.dtype).replace("torch.", ""), "state_dtype": "float32"}
+
+
+def event_ms(fn, stream=None):
+    """Device time of fn() between two events on the current stream, synchronised on both sides."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def parity_block(w, cache, sample_inputs, q, tok, K, T0, dev):
+    """One decode step of the timed configuration checked against the fp64 oracle on a sample of
+    heads (states, stored cache, page bounds, scores, page list, attention output), and the recall
+    of the planted pages over all heads for the three budgets.  Runs before the timed region."""
+    import math
+    import torch
+    import paper_2605_28640_b200 as rq
+    from paper_2605_28640_b200 import workloads as wl
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import parity
+    k_s, v_s, g_s = sample_inputs
+    nh = k_s.shape[2]
+    heads = sorted({0, nh // 3, nh - 1})
+    out = {"sampled_heads": [[0, h] for h in heads], "checked": "state, stored cache, page bounds, scores, page list, attention"}
+    try:
+        ohs = {h: parity.oracle_head(w, k_s, v_s, g_s, 0, h, T0 + 8) for h in heads}
+        kt, vt, gt = tok
+        o = torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=dev)
+        idx = torch.full((w.B, w.H, K), -7, dtype=torch.int32, device=dev)
+        rq.rq_decode_step(cache.handle, q, kt, vt, gt, K, 0.0, o, idx)
+        P = w.pages(T0 + 1)
+        scores = torch.empty(w.B, w.H, P, dtype=torch.float32, device=dev)
+        idx2 = torch.empty_like(idx)
+        rq.rq_select_pages(cache.handle, q, K, scores, idx2)
+        torch.cuda.synchronize()
+        assert torch.equal(idx, idx2), "the decode step and the stage export select different pages"
+        assert rq.rq_device_status(cache.handle) == rq.RQ_OK
+        stats = {}
+        parity.OBSERVED.clear()
+        for h, hd in ohs.items():
+            hd.append(parity.f64(kt[0, h]), parity.f64(vt[0, h]), parity.f64(gt[0, h]))
+            d = parity.check_cache_level(cache, hd, 0, h, w.dtype)
+            parity.check_query_level(d, hd, cache, 0, h, q, K, w.D ** -0.5, o, idx, scores, w.dtype, stats)
+        out.update({"passed": True, "near_tie_heads": stats.get("near_tie", 0),
+                    "near_tie_mismatches": stats.get("near_tie_mismatch", 0),
+                    "pages_shared_with_the_oracles_own_chain": stats.get("e2e_overlap", 0.0) / max(stats.get("heads", 1), 1),
+                    "state_abs_err_over_rms": parity.OBSERVED.get("state_abs_err_over_rms"),
+                    "stored_fraction_one_step_off": parity.OBSERVED.get("stored_fraction_one_step_off"),
+                    "attention_max_abs_err": stats.get("att_max"), "attention_mean_abs_err": stats.get("att_mean")})
+    except AssertionError as e:
+        out.update({"passed": False, "failure": str(e)[:300]})
+    if w.needles:
+        planted = wl.needle_pages(w, T0)
+        P = w.pages(T0 + 1)
+        rec = {}
+        for den in (4, 8, 16):
+            Kd = max(1, math.ceil(P / den))
+            if Kd > cache.cfg.max_budget_pages:
+                continue
+            idd = torch.empty(w.B, w.H, Kd, dtype=torch.int32, device=dev)
+            rq.rq_select_pages(cache.handle, q, Kd, None, idd)
+            sel = idd.cpu().numpy()
+            hit = sum(len(set(planted[b, h].tolist()) & set(sel[b, h].tolist())) for b in range(w.B) for h in range(w.H))
+            rec[f"1/{den}"] = hit / (w.B * w.H * w.needles)
+        out["planted_page_recall"] = rec
+    return out
 
 
 # ------------------------------------------------------------------------- own arm
@@ -219,9 +288,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="rq", choices=["rq", "reference"])
     ap.add_argument("--workload", default="metric")
-    ap.add_argument("--copies", type=int, default=0, help="independent caches to rotate (0 = auto)")
+    ap.add_argument("--copies", type=int, default=0, help="independent caches to rotate (0 = auto, at least 4)")
+    ap.add_argument("--path", type=int, default=0, choices=[0, 1, 2, 4, 8],
+                    help="how the step is launched: 0 the library chooses, 1 separate kernels, 2/4/8 one launch with that many groups of heads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--no-parity", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rq" else args.warmup
 
@@ -230,6 +302,7 @@ def main():
         run_reference(args, w)
         return
 
+    import dataclasses
     import torch
     import torch.distributed as dist
     import paper_2605_28640_b200 as rq
@@ -254,32 +327,35 @@ def main():
     es = 2 if w.dtype == torch.bfloat16 else 4
     T0 = w.T - 1                      # the first timed step brings the context to w.T
     total_steps = args.warmup + args.steps
-    # caches: enough copies that their streamed bytes exceed L2 several times over
+    # caches: at least four copies, and enough that their streamed bytes exceed L2 several times over
     meta_b, kv_b = step_bytes(w, w.T)
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
-    ncopies = args.copies or max(2, min(8, -(-(4 * l2) // (meta_b + kv_b))))
-    # per copy: the timed loop, two more passes for the clock sampler, the profiled and e2e passes
+    ncopies = args.copies or max(4, min(8, -(-(4 * l2) // (meta_b + kv_b))))
+    # per copy: the parity step, the timed loop, two more passes for the clock sampler, the profiled and e2e passes
     per_copy = -(-total_steps // ncopies)
-    cap = T0 + 5 * per_copy + 256
+    cap = T0 + 6 * per_copy + 256
     K = w.budget_pages(w.T)
-    maxK = w.budget_pages(cap) + 1
+    maxK = max(w.budget_pages(cap) + 1, -(-w.pages(cap) // 4) + 1)      # room for the 1/4 budget of the recall sweep
+    first = rank == 0 and world == 1
 
-    caches, prefill_ms = [], []
+    caches, first_build_ms, rebuild_ms = [], [], []
     q0 = wl.make_query(w, dev, 0)
-    import dataclasses
+    sample_inputs = None
     for c in range(ncopies):
         wc = dataclasses.replace(w, seed=w.seed + 17 * c, resets=(c == 0))
         k, v, g = wl.make_prefill(wc, dev, T0, q_for_needles=q0 if w.needles else None)
         cache = rq.Cache(w.B, w.H, w.D, w.S, cap, w.dtype, w.gdtype, max_budget_pages=maxK, device=dev)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        rq.rq_build_cache(cache.handle, k, v, g)
-        e1.record()
-        torch.cuda.synchronize()
-        prefill_ms.append(e0.elapsed_time(e1))
+        cache.handle.reserved[2] = args.path
+        first_build_ms.append(event_ms(lambda: rq.rq_build_cache(cache.handle, k, v, g)))
+        if c == 0 and not args.no_prefill:
+            # the prefill proper: rebuilds of the same cache on a kernel that has run before
+            def rebuild():
+                rq.rq_cache_reset(cache.handle)
+                rq.rq_build_cache(cache.handle, k, v, g)
+            for _ in range(7):
+                rebuild_ms.append(event_ms(rebuild))
         caches.append(cache)
-        if c == 0 and rank == 0 and not args.no_cpu_baseline:
+        if c == 0 and first and not (args.no_cpu_baseline and args.no_parity):
             nh = min(8, w.H)
             sample_inputs = (k[:1, :, :nh].clone(), v[:1, :, :nh].clone(), g[:1, :, :nh].clone())
         del k, v, g
@@ -291,12 +367,17 @@ def main():
     toks = [wl.make_token(w, dev, s) for s in range(pool)]
     outs = [torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=dev) for _ in range(4)]
 
+    parity = None
+    if first and not args.no_parity:
+        parity = parity_block(w, caches[0], sample_inputs, qs[0], toks[0], K, T0, dev)
+
     stream = torch.cuda.current_stream()
 
     def step(i):
         kt, vt, gt = toks[i % pool]
         rq.rq_decode_step(caches[i % ncopies].handle, qs[i % pool], kt, vt, gt, K, 0.0, outs[i % 4], stream=stream)
 
+    launches_per_step = rq.rq_decode_step_launches(caches[1 % ncopies].handle, K)
     for i in range(args.warmup):
         step(i)
     barrier()
@@ -329,11 +410,14 @@ def main():
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     ms_per_step = t.item() / args.steps
-    n_launches = args.steps * rq.rq_decode_step_launches(caches[0].handle)
+    n_launches = args.steps * launches_per_step
 
-    # ---- per-kernel times (separate pass, same rotation): events between the kernels of a step
+    # ---- per-kernel times of the step run as separate kernels (a separate pass, same rotation):
+    # events between the kernels of a step
     prof = {}
     nprof = min(args.steps, 50) + 3
+    for c in caches:
+        c.handle.reserved[2] = 1
     for i in range(nprof):
         # a plain step on another cache goes first, so that the profiled kernels are launched
         # behind running work as in the timed loop (on an idle GPU every kernel's time would
@@ -345,7 +429,21 @@ def main():
         if i >= 3:
             for name, us in r.items():
                 prof.setdefault(name, []).append(us)
+    for c in caches:
+        c.handle.reserved[2] = args.path
     kernel_us = {n: sum(v) / len(v) for n, v in prof.items()}
+
+    # ---- what one plain launch of the same size draws from HBM on this GPU: a read of as many
+    # bytes as a step touches (and of half as many: one of its two streams), rotating over the caches
+    sink = torch.zeros(64, dtype=torch.int32, device=dev)
+    probe = {}
+    for name, nbytes in (("step_sized", meta_b + kv_b), ("half_step_sized", (meta_b + kv_b) // 2)):
+        nbytes = min(nbytes, caches[0].kv.numel())
+        for i in range(3):
+            rq.rq_probe_read(caches[i % ncopies].kv, nbytes, sink)
+        reps = 12
+        ms_p = event_ms(lambda: [rq.rq_probe_read(caches[i % ncopies].kv, nbytes, sink) for i in range(reps)])
+        probe[name] = {"bytes": nbytes, "us": ms_p / reps * 1e3, "gbs": nbytes / (ms_p / reps * 1e-3) / 1e9}
 
     # ---- end to end through the host-buffer entry point (pinned host tensors, result read back)
     hq = [q.cpu().pin_memory() for q in qs[:8]]
@@ -380,41 +478,56 @@ def main():
     us = ms_per_step * 1e3
     step_gbs = (meta_b + kv_b) / (us * 1e-6) / 1e9
     kbytes = {"score": meta_b, "attend": kv_b}
-    dom = max(kbytes, key=lambda n: kernel_us.get(n, 0.0))
-    dom_gbs = kbytes[dom] / (kernel_us[dom] * 1e-6) / 1e9
+    separate = {n: {"us": kernel_us[n], "gbs": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9,
+                    "frac": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9 / peak} for n in kbytes if kernel_us.get(n)}
+    if launches_per_step == 1:
+        # the whole step is one kernel: its average launch duration is the step time of the timed region
+        roof = {"bound": "hbm", "kernel": "step (update, scoring, selection, flash-decode and combine in one launch)",
+                "achieved": step_gbs, "peak": peak, "unit": "GB/s", "frac": step_gbs / peak, "peak_kind": peak_kind,
+                "traffic": NCU_TRAFFIC.get("step") if args.workload == "metric" else None,
+                "bytes_per_launch": meta_b + kv_b, "launch_us": us}
+    else:
+        dom = max(kbytes, key=lambda n: kernel_us.get(n, 0.0))
+        roof = {"bound": "hbm", "kernel": dom, "achieved": separate[dom]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": separate[dom]["frac"], "peak_kind": peak_kind,
+                "traffic": NCU_TRAFFIC.get(dom) if args.workload == "metric" else None,
+                "bytes_per_launch": kbytes[dom], "launch_us": kernel_us[dom]}
+    roof["launch_sized_read_gbs"] = probe["step_sized" if launches_per_step == 1 else "half_step_sized"]["gbs"]
+    roof["plain_read_probe"] = probe
+    roof["as_separate_kernels_us"] = kernel_us
+    roof["as_separate_kernels"] = separate
     line = {
         "metric": METRIC, "value": us / world, "unit": "us/step", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w, ncopies),
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w),
+        "l2": f"inputs larger than L2: {ncopies} independent caches rotated, fresh q/k/v/g every step",
         "tokens_per_s": w.B * world / (us * 1e-6),
         "step_hbm": {"algorithmic_bytes": meta_b + kv_b, "gbs": step_gbs, "frac_of_peak": step_gbs / peak,
                      "frac_of_nominal_8tbs": step_gbs / 8000.0, "peak_gbs": peak, "peak_kind": peak_kind},
-        "kernels_us": kernel_us,
-        "roofline": {"bound": "hbm", "kernel": dom, "achieved": dom_gbs, "peak": peak, "unit": "GB/s",
-                     "frac": dom_gbs / peak, "peak_kind": peak_kind,
-                     "traffic": NCU_TRAFFIC.get(dom) if args.workload == "metric" else None,
-                     "bytes_per_launch": kbytes[dom],
-                     "others": {n: {"gbs": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9, "frac": kbytes[n] / (kernel_us[n] * 1e-6) / 1e9 / peak}
-                                for n in kbytes if n != dom}},
+        "roofline": roof,
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_us / world, "unit": "us/step", "h2d_bytes_per_step": in_bytes,
                 "d2h_bytes_per_step": out_bytes},
-        "gpu_launches": n_launches,
+        "gpu_launches": n_launches, "launches_per_step": launches_per_step,
     }
-    if not args.no_prefill:
-        pm = sorted(prefill_ms)[(len(prefill_ms) - 1) // 2]     # lower median: the first build also pays one-time set-up
+    if parity is not None:
+        line["parity"] = parity
+    if not args.no_prefill and rebuild_ms:
+        runs = sorted(rebuild_ms[2:])                            # the first two rebuilds warm the kernel up
+        pm = runs[len(runs) // 2]
         gs = 2 if w.gdtype == torch.bfloat16 else 4
         pbytes = w.B * w.H * T0 * w.D * (2 * es + gs + 2 * es) + w.B * w.H * w.pages(T0) * 2 * w.D * es
-        line["prefill"] = {"ms": pm, "tokens_per_s": w.B * T0 / (pm * 1e-3), "algorithmic_bytes": pbytes,
+        line["prefill"] = {"ms": pm, "ms_min": runs[0], "tokens_per_s": w.B * T0 / (pm * 1e-3), "algorithmic_bytes": pbytes,
                            "gbs": pbytes / (pm * 1e-3) / 1e9, "frac_of_peak": pbytes / (pm * 1e-3) / 1e9 / peak,
-                           "runs_ms": prefill_ms}
-    if not args.no_cpu_baseline:
+                           "runs_ms": rebuild_ms[2:], "first_build_ms": first_build_ms,
+                           "note": "median of five rebuilds (rq_cache_reset + rq_build_cache) after two warm-up rebuilds"}
+    if first and not args.no_cpu_baseline:
         nh = min(8, w.H)
         threads = min(os.cpu_count() or 1, nh)
         smp = oracle_sample_for(w, dev, nh, threads, 4096, inputs=sample_inputs)
         smp.step()
-        probe = sum(smp.step() for _ in range(3)) / 3
-        reps = int(max(10, min(4000, 12.0 / max(probe, 1e-6))))    # about 12 s of host work
+        probe_s = sum(smp.step() for _ in range(3)) / 3
+        reps = int(max(10, min(4000, 12.0 / max(probe_s, 1e-6))))    # about 12 s of host work
         wall = sum(smp.step() for _ in range(reps))
         rounds_sample = -(-nh // threads)
         rounds_full = -(-(w.B * w.H) // threads)

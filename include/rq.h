@@ -101,6 +101,15 @@ typedef struct rq_cache {
     void *workspace;
     int64_t len;           /* tokens currently in every sequence                           */
     int64_t page_capacity; /* ceil(capacity_tokens / page_size)                            */
+    /* reserved[0]: decode steps that ran as one launch so far (kept by the library).
+     * reserved[1]: testing aid: poll limit of the device-side waits for asynchronous copies;
+     *              0 = the built-in limit, < 0 = no poll at all, so that the first wait of every
+     *              warp gives up, the kernels let their copies land and return, and the device
+     *              status reads RQ_ERR_TIMEOUT; call rq_cache_reset before the cache is used again.
+     * reserved[2]: how rq_decode_step runs: 0 = the library chooses, 1 = always as separate
+     *              kernels, 2 / 4 / 8 = as one launch with that many groups of heads whenever the
+     *              shape allows it.  The results are the same.
+     * reserved[3]: must be 0. */
     int64_t reserved[4];
 } rq_cache;
 
@@ -142,7 +151,9 @@ RQ_API int rq_build_cache(rq_cache *cache, const void *k, const void *v, const v
  * recurrence with (k_t, v_t, g_t), append the rounded state to the cache,
  * update the newest page's min/max, len += 1; (2) score all pages with q;
  * (3) keep min(budget_pages, #pages) pages per (b,h); (4) attend over their
- * valid tokens — the query sees its own token.
+ * valid tokens — the query sees its own token.  Depending on the shape the
+ * step is one kernel launch or several (rq_decode_step_launches); the results
+ * are the same.  On an error the cache's length is unchanged.
  *   q, k_t, v_t, o : [B][H][D] contiguous, cfg.dtype;  g_t : [B][H][D], cfg.gate_dtype
  *   budget_pages   : 1 .. cfg.max_budget_pages (>= #pages means dense attention)
  *   scale          : softmax scale; <= 0 selects 1/sqrt(D)
@@ -234,11 +245,22 @@ RQ_API int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int64_t
 /* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
 RQ_API int64_t rq_cache_len(const rq_cache *cache);
 
-/* Kernel launches the next rq_decode_step on this cache will enqueue [no counterpart in the paper:
- * bookkeeping for benchmarks]: three (update + scoring, selection, attention), or two when the
- * context is short enough (at most 256 pages per head, at least 16 heads) for one CTA per head to
- * do the first two kernels' work in one launch.  Host bookkeeping; no CUDA call.  -1 for NULL. */
-RQ_API int rq_decode_step_launches(const rq_cache *cache);
+/* Kernel launches the next rq_decode_step on this cache will enqueue for this budget when
+ * sel_idx_out is NULL [no counterpart in the paper: bookkeeping for benchmarks]: ONE when the whole
+ * step runs as one launch (at most 256 (batch, head) pairs that split into 2, 4 or 8 equal groups
+ * which keep the GPU's resident CTAs busy, more than 256 pages per head, budget below the number
+ * of pages; a non-NULL sel_idx_out adds a launch that sorts the list); otherwise three (update +
+ * scoring, selection, attention), or two when the context is short enough (at most 256 pages per
+ * head, at least 16 heads) for one CTA per head to do the first two kernels' work in one launch.
+ * The first call on a device looks up launch parameters (occupancy).  -1 for an invalid cache. */
+RQ_API int rq_decode_step_launches(const rq_cache *cache, int32_t budget_pages);
+
+/* Benchmarking aid [no counterpart in the paper]: one launch that reads `bytes` bytes (rounded
+ * down to a multiple of 16) of device memory at `buf` (16-byte aligned) once, with plain 16-byte
+ * loads, and folds them into the 64 words at `sink` (device memory, 256 bytes, 4-byte aligned).
+ * Timed by the caller, it shows what a single launch of the decode step's size can draw from
+ * HBM on the GPU at hand.  Enqueued on `stream`; returns INVALID_ARG or CUDA on failure. */
+RQ_API int rq_probe_read(const void *buf, size_t bytes, void *sink, void *stream);
 
 /* Synchronises `stream`, reads the device status word into *status_out (host
  * memory; RQ_OK if no kernel reported anything) and clears it.

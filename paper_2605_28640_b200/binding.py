@@ -48,8 +48,9 @@ SIGNATURES = {
     "rq_select_pages": (C.c_int, [_cachep, _vp, _i32, _vp, _vp, _vp]),
     "rq_attend_pages": (C.c_int, [_cachep, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_attend_pages_noalloc": (C.c_int, [_cfgp, _vp, _i64, _vp, _vp, _i32, _f, _vp, _vp]),
+    "rq_probe_read": (C.c_int, [_vp, C.c_size_t, _vp, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
-    "rq_decode_step_launches": (C.c_int, [_cachep]),
+    "rq_decode_step_launches": (C.c_int, [_cachep, _i32]),
     "rq_device_status": (C.c_int, [_cachep, C.POINTER(C.c_int32), _vp]),
     "rq_status_string": (C.c_char_p, [C.c_int]),
     "rq_version": (C.c_int, []),
@@ -164,12 +165,17 @@ def rq_attend_pages_noalloc(cfg: rq_config, kv, length, q, idx, n_idx, scale, o,
                                          _ptr(o), _stream(stream)), "rq_attend_pages_noalloc")
 
 
+def rq_probe_read(buf, nbytes, sink, stream=None):
+    """One launch that reads nbytes of the device tensor `buf` once (benchmarking aid)."""
+    _check(lib().rq_probe_read(_ptr(buf), nbytes, _ptr(sink), _stream(stream)), "rq_probe_read")
+
+
 def rq_cache_len(cache: rq_cache) -> int:
     return lib().rq_cache_len(C.byref(cache))
 
 
-def rq_decode_step_launches(cache: rq_cache) -> int:
-    return lib().rq_decode_step_launches(C.byref(cache))
+def rq_decode_step_launches(cache: rq_cache, budget_pages: int) -> int:
+    return lib().rq_decode_step_launches(C.byref(cache), budget_pages)
 
 
 def rq_device_status(cache: rq_cache, stream=None) -> int:

@@ -36,6 +36,11 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     size_t off = 0;
     w.status = off;  off += align256(64 * sizeof(int32_t));
     w.tickets = off; off += align256(BH * (size_t)kCtrStride * sizeof(int32_t));
+    const size_t SH = BH <= (size_t)kStepMaxHeads ? BH : 0;      // heads the one-launch step keeps records for
+    w.absmax = off;   off += align256(2 * SH * sizeof(float));
+    w.step_ctr = off; off += align256(2 * SH * (size_t)kStepCtrInts * sizeof(int32_t));
+    w.list = off;     off += align256(SH * (size_t)c.max_budget_pages * sizeof(int2));
+    w.hist = off;     off += align256(SH * (size_t)kStepBins * sizeof(uint32_t));
     w.scores = off;  off += align256(BH * pc * sizeof(float));
     w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
     const size_t slots = (size_t)attend_slots_per_head((int64_t)c.max_budget_pages * (c.page_size / 16));
@@ -61,23 +66,41 @@ int rq::stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_c
 
 namespace rq {
 
-static int sm_count()
+// SMs of the current device, looked up once per device.  (These per-device tables, like the ones
+// in the launchers, are filled without a lock: two threads that make their first call on a device
+// at the same time both look the value up and store the same number.)
+int sm_count()
 {
-    static int cached = 0;
-    if (cached == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            cached = n;
+    static int cached[64];
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kTargetSMs;
+    if (cached[dev] == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached[dev] = n;
         else
-            cached = kTargetSMs;
+            cached[dev] = kTargetSMs;
     }
-    return cached;
+    return cached[dev];
+}
+
+// rq_cache::reserved: [0] number of decode steps that ran as one launch (that path alternates between
+// two sets of counters and two copies of the heads' largest |stored key|; every step, whatever its
+// path, works as step number reserved[0] + 1 and only a one-launch step commits that number, so the
+// copy with parity reserved[0] + 1 is always the up-to-date one), [1] poll limit of device-side copy waits (0: the default, < 0: none at all; a
+// testing aid), [2] choice of the decode path (0: automatic, 1: always the separate kernels,
+// 2, 4, 8: the one-launch step with that many waves whenever the shape allows it)
+static float *absmax_of(const rq_cache *c)
+{
+    if ((int64_t)c->cfg.batch * c->cfg.heads > kStepMaxHeads) return nullptr;
+    return (float *)((char *)c->workspace + workspace_layout(c->cfg).absmax);
 }
 
 static DecodeArgs decode_args(const rq_cache *c, int64_t len)
 {
     DecodeArgs a;
+    a.absmax = absmax_of(c);
+    a.epoch = (int32_t)((c->reserved[0] + 1) & 0x3fffffff);
+    a.poll_limit = (int32_t)c->reserved[1];
     a.kv = c->kv; a.meta = c->meta; a.state = (float *)c->state;
     a.B = c->cfg.batch; a.H = c->cfg.heads; a.D = c->cfg.head_dim; a.S = c->cfg.page_size;
     a.dtype = c->cfg.dtype; a.gate_dtype = c->cfg.gate_dtype;
@@ -142,6 +165,34 @@ static int attend_from(const rq_cache *c, int64_t len, const void *q, const int3
     return RQ_OK;
 }
 
+static StepBuffers step_buffers(const rq_cache *c, const WorkspaceLayout &w)
+{
+    StepBuffers b;
+    char *ws = (char *)c->workspace;
+    b.scores = (float *)(ws + w.scores);
+    b.list = (int2 *)(ws + w.list);
+    b.list_stride = c->cfg.max_budget_pages;
+    b.partial = (float *)(ws + w.partial);
+    b.slots = attend_slots_per_head((int64_t)c->cfg.max_budget_pages * (c->cfg.page_size / 16));
+    b.ctr = (int32_t *)(ws + w.step_ctr);
+    b.hist = (uint32_t *)(ws + w.hist);
+    return b;
+}
+
+// Waves of the one-launch step for the next decode step (args for the length after the append),
+// 0 if the step runs as separate kernels.
+static int step_waves(const rq_cache *c, const DecodeArgs &a, int budget, int *grid)
+{
+    const int64_t choice = c->reserved[2];
+    if (choice == 1) return 0;
+    const int forced = choice == 2 || choice == 4 || choice == 8 ? (int)choice : 0;
+    const int waves = step_plan(a, budget, sm_count(), forced, grid);
+    if (waves <= 0) return 0;
+    const int team = *grid / (a.B * a.H / waves);
+    const int slots = attend_slots_per_head((int64_t)c->cfg.max_budget_pages * (c->cfg.page_size / 16));
+    return team <= slots ? waves : 0;
+}
+
 static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, const void *v_t,
                             const void *g_t, int32_t budget_pages, float scale, void *o,
                             int32_t *sel_idx_out, cudaStream_t s, cudaEvent_t *ev)
@@ -157,12 +208,35 @@ static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, con
     int32_t *sel = sel_idx_out ? sel_idx_out : (int32_t *)((char *)cache->workspace + w.sel);
 
     mark(ev, 0, s);
-    cache->len += 1;
-    const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
-    int st = select_into(cache, cache->len, q, k_t, v_t, g_t, 1, budget_pages, scores, sel, budget_pages, s, ev);
+    // the length and the step number are committed only when every launch of the step succeeded
+    const int64_t new_len = cache->len + 1;
+    const int64_t P = (new_len + c.page_size - 1) / c.page_size;
+    int st;
+    int grid = 0;
+    DecodeArgs a = decode_args(cache, new_len);
+    const int waves = step_waves(cache, a, budget_pages, &grid);
+    if (waves > 0) {
+        // one launch; the list lands in the workspace in no particular order and is sorted for the caller
+        const StepBuffers b = step_buffers(cache, w);
+        if (!(scale > 0.0f)) scale = 1.0f / sqrtf((float)a.D);
+        st = launch_step(a, q, k_t, v_t, g_t, budget_pages, scale, b, o, waves, grid, s) == cudaSuccess ? RQ_OK : RQ_ERR_CUDA;
+        mark(ev, 1, s);
+        if (st == RQ_OK && sel_idx_out &&
+            launch_sort_list(b.list, b.list_stride, budget_pages, (int)P, a.B * a.H, sel_idx_out, budget_pages, s) != cudaSuccess)
+            st = RQ_ERR_CUDA;
+        mark(ev, 2, s);
+        mark(ev, 3, s);
+        if (st == RQ_OK) cache->reserved[0] += 1;
+    } else {
+        st = select_into(cache, new_len, q, k_t, v_t, g_t, 1, budget_pages, scores, sel, budget_pages, s, ev);
+        if (st == RQ_OK) {
+            const int n_idx = (int)(budget_pages < P ? budget_pages : P);
+            st = attend_from(cache, new_len, q, sel, n_idx, budget_pages, scale, o, s, ev);
+        }
+    }
     if (st != RQ_OK) return st;
-    const int n_idx = (int)(budget_pages < P ? budget_pages : P);
-    return attend_from(cache, cache->len, q, sel, n_idx, budget_pages, scale, o, s, ev);
+    cache->len = new_len;
+    return RQ_OK;
 }
 
 // Gather of the four per-step input tensors from pinned host memory (read over the bus by the
@@ -178,6 +252,28 @@ __global__ void stage_in_kernel(const uint4 *q, const uint4 *k, const uint4 *v, 
     if (i < nv) { dv[i] = v[i]; return; }
     i -= nv;
     if (i < ng) dg[i] = g[i];
+}
+
+// Plain streaming read of a buffer: 16-byte loads, eight in flight per thread, the words folded
+// into one value per CTA so that the loads cannot be dropped.  A yardstick for what one launch of
+// a given size can draw from HBM, nothing of the method.
+__global__ void __launch_bounds__(256) probe_read_kernel(const uint4 *src, size_t n16, uint32_t *sink)
+{
+    constexpr int U = 8;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    uint32_t acc = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += stride * U) {
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t j = i + (size_t)u * stride;
+            v[u] = j < n16 ? __ldcs(src + j) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+    }
+    acc = __reduce_xor_sync(0xffffffffu, acc);
+    if ((threadIdx.x & 31) == 0) atomicXor(sink + (blockIdx.x & 63), acc);
 }
 
 // Device address of a host buffer if it is pinned (or registered) and 16-byte aligned.
@@ -270,6 +366,7 @@ int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
     a.B = c.batch; a.H = c.heads; a.D = c.head_dim; a.S = c.page_size;
     a.dtype = c.dtype; a.gate_dtype = c.gate_dtype;
     a.len0 = cache->len; a.T = T; a.page_cap = cache->page_capacity;
+    a.absmax = absmax_of(cache);
     if (launch_scan(a, (cudaStream_t)stream) != cudaSuccess) return RQ_ERR_CUDA;
     cache->len += T;
     return RQ_OK;
@@ -309,6 +406,7 @@ int rq_decode_step_profiled(rq_cache *cache, const void *q, const void *k_t, con
 
 const char *rq_profile_slot_name(int slot)
 {
+    // (when the step runs as one launch, slot 0 holds the whole step and slot 1 the sorting of the list)
     static const char *names[RQ_PROFILE_SLOTS] = {"score", "topk", "attend"};
     return slot >= 0 && slot < RQ_PROFILE_SLOTS ? names[slot] : "";
 }
@@ -405,13 +503,27 @@ int rq_attend_pages(rq_cache *cache, const void *q, const int32_t *idx, int32_t 
     return attend_from(cache, cache->len, q, idx, n_idx, n_idx, scale, o, (cudaStream_t)stream);
 }
 
+int rq_probe_read(const void *buf, size_t bytes, void *sink, void *stream)
+{
+    if (!buf || !sink || bytes < 16 || !aligned(buf, 16) || !aligned(sink, 4)) return RQ_ERR_INVALID_ARG;
+    const size_t n16 = bytes / 16;
+    size_t ctas = (n16 + 256 * 8 - 1) / (256 * 8);
+    const size_t most = (size_t)sm_count() * 8;
+    if (ctas > most) ctas = most;
+    probe_read_kernel<<<(unsigned)ctas, 256, 0, (cudaStream_t)stream>>>((const uint4 *)buf, n16, (uint32_t *)sink);
+    return cudaGetLastError() == cudaSuccess ? RQ_OK : RQ_ERR_CUDA;
+}
+
 int64_t rq_cache_len(const rq_cache *cache) { return cache ? cache->len : -1; }
 
-int rq_decode_step_launches(const rq_cache *cache)
+int rq_decode_step_launches(const rq_cache *cache, int32_t budget_pages)
 {
-    if (!cache) return -1;
+    if (!cache || check_cache(cache) != RQ_OK) return -1;
     const rq_config &c = cache->cfg;
     const int64_t P = (cache->len + 1 + c.page_size - 1) / c.page_size;     // after the step's append
+    int grid = 0;
+    const DecodeArgs a = decode_args(cache, cache->len + 1);
+    if (budget_pages >= 1 && step_waves(cache, a, budget_pages, &grid) > 0) return 1;
     return P <= kSmallStepPages && c.batch * c.heads >= kSmallStepMinHeads ? 2 : 3;
 }
 

@@ -43,10 +43,10 @@ constexpr uint32_t kMbarSuspendNs = 2000;
 
 // Wait for the phase with the given parity to complete.  Returns false if the
 // poll limit ran out first.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, int limit = kMbarPollLimit)
 {
     const uint32_t addr = smem_addr(bar);
-    for (int it = 0; it < kMbarPollLimit; ++it) {
+    for (int it = 0; it < limit; ++it) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -116,12 +116,56 @@ __device__ __forceinline__ float4 ld_cg_now(const float4 *p)
     asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
     return r;
 }
+__device__ __forceinline__ uint4 ld_cg_now(const uint4 *p)
+{
+    uint4 r;
+    asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
 __device__ __forceinline__ float2 ld_cg_now(const float2 *p)
 {
     float2 r;
     asm volatile("ld.global.cg.v2.f32 {%0, %1}, [%2];" : "=f"(r.x), "=f"(r.y) : "l"(p));
     return r;
 }
+
+// Flag shared between CTAs: a release store publishes everything the storing thread has
+// written (or has observed through a barrier) before it; the acquire load pairs with it.
+__device__ __forceinline__ void st_release(int32_t *p, int32_t v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int32_t ld_acquire(const int32_t *p)
+{
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Polling form of the same: a relaxed load does not hold back the thread's later memory
+// operations while it is under way; once it has seen the awaited value, the fence makes the
+// publisher's earlier writes visible to what follows.
+__device__ __forceinline__ int32_t ld_relaxed(const int32_t *p)
+{
+    int32_t v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_acquire() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+// add with acquire-release ordering at device scope; returns the value before
+__device__ __forceinline__ int32_t atom_add_acq_rel(int32_t *p, int32_t v)
+{
+    int32_t old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+// fire-and-forget increment of a counter in global memory
+__device__ __forceinline__ void red_inc(uint32_t *p)
+{
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
+// Poll limit and pause of a wait for another CTA's flag: 2^22 polls 128 ns apart, about half a second.
+constexpr int kFlagPollLimit = 1 << 22;
+constexpr unsigned kFlagPollNs = 128;
 
 __device__ __forceinline__ int ld_volatile(const int32_t *p) { return *reinterpret_cast<const volatile int32_t *>(p); }
 

@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
     const int wg = blockIdx.x * NW + warp;
 
     const uint64_t stream_policy = l2_evict_first_policy();
+    const int poll_limit = a.poll_limit == 0 ? kMbarPollLimit : (a.poll_limit < 0 ? 0 : a.poll_limit);
     uint64_t *mybars = bars + warp * DEPTH;
     int2 *myinfo = infos + warp * DEPTH;
     unsigned char *myring = ring + (size_t)warp * DEPTH * G::STAGE_BYTES;
@@ -266,10 +267,10 @@ __global__ void __launch_bounds__(kAttendWarps * 32) attend_kernel(DecodeArgs a,
         }
         const int valid = inf.y;
         if (valid > 0 && !dead) {
-            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u)) {
-                // give the copies still in flight the same bounded chance to land, then stop
+            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u, poll_limit)) {
+                // give every copy in flight (this one too) the usual bounded chance to land, then stop
                 for (int s = 0; s < DEPTH; ++s)
-                    if (s != stage && myinfo[s].x >= 0 && myinfo[s].y > 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
+                    if (myinfo[s].x >= 0 && myinfo[s].y > 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
                 if (lane == 0) atomicExch(a.status, RQ_ERR_TIMEOUT);
                 dead = true;
             }
@@ -499,10 +500,7 @@ extern "C" int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int
     const int64_t per_head = (int64_t)n_idx * tpp;
     if (per_head > kDoneTileMask) return RQ_ERR_CAPACITY;
 
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
-        return RQ_ERR_CUDA;
+    const int sms = sm_count();
 
     DecodeArgs a = {};
     a.kv = const_cast<void *>(kv);

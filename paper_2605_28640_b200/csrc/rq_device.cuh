@@ -107,4 +107,10 @@ __device__ __forceinline__ uint32_t order_key(float x)
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 
+// the float a key was made from (inverse of order_key)
+__device__ __forceinline__ float order_key_value(uint32_t k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
 }  // namespace rq

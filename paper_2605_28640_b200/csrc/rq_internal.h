@@ -28,6 +28,11 @@ constexpr int kSmallStepMinHeads = 16; // ... when there are at least this many 
 constexpr int kTopkMaxPerThread = 32;  // => at most 32768 pages per head
 constexpr int kTargetSMs = 148;        // B200
 
+// ---- the one-launch decode step (rq_step.cu) ----
+constexpr int kStepMaxHeads = 256;     // the one-launch step serves at most this many (batch, head) pairs
+constexpr int kStepBins = 2048;        // value buckets of a head's score histogram
+constexpr int kStepCtrInts = 16;       // int32 per head and counter set (64 bytes)
+
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
     size_t status;    // int32[64]
@@ -36,12 +41,18 @@ struct WorkspaceLayout {
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
     size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
+    // the one-launch step (present when BH <= kStepMaxHeads, otherwise empty); everything from
+    // `status` up to `scores` is cleared by rq_cache_reset, which is why these regions sit there
+    size_t absmax;    // float [2][BH]: largest |stored key| of every head, two copies (read one, write the other)
+    size_t step_ctr;  // int32 [2][BH][kStepCtrInts]: two sets of per-head counters, used by alternate steps
+    size_t list;      // int2 [BH][max_budget]: page lists of the one-launch step, entries (page, step number)
+    size_t hist;      // uint32 [BH][kStepBins]: score histogram of a head, all zero between steps
     size_t total;
 };
 
 WorkspaceLayout workspace_layout(const rq_config &c);
 
-// ---- kernel launchers (defined in rq_scan.cu / rq_decode.cu) ----
+// ---- kernel launchers (defined in rq_scan.cu, rq_score.cu, rq_topk.cu, rq_attend.cu, rq_step.cu) ----
 struct ScanArgs {
     const void *k, *v, *g;
     int64_t sb, st, sh;     // element strides of k, v, g
@@ -49,6 +60,7 @@ struct ScanArgs {
     float *state;
     int B, H, D, S, dtype, gate_dtype;
     int64_t len0, T, page_cap;
+    float *absmax;      // [2][BH] largest |stored key| per head, both copies brought up to date (NULL: not tracked)
 };
 cudaError_t launch_scan(const ScanArgs &a, cudaStream_t s);
 
@@ -60,6 +72,9 @@ struct DecodeArgs {
     int64_t page_cap;
     int n_sink, n_local;
     int32_t *status;
+    float *absmax;      // [2][BH] largest |stored key| per head (NULL: not tracked); copy `epoch & 1` is current
+    int32_t epoch;      // number of the decode step (1, 2, ...); 0 outside decode steps
+    int32_t poll_limit; // polls after which a device-side wait gives up
 };
 // a.len is the length the scores are for.  do_update: first append the token (k_t, v_t, g_t) as
 // position a.len - 1 (state, cache row, newest page's bounds).  next: the scoring ticket counters
@@ -85,6 +100,27 @@ struct AttendCounters {
 cudaError_t launch_attend(const DecodeArgs &a, const void *q, const int32_t *idx, int n_idx,
                           int idx_stride, float scale, float *partial, const AttendCounters &ctr, void *o,
                           int sm_count, cudaStream_t s);
+// The whole decode step in one launch (rq_step.cu): append, scoring, selection, flash-decode and
+// combine, the heads split into `waves` groups so that the selection of one group runs behind the
+// streams of the others.  step_plan says whether the shape qualifies and with how many waves
+// (0: use the separate kernels); list receives every head's pages in no particular order, every
+// entry tagged with the step's number.
+struct StepBuffers {
+    float *scores;      // [BH][page_cap]
+    int2 *list;         // [BH][list_stride]
+    int list_stride;
+    float *partial;     // [BH][slots][D + 4]
+    int slots;
+    int32_t *ctr;       // [2][BH][kStepCtrInts]
+    uint32_t *hist;     // [BH][kStepBins]
+};
+int step_plan(const DecodeArgs &a, int budget, int sm_count, int forced_waves, int *grid_out);
+cudaError_t launch_step(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t, int budget,
+                        float scale, const StepBuffers &b, void *o, int waves, int grid, cudaStream_t s);
+// sel (any order, K valid entries per head) -> out ascending, tail -1
+cudaError_t launch_sort_list(const int2 *sel, int sel_stride, int K, int P, int BH, int32_t *out, int out_stride,
+                             cudaStream_t s);
+
 // Grid of a streaming kernel for a number of work units spread evenly over `heads` heads: at
 // most what the device holds at once, at least two units per warp, and a whole number of CTAs per
 // head if that keeps at least 85 % of the CTAs (heads served by more CTAs than others would
@@ -95,5 +131,7 @@ int stream_grid(int64_t units, int heads, int resident_ctas, int warps_per_cta, 
 int attend_grid(int64_t tiles, int heads, int resident_ctas);
 // partial records a head can need when it has this many tiles
 int attend_slots_per_head(int64_t tiles_per_head);
+// SMs of the current device
+int sm_count();
 
 }  // namespace rq

@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
 
     T *kv = static_cast<T *>(a.kv);
     T *meta = static_cast<T *>(a.meta);
+    float amax = 0.0f;                           // largest |stored key| this thread has written
 
     // one tile; FULL: every row of the tile is a new token, so no row needs a range check
     auto tile = [&](auto full_tag, int i, int lo, int hi, int fill_hi) {
@@ -282,6 +283,7 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
                 store2(vs + e, z0, z1);
             }
         }
+        if (mn0 <= mx0) amax = fmaxf(amax, fmaxf(fmaxf(-mn0, mx0), fmaxf(-mn1, mx1)));   // this run held new tokens
         // the warp's two runs together (16 positions)
         mn0 = fminf(mn0, __shfl_xor_sync(FULLMASK, mn0, 16)); mn1 = fminf(mn1, __shfl_xor_sync(FULLMASK, mn1, 16));
         mx0 = fmaxf(mx0, __shfl_xor_sync(FULLMASK, mx0, 16)); mx1 = fmaxf(mx1, __shfl_xor_sync(FULLMASK, mx1, 16));
@@ -354,6 +356,14 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
     if (tid < CG) {                              // the state after the last token
         a.state[(int64_t)bh * 2 * D + c0 + tid] = carry[ntiles & 1][0][tid];
         a.state[(int64_t)bh * 2 * D + D + c0 + tid] = carry[ntiles & 1][1][tid];
+    }
+    if (a.absmax) {
+        // the head's largest |stored key| (both copies): non-negative floats order like their bit patterns
+        const unsigned m = __reduce_max_sync(FULLMASK, __float_as_uint(amax));
+        if (lane == 0 && m != 0u) {
+            atomicMax(reinterpret_cast<unsigned *>(a.absmax) + bh, m);
+            atomicMax(reinterpret_cast<unsigned *>(a.absmax) + (int64_t)a.B * a.H + bh, m);
+        }
     }
 }
 

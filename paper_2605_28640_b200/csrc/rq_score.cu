@@ -61,6 +61,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     const int wg = blockIdx.x * NW + warp;
 
     const uint64_t stream_policy = l2_evict_first_policy();
+    const int poll_limit = a.poll_limit == 0 ? kMbarPollLimit : (a.poll_limit < 0 ? 0 : a.poll_limit);
     uint64_t *mybars = bars + warp * DEPTH;
     int4 *myinfo = infos + warp * DEPTH;
     unsigned char *myring = ring + (size_t)warp * DEPTH * kUnitBytes;
@@ -175,9 +176,10 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
             score_load_q<T, D>(q, cur, lane, qs);
         }
         if (!dead) {
-            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u)) {
+            if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u, poll_limit)) {
+                // give every copy in flight (this one too) the usual bounded chance to land, then stop
                 for (int s = 0; s < DEPTH; ++s)
-                    if (s != stage && myinfo[s].x >= 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
+                    if (myinfo[s].x >= 0) mbar_wait(&mybars[s], (phase >> s) & 1u);
                 if (lane == 0) atomicExch(a.status, RQ_ERR_TIMEOUT);
                 dead = true;
             }

@@ -1,5 +1,5 @@
 // Arithmetic of the two streaming kernels on ONE unit of data that already sits in shared
-// memory, shared by the stand-alone kernels and the fused decode kernel:
+// memory, shared by the stand-alone kernels and the one-launch decode step:
 //   score_unit   — Quest upper bounds of the page records of one 8 KiB unit (Eq. 3)
 //   attend_tile  — one 16-row tile of a selected page folded into a warp's online softmax (Eq. 4)
 //   combine_head — merge of a head's partial results
@@ -59,10 +59,15 @@ __device__ __forceinline__ void score_load_q(const T *q, int h, int lane, float 
     }
 }
 
-// Scores of the first `n` records of the unit at `ub` (shared memory) -> out[0 .. n).
-template <typename T, int D>
+struct NoEmit {
+    __device__ __forceinline__ void operator()(int, float) const {}
+};
+
+// Scores of the first `n` records of the unit at `ub` (shared memory) -> out[0 .. n); emit(r, score)
+// is called by the lane that writes record r's score.
+template <typename T, int D, typename Emit = NoEmit>
 __device__ __forceinline__ void score_unit(const unsigned char *ub, const float (*qs)[VecOf<T>::N], int n,
-                                           float *out, int lane)
+                                           float *out, int lane, Emit emit = Emit())
 {
     using G = ScoreGeom<T, D>;
     constexpr int CH = G::CH, LPP = G::LPP, VPL = G::VPL, PPW = G::PPW, NR = G::NR;
@@ -110,7 +115,10 @@ __device__ __forceinline__ void score_unit(const unsigned char *ub, const float 
     const int gi = (c >> (LOG_LPP - LOG_NR)) & (NR - 1);
     const bool writer = (c & ((1 << (LOG_LPP - LOG_NR)) - 1)) == 0;
     const int r = gi * PPW + sub;
-    if (writer && r < n) out[r] = val[0];
+    if (writer && r < n) {
+        out[r] = val[0];
+        emit(r, val[0]);
+    }
 }
 
 // ---------------------------------------------------------------- attention
@@ -302,17 +310,20 @@ __device__ __forceinline__ void combine_head(const float *src, int n, T *o_row, 
 
 // ---------------------------------------------------------------- append
 // One step of Eq. 1 for head h (thread d < D owns channel d): new state, cache row, bounds of
-// the newest page, and that page's score.  `len` is the length AFTER the append.
+// the newest page, and that page's score (returned to thread 0).  `len` is the length AFTER the
+// append.  red: 16 floats of shared memory.  The head's largest |stored key| is brought up to date
+// in the copy that the NEXT step reads; with write_current also in the copy of this step (only
+// when nobody reads that copy while this runs).
 template <typename T, int D>
-__device__ __forceinline__ void update_head(const DecodeArgs &a, int h, const T *q, const T *k_t, const T *v_t,
-                                            const void *g_t, float *scores, float *red)
+__device__ __forceinline__ float update_head(const DecodeArgs &a, int h, const T *q, const T *k_t, const T *v_t,
+                                             const void *g_t, float *scores, float *red, bool write_current = true)
 {
     const int d = threadIdx.x;
     const int S = a.S;
     const int64_t pos = a.len - 1;
     const int64_t page = pos / S;
     const int slot = (int)(pos % S);
-    float term = 0.0f;
+    float term = 0.0f, amax = 0.0f;
     if (d < D) {
         float *st = a.state + (int64_t)h * 2 * D;
         const float g = a.gate_dtype == RQ_BF16 ? load1<bf16>(static_cast<const bf16 *>(g_t) + (int64_t)h * D + d)
@@ -326,6 +337,7 @@ __device__ __forceinline__ void update_head(const DecodeArgs &a, int h, const T 
         store1<T>(pg + (int64_t)slot * D + d, sk);
         store1<T>(pg + (int64_t)(S + slot) * D + d, sv);
         const float r = round_storage<T>(sk);
+        amax = fabsf(r);
         T *m = static_cast<T *>(a.meta) + (((int64_t)h * a.page_cap + page) * 2) * D;
         float mn = r, mx = r;
         if (slot == 0) {
@@ -343,18 +355,61 @@ __device__ __forceinline__ void update_head(const DecodeArgs &a, int h, const T 
         const float qd = load1<T>(q + (int64_t)h * D + d);
         term = fmaxf(qd * mn, qd * mx);
     }
-    // score of the newest page: sum of the D terms
+    // score of the newest page: sum of the D terms; largest |stored key| of the new row
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) term += __shfl_xor_sync(0xffffffffu, term, off);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = term;
+    for (int off = 16; off > 0; off >>= 1) {
+        term += __shfl_xor_sync(0xffffffffu, term, off);
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+    }
+    if ((threadIdx.x & 31) == 0 && threadIdx.x < D) { red[threadIdx.x >> 5] = term; red[8 + (threadIdx.x >> 5)] = amax; }
     __syncthreads();
+    float s = 0.0f;
     if (threadIdx.x == 0) {
-        float s = 0.0f;
-        for (int w = 0; w < (D + 31) / 32; ++w) s += red[w];
+        float m = 0.0f;
+        for (int w = 0; w < (D + 31) / 32; ++w) { s += red[w]; m = fmaxf(m, red[8 + w]); }
         scores[(int64_t)h * a.page_cap + page] = s;
+        if (a.absmax) {
+            const int BH = a.B * a.H, cur = a.epoch & 1;
+            const float nv = fmaxf(a.absmax[cur * BH + h], m);
+            a.absmax[(cur ^ 1) * BH + h] = nv;
+            if (write_current) a.absmax[cur * BH + h] = nv;
+        }
     }
     __syncthreads();
+    return s;
 }
+
+// ---------------------------------------------------------------- a-priori score range
+// Every page score of head h lies in [-R, R] with R = A * sum_i |q_i|, A the largest |stored key|
+// of the head (|U_p| <= sum_i |q_i| max(|min_p[i]|, |max_p[i]|)).  The one-launch step spreads
+// kStepBins value buckets over that range BEFORE any score exists: bucket(u) = clamp(floor((u + R) *
+// scale)), monotone in u whatever R is, so a stale or loose range costs resolution, never
+// correctness.  Every warp computes the same bits (same order of operations).
+struct ScoreRange {
+    float lo, scale;
+    __device__ __forceinline__ int bucket(float u) const
+    {
+        const float f = (u - lo) * scale;
+        return min(max((int)f, 0), kStepBins - 1);   // a NaN product lands in bucket 0
+    }
+};
+template <typename T, int D>
+__device__ __forceinline__ ScoreRange score_range(const T *q, int h, float amax, int lane)
+{
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) s += fabsf(load1<T>(q + (int64_t)h * D + lane + 32 * i));
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    const float R = amax * s;
+    ScoreRange r;
+    r.lo = -R;
+    r.scale = (0.5f * (float)kStepBins) / R;
+    // an empty or unbounded range: one bucket for everything (the selection then works on the key bits)
+    if (!(R > 0.0f) || !(r.scale < CUDART_INF_F) || !(R < CUDART_INF_F)) { r.lo = 0.0f; r.scale = 0.0f; }
+    return r;
+}
+
 
 
 }  // namespace rq

@@ -135,11 +135,7 @@ __device__ __forceinline__ void scan_warp_counts(SelectScratch &sh, uint32_t wgt
     eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
 }
 
-// the score a key was made from (inverse of order_key)
-__device__ __forceinline__ float key_value(uint32_t k)
-{
-    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
+__device__ __forceinline__ float key_value(uint32_t k) { return order_key_value(k); }
 
 // clears what select_rows expects to find clear; a CTA barrier must lie between the two
 __device__ __forceinline__ void select_prepare(SelectScratch &sh)

@@ -26,3 +26,15 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Worst errors and near-tie counts the staged comparison saw in this run."""
+    try:
+        import parity
+    except Exception:
+        return
+    if parity.OBSERVED:
+        terminalreporter.write_sep("-", "staged comparison with the oracle: observed")
+        for k in sorted(parity.OBSERVED):
+            terminalreporter.write_line(f"{k}: {parity.OBSERVED[k]:.6g}")

@@ -27,11 +27,30 @@ import torch
 import oracle
 
 ODT = {torch.float32: oracle.F32, torch.bfloat16: oracle.BF16}
+
+# Worst values and counts seen by the checks of this process; a test run prints them at its end
+# (tests/conftest.py) and the benchmark puts them into its `parity` block.
+OBSERVED = {}
+
+
+def note_max(name, value):
+    OBSERVED[name] = max(OBSERVED.get(name, 0.0), float(value))
+
+
+def note_count(name, n=1):
+    OBSERVED[name] = OBSERVED.get(name, 0) + n
 ATT_TOL = {torch.bfloat16: (2e-2, 5e-3), torch.float32: (1e-4, 1e-5)}
 
 
 def f64(t):
     return t.detach().to(torch.float64).cpu().numpy()
+
+
+# Absolute floor of the state comparison, in units of the state's rms: a channel that cancels to
+# near zero carries the rounding error of its terms, not of its value.  fp32 rounding of the
+# recurrence leaves about eps/(1-g) relative to the terms' size; the largest error observed over
+# the whole GPU suite (tests/conftest.py prints it) is well below this floor.
+STATE_FLOOR = 1e-5
 
 
 def storage_ulp(x, dtype):
@@ -44,7 +63,11 @@ def storage_ulp(x, dtype):
 def assert_state_close(gpu, ref, what):
     rms = float(np.sqrt(np.mean(ref ** 2))) or 1.0
     err = np.abs(gpu - ref)
-    tol = 1e-4 * np.abs(ref) + 1e-5 * rms
+    note_max("state_abs_err_over_rms", err.max() / rms)
+    big = np.abs(ref) >= 0.05 * rms
+    if big.any():
+        note_max("state_rel_err_where_ref_ge_0.05rms", (err[big] / np.abs(ref[big])).max())
+    tol = 1e-4 * np.abs(ref) + STATE_FLOOR * rms
     assert (err <= tol).all(), f"{what}: max excess {(err - tol).max():.3e} (rms {rms:.3e})"
 
 
@@ -86,6 +109,7 @@ def check_cache_level(cache, hd, b, h, dtype):
             continue
         ne = a != r
         frac = ne.mean() if a.size else 0.0
+        note_max("stored_fraction_one_step_off", frac)
         assert frac <= 1e-3, f"{name}[{b},{h}]: {frac:.2e} of stored values differ"
         if ne.any():
             # one rounding step apart, or (for values that are near zero by cancellation, where
@@ -93,7 +117,7 @@ def check_cache_level(cache, hd, b, h, dtype):
             gap = np.abs(a - r)[ne]
             ulp = storage_ulp(np.maximum(np.abs(a), np.abs(r)), dtype)[ne]
             rms = float(np.sqrt(np.mean(r ** 2)))
-            slack = (1e-4 * np.abs(r) + 1e-5 * rms)[ne]
+            slack = (1e-4 * np.abs(r) + STATE_FLOOR * rms)[ne]
             bad = gap > np.maximum(ulp * 1.0000001, slack)
             assert not bad.any(), (f"{name}[{b},{h}]: {bad.sum()} stored values are more than one "
                                    f"rounding step off (worst gap {gap[bad].max():.3e})")
@@ -127,7 +151,11 @@ def check_query_level(dev, hd, cache, b, h, q, K, scale, o, idx, scores, dtype, 
     got = got[:n]
     assert (np.diff(got) > 0).all(), "page list must be strictly ascending"
     stats["heads"] = stats.get("heads", 0) + 1
+    note_count("heads_checked")
+    if near:
+        note_count("near_tie_heads")
     if not np.array_equal(got, want):
+        note_count("near_tie_mismatches")
         assert near, f"pages [{b},{h}] differ from the oracle's with no near-tie at the cut"
         # whatever was swapped must sit within 1e-5 relative of the cut
         sel_o = set(want.tolist())
@@ -147,6 +175,9 @@ def check_query_level(dev, hd, cache, b, h, q, K, scale, o, idx, scores, dtype, 
     assert err.max() <= mx_tol and err.mean() <= mean_tol, \
         f"attention[{b},{h}]: max {err.max():.3e} mean {err.mean():.3e}"
     stats["att_max"] = max(stats.get("att_max", 0.0), float(err.max()))
+    stats["att_mean"] = max(stats.get("att_mean", 0.0), float(err.mean()))
+    note_max("attention_max_abs_err_" + str(dtype).replace("torch.", ""), err.max())
+    note_max("attention_mean_abs_err_" + str(dtype).replace("torch.", ""), err.mean())
     # end to end: the oracle's own chain from the raw inputs
     e2e = hd.query(q64, K, scale)
     if np.array_equal(e2e["idx"], got):

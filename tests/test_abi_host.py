@@ -123,6 +123,31 @@ def test_argument_checks_on_a_filled_in_handle(lib):
     assert lib.rq_select_pages(C.byref(cache), 256, 1, None, 256, None) == rq.RQ_ERR_INVALID_ARG   # empty cache
 
 
+def _no_gpu():
+    import torch
+    return not torch.cuda.is_available()
+
+
+@pytest.mark.skipif(not _no_gpu(), reason="drives the launch code with made-up pointers: only where no launch can succeed")
+def test_failed_launch_leaves_length_and_step_count_unchanged(lib):
+    """Without a device every CUDA call fails: the step must return RQ_ERR_CUDA and roll nothing forward."""
+    c = cfg(capacity_tokens=1 << 16, max_budget_pages=64)
+    cache = rq.rq_cache()
+    cache.cfg = c
+    cache.kv = cache.meta = cache.state = cache.workspace = 4096
+    cache.page_capacity = (1 << 16) // 16
+    cache.len = 20000
+    cache.reserved[0] = 7
+    for path in (0, 1, 2):
+        cache.reserved[2] = path
+        assert lib.rq_decode_step(C.byref(cache), 256, 256, 256, 256, 64, 0.0, 256, None, None) == rq.RQ_ERR_CUDA
+        assert cache.len == 20000 and cache.reserved[0] == 7
+    assert lib.rq_build_cache(C.byref(cache), 256, 256, 256, 16, 1 << 20, 4096, 128, None) == rq.RQ_ERR_CUDA
+    assert cache.len == 20000
+    assert lib.rq_decode_step_launches(C.byref(cache), 64) == 3       # no device: nothing to plan a single launch with
+    assert lib.rq_decode_step_launches(None, 64) == -1
+
+
 def test_workload_generators_are_seeded_and_shaped():
     import torch
     from paper_2605_28640_b200 import workloads as wl

@@ -18,13 +18,16 @@ DEV = "cuda"
 
 
 def run_case(w, T_prefill, steps=1, heads=None, n_sink=1, n_local=1, scale=0.0, chunks=None,
-             budget=None, stats=None):
+             budget=None, stats=None, path=0, want_launches=None):
     """Prefill T_prefill tokens (optionally in several rq_build_cache calls), then run decode
-    steps, checking every level after the prefill and after every step for the sampled heads."""
+    steps, checking every level after the prefill and after every step for the sampled heads.
+    path: rq_cache.reserved[2] (0: the library chooses how the step is launched, 1: separate
+    kernels, 2 / 4 / 8: one launch with that many groups of heads)."""
     stats = {} if stats is None else stats
     cap = T_prefill + steps + 3
     maxK = max(w.pages(cap), budget or 1)
     cache = rq.Cache(w.B, w.H, w.D, w.S, cap, w.dtype, w.gdtype, n_sink, n_local, maxK)
+    cache.handle.reserved[2] = path
     q0 = wl.make_query(w, DEV, 0)
     k, v, g = wl.make_prefill(w, DEV, T_prefill, q_for_needles=q0 if w.needles else None)
     bounds = [0, *(chunks or []), T_prefill]
@@ -44,6 +47,8 @@ def run_case(w, T_prefill, steps=1, heads=None, n_sink=1, n_local=1, scale=0.0, 
         K = budget if budget is not None else w.budget_pages(T)
         o = torch.empty(w.B, w.H, w.D, dtype=w.dtype, device=DEV)
         idx = torch.full((w.B, w.H, K), -7, dtype=torch.int32, device=DEV)
+        if want_launches is not None:
+            assert rq.rq_decode_step_launches(cache.handle, K) == want_launches
         rq.rq_decode_step(cache.handle, q, kt, vt, gt, K, scale, o, idx)
         assert len(cache) == T
         P = w.pages(T)
@@ -149,7 +154,7 @@ def test_multistep_decode_batched():
 def test_config1_all_heads():
     """Config 1: batch 1, 32 heads, D 128, context 16384, budget 1/16 (64 pages), bf16."""
     w = wl.CONFIGS[1]
-    _, stats = run_case(w, w.T - 1, steps=1)
+    _, stats = run_case(w, w.T - 1, steps=1, want_launches=1)     # the whole step is one launch at this shape
     assert stats["heads"] == 32
     assert stats["e2e_overlap"] / stats["heads"] >= 0.99
 
