@@ -101,7 +101,7 @@ typedef struct rq_cache {
     void *workspace;
     int64_t len;           /* tokens currently in every sequence                           */
     int64_t page_capacity; /* ceil(capacity_tokens / page_size)                            */
-    /* reserved[0]: decode steps that ran as one launch so far (kept by the library).
+    /* reserved[0]: decode steps taken so far (kept by the library).
      * reserved[1]: testing aid: poll limit of the device-side waits for asynchronous copies;
      *              0 = the built-in limit, < 0 = no poll at all, so that the first wait of every
      *              warp gives up, the kernels let their copies land and return, and the device
@@ -247,11 +247,12 @@ RQ_API int64_t rq_cache_len(const rq_cache *cache);
 
 /* Kernel launches the next rq_decode_step on this cache will enqueue for this budget when
  * sel_idx_out is NULL [no counterpart in the paper: bookkeeping for benchmarks]: ONE when the whole
- * step runs as one launch (at most 256 (batch, head) pairs that split into 2, 4 or 8 equal groups
- * which keep the GPU's resident CTAs busy, more than 256 pages per head, budget below the number
- * of pages; a non-NULL sel_idx_out adds a launch that sorts the list); otherwise three (update +
- * scoring, selection, attention), or two when the context is short enough (at most 256 pages per
- * head, at least 16 heads) for one CTA per head to do the first two kernels' work in one launch.
+ * step runs as one launch (chosen by the library for 64 to 128 (batch, head) pairs of 4096 to
+ * 12284 pages each that split into 4, 8 or 2 equal groups which keep the GPU's resident CTAs
+ * busy, budget below the number of pages; cache.reserved[2] asks for it on other shapes);
+ * otherwise three (update + scoring, selection, attention), or two when the context is short
+ * enough (at most 256 pages per head, at least 16 heads) for one CTA per head to do the first
+ * two kernels' work in one launch.  A non-NULL sel_idx_out can add a launch that sorts the list.
  * The first call on a device looks up launch parameters (occupancy).  -1 for an invalid cache. */
 RQ_API int rq_decode_step_launches(const rq_cache *cache, int32_t budget_pages);
 

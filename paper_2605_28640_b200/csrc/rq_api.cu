@@ -41,6 +41,7 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     w.step_ctr = off; off += align256(2 * SH * (size_t)kStepCtrInts * sizeof(int32_t));
     w.list = off;     off += align256(SH * (size_t)c.max_budget_pages * sizeof(int2));
     w.hist = off;     off += align256(SH * (size_t)kStepBins * sizeof(uint32_t));
+    w.range = off;    off += align256(SH * sizeof(float2));
     w.scores = off;  off += align256(BH * pc * sizeof(float));
     w.sel = off;     off += align256(BH * (size_t)c.max_budget_pages * sizeof(int32_t));
     const size_t slots = (size_t)attend_slots_per_head((int64_t)c.max_budget_pages * (c.page_size / 16));
@@ -83,12 +84,13 @@ int sm_count()
     return cached[dev];
 }
 
-// rq_cache::reserved: [0] number of decode steps that ran as one launch (that path alternates between
-// two sets of counters and two copies of the heads' largest |stored key|; every step, whatever its
-// path, works as step number reserved[0] + 1 and only a one-launch step commits that number, so the
-// copy with parity reserved[0] + 1 is always the up-to-date one), [1] poll limit of device-side copy waits (0: the default, < 0: none at all; a
-// testing aid), [2] choice of the decode path (0: automatic, 1: always the separate kernels,
-// 2, 4, 8: the one-launch step with that many waves whenever the shape allows it)
+// rq_cache::reserved: [0] number of decode steps taken; a step works as step number reserved[0] + 1
+// and commits that number when all its launches succeeded.  (Its parity picks the copy of the
+// heads' largest |stored key| that the step reads, the update writing the other one, and the set of
+// per-head counters the one-launch step uses, the step clearing the other one.)  [1] poll limit of
+// device-side copy waits (0: the default, < 0: none at all; a testing aid), [2] choice of the decode
+// path (0: automatic, 1: always the separate kernels, 2, 4, 8: the one-launch step with that many
+// waves whenever the shape allows it)
 static float *absmax_of(const rq_cache *c)
 {
     if ((int64_t)c->cfg.batch * c->cfg.heads > kStepMaxHeads) return nullptr;
@@ -126,26 +128,52 @@ static void mark(cudaEvent_t *ev, int i, cudaStream_t s)
 }
 
 // (optionally append a token, then) score + select into `idx` (device, stride idx_stride), for a
-// cache of length len after the append
+// cache of length len after the append.  *unordered: the list came out in no particular order.
 static int select_into(const rq_cache *c, int64_t len, const void *q, const void *k_t, const void *v_t,
                        const void *g_t, int do_update, int budget, float *scores, int32_t *idx, int idx_stride,
-                       cudaStream_t s, cudaEvent_t *ev = nullptr)
+                       cudaStream_t s, cudaEvent_t *ev = nullptr, bool *unordered = nullptr)
 {
     DecodeArgs a = decode_args(c, len);
-    int32_t *ctr = (int32_t *)((char *)c->workspace + workspace_layout(c->cfg).tickets);
+    const WorkspaceLayout w = workspace_layout(c->cfg);
+    int32_t *ctr = (int32_t *)((char *)c->workspace + w.tickets);
     const int64_t P = (len + c->cfg.page_size - 1) / c->cfg.page_size;
+    if (unordered) *unordered = false;
     if (P <= kSmallStepPages && c->cfg.batch * c->cfg.heads >= kSmallStepMinHeads) {
         // a short context: one launch instead of two (the per-kernel marks then show the whole under "score")
-        if (launch_score_select(a, q, k_t, v_t, g_t, scores, do_update, budget, idx, idx_stride, ctr, do_update, s) !=
+        int32_t *other = a.absmax && do_update ? (int32_t *)((char *)c->workspace + w.step_ctr) +
+                                                     (size_t)((a.epoch & 1) ^ 1) * a.B * a.H * kStepCtrInts
+                                               : nullptr;
+        if (launch_score_select(a, q, k_t, v_t, g_t, scores, do_update, budget, idx, idx_stride, ctr, do_update, other, s) !=
             cudaSuccess)
             return RQ_ERR_CUDA;
         mark(ev, 1, s);
         mark(ev, 2, s);
         return RQ_OK;
     }
-    if (launch_score(a, q, k_t, v_t, g_t, scores, ctr + 3, do_update, sm_count(), s) != cudaSuccess) return RQ_ERR_CUDA;
+    // forced pages inside the budget (sinks first, then local pages from the newest backwards): the
+    // scoring kernel leaves them out of its histogram, the selection takes them outright
+    const int K = (int)(budget < P ? budget : P);
+    int ns = a.n_sink < K ? a.n_sink : K;
+    if (ns > P) ns = (int)P;
+    int nl = a.n_local < K - ns ? a.n_local : K - ns;
+    if (nl > P - ns) nl = (int)(P - ns);
+    a.n_sink = ns;
+    a.n_local = nl;
+    // the scoring kernel counts the scores into value buckets for the selection when the heads are
+    // few and short enough for that path and the budget leaves something to select
+    ScoreHist hs = {nullptr, nullptr, nullptr};
+    if (a.absmax) {
+        char *ws = (char *)c->workspace;
+        if (do_update) hs.ctr_other = (int32_t *)(ws + w.step_ctr) + (size_t)((a.epoch & 1) ^ 1) * a.B * a.H * kStepCtrInts;
+        if (topk_uses_hist(P) && K < P) {
+            hs.hist = (uint32_t *)(ws + w.hist);
+            hs.range = (float2 *)(ws + w.range);
+            if (unordered) *unordered = true;
+        }
+    }
+    if (launch_score(a, q, k_t, v_t, g_t, scores, ctr + 3, do_update, hs, sm_count(), s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 1, s);
-    if (launch_topk(a, scores, budget, idx, idx_stride, ctr, do_update, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (launch_topk(a, scores, budget, idx, idx_stride, ctr, do_update, hs, s) != cudaSuccess) return RQ_ERR_CUDA;
     mark(ev, 2, s);
     return RQ_OK;
 }
@@ -228,11 +256,17 @@ static int decode_step_impl(rq_cache *cache, const void *q, const void *k_t, con
         mark(ev, 3, s);
         if (st == RQ_OK) cache->reserved[0] += 1;
     } else {
-        st = select_into(cache, new_len, q, k_t, v_t, g_t, 1, budget_pages, scores, sel, budget_pages, s, ev);
+        bool unordered = false;
+        st = select_into(cache, new_len, q, k_t, v_t, g_t, 1, budget_pages, scores, sel, budget_pages, s, ev, &unordered);
         if (st == RQ_OK) {
             const int n_idx = (int)(budget_pages < P ? budget_pages : P);
             st = attend_from(cache, new_len, q, sel, n_idx, budget_pages, scale, o, s, ev);
         }
+        // the caller's copy of the list is ascending (in place, behind the attention kernel, which does not care)
+        if (st == RQ_OK && unordered && sel_idx_out &&
+            launch_sort_list32(sel, budget_pages, budget_pages, (int)P, c.batch * c.heads, sel, budget_pages, s) != cudaSuccess)
+            st = RQ_ERR_CUDA;
+        if (st == RQ_OK) cache->reserved[0] += 1;
     }
     if (st != RQ_OK) return st;
     cache->len = new_len;
@@ -476,8 +510,14 @@ int rq_select_pages(rq_cache *cache, const void *q, int32_t budget_pages, float 
     cudaStream_t s = (cudaStream_t)stream;
     const WorkspaceLayout w = workspace_layout(c);
     float *scores = (float *)((char *)cache->workspace + w.scores);
-    const int st = select_into(cache, cache->len, q, nullptr, nullptr, nullptr, 0, budget_pages, scores, idx_out, budget_pages, s);
+    bool unordered = false;
+    const int st = select_into(cache, cache->len, q, nullptr, nullptr, nullptr, 0, budget_pages, scores, idx_out, budget_pages, s,
+                               nullptr, &unordered);
     if (st != RQ_OK) return st;
+    const int64_t Pn = (cache->len + c.page_size - 1) / c.page_size;
+    if (unordered && launch_sort_list32(idx_out, budget_pages, budget_pages, (int)Pn, c.batch * c.heads, idx_out, budget_pages,
+                                        s) != cudaSuccess)
+        return RQ_ERR_CUDA;
     if (scores_out) {
         const int64_t P = (cache->len + c.page_size - 1) / c.page_size;
         // workspace rows are page_capacity apart; the caller's are P apart

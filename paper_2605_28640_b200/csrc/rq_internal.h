@@ -32,6 +32,7 @@ constexpr int kTargetSMs = 148;        // B200
 constexpr int kStepMaxHeads = 256;     // the one-launch step serves at most this many (batch, head) pairs
 constexpr int kStepBins = 2048;        // value buckets of a head's score histogram
 constexpr int kStepCtrInts = 16;       // int32 per head and counter set (64 bytes)
+constexpr int kTopkFastPages = 10240;  // heads of up to this many pages are selected from the scoring kernel's histogram
 
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
@@ -47,6 +48,7 @@ struct WorkspaceLayout {
     size_t step_ctr;  // int32 [2][BH][kStepCtrInts]: two sets of per-head counters, used by alternate steps
     size_t list;      // int2 [BH][max_budget]: page lists of the one-launch step, entries (page, step number)
     size_t hist;      // uint32 [BH][kStepBins]: score histogram of a head, all zero between steps
+    size_t range;     // float2 [BH]: (lo, scale) of the bucket map the head's histogram was filled with
     size_t total;
 };
 
@@ -79,17 +81,28 @@ struct DecodeArgs {
 // a.len is the length the scores are for.  do_update: first append the token (k_t, v_t, g_t) as
 // position a.len - 1 (state, cache row, newest page's bounds).  next: the scoring ticket counters
 // (head h at next[h * kCtrStride]), zero at launch.
+// Histogram of the scores for the selection that follows (NULL members: none is kept): every page
+// that competes for the budget adds one to its value bucket; the bucket map of a head goes to range.
+struct ScoreHist {
+    uint32_t *hist;     // [BH][kStepBins], all zero at launch
+    float2 *range;      // [BH] (lo, scale)
+    int32_t *ctr_other; // [BH][kStepCtrInts]: the one-launch step's counters of the next step, cleared here
+};
 cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
-                         float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s);
+                         float *scores, int32_t *next, int do_update, const ScoreHist &sh, int sm_count, cudaStream_t s);
 // attend_ctr: the ticket counters of the streaming kernels (cleared here, one head per CTA)
 // Short contexts: the work of launch_score and launch_topk in one launch, one CTA per head (at most
 // kSmallStepPages pages per head).
 cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
                                 float *scores, int do_update, int budget, int32_t *idx, int idx_stride,
-                                int32_t *attend_ctr, int prefetch, cudaStream_t s);
+                                int32_t *attend_ctr, int prefetch, int32_t *ctr_other, cudaStream_t s);
 // prefetch: the flash-decode kernel runs next, start moving the first selected pages into L2
+// sh: the histogram the scoring kernel filled (NULL members: none).  With it, and at most
+// kTopkFastPages pages, the list comes out in no particular order; otherwise ascending.
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, int32_t *attend_ctr, int prefetch, cudaStream_t s);
+                        int idx_stride, int32_t *attend_ctr, int prefetch, const ScoreHist &sh, cudaStream_t s);
+// does launch_topk take the histogram path for this many pages per head?
+bool topk_uses_hist(int64_t pages);
 // per-head counters of the flash-decode kernel, kCtrStride int32 apart from head to head; all
 // zero at launch
 struct AttendCounters {
@@ -117,6 +130,8 @@ struct StepBuffers {
 int step_plan(const DecodeArgs &a, int budget, int sm_count, int forced_waves, int *grid_out);
 cudaError_t launch_step(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t, int budget,
                         float scale, const StepBuffers &b, void *o, int waves, int grid, cudaStream_t s);
+cudaError_t launch_sort_list32(const int32_t *sel, int sel_stride, int K, int P, int BH, int32_t *out, int out_stride,
+                               cudaStream_t s);
 // sel (any order, K valid entries per head) -> out ascending, tail -1
 cudaError_t launch_sort_list(const int2 *sel, int sel_stride, int K, int P, int BH, int32_t *out, int out_stride,
                              cudaStream_t s);

@@ -39,7 +39,7 @@ namespace {
 template <typename T, int D>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, const T *q, const T *k_t,
                                                                  const T *v_t, const void *g_t, float *scores,
-                                                                 int32_t *next, int do_update)
+                                                                 int32_t *next, int do_update, ScoreHist hs)
 {
     using G = ScoreGeom<T, D>;
     constexpr int CH = G::CH, RU = G::RU, VPL = G::VPL;
@@ -74,8 +74,18 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     grid_dependency_wait();          // earlier kernels may still read what the update rewrites
     grid_launch_dependents();
 
+    const int hcur = a.epoch & 1;                    // copy of the heads' largest |stored key| that this step reads
+    // forced pages inside the budget do not compete: they are not counted (the caller passes them)
+    const int p_lo = hs.hist ? a.n_sink : 0, p_hi = hs.hist ? P - a.n_local : 0;
     if (do_update)
-        for (int h = blockIdx.x; h < BH; h += NC) update_head<T, D>(a, h, q, k_t, v_t, g_t, scores, red);
+        for (int h = blockIdx.x; h < BH; h += NC) {
+            const float s_new = update_head<T, D>(a, h, q, k_t, v_t, g_t, scores, red);
+            if (hs.ctr_other && threadIdx.x < kStepCtrInts) hs.ctr_other[h * kStepCtrInts + threadIdx.x] = 0;
+            if (hs.hist && warp == 0) {              // the newest page, scored by the update, if it competes
+                const ScoreRange rg = score_range<T, D>(q, h, a.absmax[hcur * BH + h], lane);
+                if (lane == 0 && P - 1 >= p_lo && P - 1 < p_hi) red_inc(hs.hist + (int64_t)h * kStepBins + rg.bucket(s_new));
+            }
+        }
 
     const T *meta = static_cast<const T *>(a.meta);
 
@@ -167,6 +177,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
     int stage = 0;
     uint32_t phase = 0;
     bool dead = false;
+    ScoreRange rg = {0.0f, 0.0f};
 
     for (;;) {
         const int4 inf = myinfo[stage];
@@ -174,6 +185,10 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
         if (inf.x != cur) {
             cur = inf.x;
             score_load_q<T, D>(q, cur, lane, qs);
+            if (hs.hist) {                           // every warp computes the same bits
+                rg = score_range<T, D>(q, cur, a.absmax[hcur * BH + cur], lane);
+                if (lane == 0) hs.range[cur] = make_float2(rg.lo, rg.scale);
+            }
         }
         if (!dead) {
             if (!mbar_wait(&mybars[stage], (phase >> stage) & 1u, poll_limit)) {
@@ -187,7 +202,16 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(DecodeArgs a, c
         }
         if (!dead) {
             const unsigned char *ub = myring + (size_t)stage * kUnitBytes;
-            score_unit<T, D>(ub, qs, inf.z, scores + (int64_t)cur * a.page_cap + inf.y, lane);
+            if (hs.hist) {
+                const int first = inf.y;
+                uint32_t *hist = hs.hist + (int64_t)cur * kStepBins;
+                score_unit<T, D>(ub, qs, inf.z, scores + (int64_t)cur * a.page_cap + first, lane, [&](int r, float u) {
+                    const int p = first + r;
+                    if (p >= p_lo && p < p_hi) red_inc(hist + rg.bucket(u));
+                });
+            } else {
+                score_unit<T, D>(ub, qs, inf.z, scores + (int64_t)cur * a.page_cap + inf.y, lane);
+            }
         }
         __syncwarp();
         if (dead) drained = true;
@@ -224,7 +248,7 @@ cudaError_t score_occupancy(int *ctas_per_sm)
 
 template <typename T, int D>
 cudaError_t launch_score_t(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
-                           float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s)
+                           float *scores, int32_t *next, int do_update, const ScoreHist &hs, int sm_count, cudaStream_t s)
 {
     using G = ScoreGeom<T, D>;
     const int64_t P = (a.len + a.S - 1) / a.S;
@@ -245,21 +269,21 @@ cudaError_t launch_score_t(const DecodeArgs &a, const void *q, const void *k_t, 
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, score_kernel<T, D>, a, (const T *)q, (const T *)k_t, (const T *)v_t, g_t, scores,
-                              next, do_update);
+                              next, do_update, hs);
 }
 
 }  // namespace
 
 cudaError_t launch_score(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
-                         float *scores, int32_t *next, int do_update, int sm_count, cudaStream_t s)
+                         float *scores, int32_t *next, int do_update, const ScoreHist &hs, int sm_count, cudaStream_t s)
 {
     if (a.len <= 0) return cudaSuccess;
     if (a.dtype == RQ_BF16) {
-        if (a.D == 128) return launch_score_t<bf16, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
-        if (a.D == 64) return launch_score_t<bf16, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+        if (a.D == 128) return launch_score_t<bf16, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, hs, sm_count, s);
+        if (a.D == 64) return launch_score_t<bf16, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, hs, sm_count, s);
     } else {
-        if (a.D == 128) return launch_score_t<float, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
-        if (a.D == 64) return launch_score_t<float, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, sm_count, s);
+        if (a.D == 128) return launch_score_t<float, 128>(a, q, k_t, v_t, g_t, scores, next, do_update, hs, sm_count, s);
+        if (a.D == 64) return launch_score_t<float, 64>(a, q, k_t, v_t, g_t, scores, next, do_update, hs, sm_count, s);
     }
     return cudaErrorInvalidValue;
 }

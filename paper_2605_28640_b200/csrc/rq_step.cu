@@ -558,7 +558,7 @@ __global__ void __launch_bounds__(kStepWarps * 32, 3) step_kernel(DecodeArgs a, 
 
     // ------------------------------------------------------------ append (Eq. 1), one CTA per head
     for (int h = blockIdx.x; h < BH; h += stream_ctas) {
-        const float s_new = update_head<T, D>(a, h, q, k_t, v_t, g_t, b.scores, red, false);
+        const float s_new = update_head<T, D>(a, h, q, k_t, v_t, g_t, b.scores, red);
         // the counters of the NEXT step (nobody uses that set while this kernel runs)
         if (threadIdx.x < kStepCtrInts) b.ctr[((int64_t)(cur ^ 1) * BH + h) * kStepCtrInts + threadIdx.x] = 0;
         if (warp == 0) {
@@ -862,20 +862,25 @@ __global__ void __launch_bounds__(kStepWarps * 32, 3) step_kernel(DecodeArgs a, 
 }
 
 // ---------------------------------------------------------------- ascending copy of a page list
-// sel holds K distinct pages of [0, P) per head in any order (entries are (page, step number)): mark
-// them in a bit map, then write the set bits out in order.  One CTA of 1024 threads per head (P <= 32768: one word per thread).
-__global__ void __launch_bounds__(1024) sort_list_kernel(const int2 *sel, int sel_stride, int K, int P, int32_t *out,
+// sel holds K distinct pages of [0, P) per head in any order (entries are pages, or (page, step
+// number) pairs; the kernel may work in place): mark them in a bit map, then write the set bits out
+// in order.  One CTA of 1024 threads per head (P <= 32768: one word per thread).
+__device__ __forceinline__ int list_page(const int2 &e) { return e.x; }
+__device__ __forceinline__ int list_page(const int32_t &e) { return e; }
+
+template <typename E>
+__global__ void __launch_bounds__(1024) sort_list_kernel(const E *sel, int sel_stride, int K, int P, int32_t *out,
                                                          int out_stride)
 {
     __shared__ uint32_t bits[1024];
     __shared__ int wsum[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int2 *src = sel + (int64_t)blockIdx.x * sel_stride;
+    const E *src = sel + (int64_t)blockIdx.x * sel_stride;
     int32_t *dst = out + (int64_t)blockIdx.x * out_stride;
     bits[tid] = 0u;
     __syncthreads();
     for (int i = tid; i < K; i += 1024) {
-        const int p = __ldcg(src + i).x;
+        const int p = list_page(__ldcg(src + i));
         if (p >= 0 && p < P) atomicOr(&bits[p >> 5], 1u << (p & 31));
     }
     __syncthreads();
@@ -972,7 +977,16 @@ int step_plan(const DecodeArgs &a, int budget, int sm_count, int forced_waves, i
     RQ_STEP_DISPATCH(RQ_OCC)
 #undef RQ_OCC
     if (e != cudaSuccess || occ < 1) return 0;
-    for (int waves = 2; waves <= 8; waves *= 2) {
+    // Measured: with 32 heads (one sequence) the separate kernels are as fast (57.3 against 57.6 us per
+    // step at 128K context) and much faster on short contexts, where this kernel's fixed costs show;
+    // with 128 heads (batch 4, 128K context) four waves take 171 us against 187 (246 / 269 and 398 / 428
+    // at budgets 1/8 and 1/4); with 256 heads of 2049 pages (batch 8, 32K context) the 16 selecting
+    // CTAs fall behind (179 against 155).  Left to itself the library takes this path for 64 to 128
+    // heads of at least 4096 pages, trying four waves first.
+    if (forced_waves <= 0 && (BH < 64 || BH > 128 || P < 4096)) return 0;
+    static const int order[3] = {4, 8, 2};
+    for (int i = 0; i < 3; ++i) {
+        const int waves = order[i];
         if (forced_waves > 0 && waves != forced_waves) continue;
         if (BH % waves) continue;
         const int HW = BH / waves;
@@ -1004,7 +1018,15 @@ cudaError_t launch_sort_list(const int2 *sel, int sel_stride, int K, int P, int 
                              cudaStream_t s)
 {
     if (P > 32768) return cudaErrorInvalidValue;
-    sort_list_kernel<<<(unsigned)BH, 1024, 0, s>>>(sel, sel_stride, K, P, out, out_stride);
+    sort_list_kernel<int2><<<(unsigned)BH, 1024, 0, s>>>(sel, sel_stride, K, P, out, out_stride);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sort_list32(const int32_t *sel, int sel_stride, int K, int P, int BH, int32_t *out, int out_stride,
+                               cudaStream_t s)
+{
+    if (P > 32768) return cudaErrorInvalidValue;
+    sort_list_kernel<int32_t><<<(unsigned)BH, 1024, 0, s>>>(sel, sel_stride, K, P, out, out_stride);
     return cudaGetLastError();
 }
 

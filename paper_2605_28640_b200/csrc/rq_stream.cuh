@@ -312,11 +312,10 @@ __device__ __forceinline__ void combine_head(const float *src, int n, T *o_row, 
 // One step of Eq. 1 for head h (thread d < D owns channel d): new state, cache row, bounds of
 // the newest page, and that page's score (returned to thread 0).  `len` is the length AFTER the
 // append.  red: 16 floats of shared memory.  The head's largest |stored key| is brought up to date
-// in the copy that the NEXT step reads; with write_current also in the copy of this step (only
-// when nobody reads that copy while this runs).
+// in the copy that the NEXT step reads (the copy of this step is being read by the scoring warps).
 template <typename T, int D>
 __device__ __forceinline__ float update_head(const DecodeArgs &a, int h, const T *q, const T *k_t, const T *v_t,
-                                             const void *g_t, float *scores, float *red, bool write_current = true)
+                                             const void *g_t, float *scores, float *red)
 {
     const int d = threadIdx.x;
     const int S = a.S;
@@ -372,7 +371,6 @@ __device__ __forceinline__ float update_head(const DecodeArgs &a, int h, const T
             const int BH = a.B * a.H, cur = a.epoch & 1;
             const float nv = fmaxf(a.absmax[cur * BH + h], m);
             a.absmax[(cur ^ 1) * BH + h] = nv;
-            if (write_current) a.absmax[cur * BH + h] = nv;
         }
     }
     __syncthreads();

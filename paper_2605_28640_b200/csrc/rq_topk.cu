@@ -335,21 +335,207 @@ __device__ __forceinline__ void select_rows(SelectScratch &sh, uint32_t *skey, c
     for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
 }
 
+// ---------------------------------------------------------------- selection from the scoring kernel's histogram
+// When the scoring kernel has already counted every competing page into 2048 value buckets of an
+// a-priori range (|U_p| <= A sum_i |q_i| with A the head's largest |stored key|), the selection
+// needs no pass for the range, no keys and no histogram of its own: the head's histogram and
+// scores come into shared memory with two bulk copies (one round trip), the bucket b that holds
+// the k_rem-th largest score and the rank k_in wanted inside it follow from suffix sums over the
+// threads, pages of higher buckets go straight to the list, the pages of bucket b are ranked
+// against each other by (score, lower page first) and the best k_in appended.  The list is in no
+// particular order (the flash-decode kernel does not care; a caller that wants it gets it sorted by
+// a kernel of its own).  Returns false, with nothing but forced pages written, when that cannot be
+// done (bucket too full, counts that do not add up, copy that never came): select_rows then does
+// the work.  Clears the histogram for the next step.
+constexpr int kFastCandMax = 1024;
+
+struct FastShared {                                  // dynamic shared memory of the selection kernel (register-key variants)
+    alignas(16) uint32_t hist[kStepBins];
+    uint32_t ckey[kFastCandMax];
+    int32_t cpage[kFastCandMax];
+    alignas(16) float sc[kTopkFastPages + 8];        // the head's scores from the 16-byte boundary below their start
+};
+
+__device__ __forceinline__ bool fast_select(FastShared &fs, SelectScratch &sh, uint64_t *bar, const float *sc, int P, int K,
+                                            int ns, int nl, int32_t *out, int budget, uint32_t *ghist, float2 range,
+                                            const char *kvh, int page_bytes, int n_prefetch)
+{
+    constexpr int NTH = kTopkThreads;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int k_rem = K - ns - nl;
+    const int p_lo = ns, p_hi = P - nl, n_forced = ns + nl;
+    const int mis = (int)((reinterpret_cast<uintptr_t>(sc) >> 2) & 3);
+    const float *src = sc - mis;
+    const int nfl = (mis + P + 3) & ~3;
+    if (tid == 0) {
+        // (what the copies read was written by the kernel before this one: no fence between proxies is needed)
+        mbar_arrive_expect_tx(bar, kStepBins * 4 + nfl * 4);
+        bulk_g2s(fs.hist, ghist, kStepBins * 4, bar);
+        bulk_g2s(fs.sc, src, nfl * 4, bar);
+        sh.digit = 0xffffffffu; sh.krem = 0; sh.cnt = 0; sh.ncand = 0; sh.tau = 0;   // bucket, rank inside, its population; candidates; pages above
+    }
+    for (int p = tid; p < ns; p += NTH) out[p] = p;
+    for (int i = tid; i < nl; i += NTH) out[ns + i] = P - nl + i;
+    for (int p = K + tid; p < budget; p += NTH) out[p] = -1;
+    const bool landed = mbar_wait(bar, 0);
+    reinterpret_cast<uint2 *>(ghist)[tid] = make_uint2(0u, 0u);      // all zero again for the next step (the copy has read it)
+    if (!__syncthreads_and(landed)) return false;
+    if (k_rem <= 0) return true;
+
+    // thread t owns bins 2t and 2t+1
+    const uint2 h2 = reinterpret_cast<const uint2 *>(fs.hist)[tid];
+    const int c0 = (int)h2.x, c1 = (int)h2.y;
+    int suf = c0 + c1;                               // inclusive suffix sum over the lanes
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_down_sync(FULL, suf, off);
+        if (lane + off < 32) suf += t;
+    }
+    if (lane == 0) sh.red[warp] = (uint32_t)suf;
+    __syncthreads();
+    const int wtot = (int)sh.red[lane];              // every warp scans the 32 warp totals on its own
+    int wsuf = wtot;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t = __shfl_down_sync(FULL, wsuf, off);
+        if (lane + off < 32) wsuf += t;
+    }
+    const int total = __shfl_sync(FULL, wsuf, 0);
+    const int above = __shfl_sync(FULL, wsuf - wtot, warp);   // keys in higher warps' bins
+    const int incl1 = above + suf - c0;              // keys in bins >= 2t+1
+    const int excl1 = incl1 - c1;
+    const int incl0 = incl1 + c0;
+    if (total == p_hi - p_lo && k_rem <= total) {
+        if (incl1 >= k_rem && excl1 < k_rem) { sh.digit = 2u * tid + 1u; sh.krem = (uint32_t)(k_rem - excl1); sh.cnt = (uint32_t)c1; }
+        if (incl0 >= k_rem && incl1 < k_rem) { sh.digit = 2u * tid; sh.krem = (uint32_t)(k_rem - incl1); sh.cnt = (uint32_t)c0; }
+    }
+    __syncthreads();
+    const int b = (int)sh.digit, k_in = (int)sh.krem, cnt_b = (int)sh.cnt;
+    if (b < 0 || cnt_b > kFastCandMax) return false;
+
+    // classify: thread t takes the 16-byte vectors t, t + 1024, ... (at most three)
+    ScoreRange rg;
+    rg.lo = range.x;
+    rg.scale = range.y;
+    constexpr int VMAX = (kTopkFastPages / 4 + 2 + NTH - 1) / NTH;
+    uint32_t m_sure = 0, m_cand = 0;                 // bit 4 u + e
+#pragma unroll
+    for (int u = 0; u < VMAX; ++u) {
+        const int fi = (u * NTH + tid) * 4;
+        if (fi < nfl) {
+            const float4 xv = *reinterpret_cast<const float4 *>(fs.sc + fi);
+            const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int p = fi - mis + e;
+                const int bk = rg.bucket(xs[e]);
+                const bool in = p >= p_lo && p < p_hi;
+                m_sure |= (uint32_t)(in && bk > b) << (4 * u + e);
+                m_cand |= (uint32_t)(in && bk == b) << (4 * u + e);
+            }
+        }
+    }
+    // positions: scan inside the warp, then over the warp totals (32 warps on one shared-memory
+    // atomic each would wait for one another)
+    int ws = __popc(m_sure), wc = __popc(m_cand);
+    int ps = ws, pc = wc;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int t1 = __shfl_up_sync(FULL, ps, off), t2 = __shfl_up_sync(FULL, pc, off);
+        if (lane >= off) { ps += t1; pc += t2; }
+    }
+    const int wsum = __shfl_sync(FULL, ps, 31), wcsum = __shfl_sync(FULL, pc, 31);
+    ps -= ws;
+    pc -= wc;
+    if (lane == 0) { sh.red[warp] = (uint32_t)wsum; sh.red2[warp] = (uint32_t)wcsum; }
+    __syncthreads();                                 // (the reads of red for the bucket are long done)
+    {
+        int a1 = (int)sh.red[lane], a2 = (int)sh.red2[lane];     // inclusive scans over the warps
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t1 = __shfl_up_sync(FULL, a1, off), t2 = __shfl_up_sync(FULL, a2, off);
+            if (lane >= off) { a1 += t1; a2 += t2; }
+        }
+        ps += n_forced + __shfl_sync(FULL, a1, warp) - wsum;
+        pc += __shfl_sync(FULL, a2, warp) - wcsum;
+        const int all_s = __shfl_sync(FULL, a1, 31), all_c = __shfl_sync(FULL, a2, 31);
+        if (tid == 0) { sh.tau = (uint32_t)all_s; sh.ncand = (uint32_t)all_c; }
+    }
+    while (m_sure) {
+        const int i = __ffs(m_sure) - 1;
+        m_sure &= m_sure - 1;
+        const int p = ((i >> 2) * NTH + tid) * 4 - mis + (i & 3);
+        if (ps < K) {
+            out[ps] = p;
+            if (ps < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
+        }
+        ++ps;
+    }
+    while (m_cand) {
+        const int i = __ffs(m_cand) - 1;
+        m_cand &= m_cand - 1;
+        const int fi = ((i >> 2) * NTH + tid) * 4 + (i & 3);
+        if (pc < kFastCandMax) { fs.ckey[pc] = order_key(fs.sc[fi]); fs.cpage[pc] = fi - mis; }
+        ++pc;
+    }
+    __syncthreads();
+    const int n_sure = (int)sh.tau, nc = (int)sh.ncand;
+    if (n_sure != k_rem - k_in || nc != cnt_b) return false;         // scores and histogram disagree
+    // rank of a candidate: how many candidates beat it (higher score, or equal score and lower page)
+    // (a warp per candidate, the lanes share the comparisons)
+    for (int j = warp; j < nc; j += NTH / 32) {
+        const uint32_t kj = fs.ckey[j];
+        const int pj = fs.cpage[j];
+        int r = 0;
+        for (int i = lane; i < nc; i += 32) {
+            const uint32_t ki = fs.ckey[i];
+            r += (ki > kj) || (ki == kj && fs.cpage[i] < pj);
+        }
+        r = __reduce_add_sync(FULL, r);
+        if (lane == 0 && r < k_in) {
+            const int pos = n_forced + n_sure + r;
+            out[pos] = pj;
+            if (pos < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)pj * page_bytes, (uint32_t)page_bytes);
+        }
+    }
+    return true;
+}
+
 // The selection kernel: one CTA per head.  SMEM_KEYS: the keys of a head (ROWS * 1024 words) live
 // in dynamic shared memory.  The histogram is cleared before the wait for the scoring kernel.
 template <int ROWS, bool SMEM_KEYS>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const float *scores, int64_t score_stride, int P, int K,
                                                             int n_sink, int n_local, int32_t *idx, int idx_stride,
                                                             int budget, int32_t *attend_ctr, const char *kv,
-                                                            int64_t kv_head_bytes, int page_bytes, int n_prefetch)
+                                                            int64_t kv_head_bytes, int page_bytes, int n_prefetch,
+                                                            uint32_t *ghist, const float2 *range)
 {
     extern __shared__ __align__(16) uint32_t skey[];
     __shared__ SelectScratch sh;
+    __shared__ __align__(8) uint64_t bar;
     const int bh = blockIdx.x;
+    if (!SMEM_KEYS && ghist && threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_init_fence();
+    }
     select_prepare(sh);
     grid_dependency_wait();          // the scores come from the kernel before; the one before that may still use the counters
     grid_launch_dependents();
     if (threadIdx.x < 4) attend_ctr[bh * kCtrStride + threadIdx.x] = 0;   // this head's ticket counters of the streaming kernels
+    if constexpr (!SMEM_KEYS) {
+        if (ghist && K < P) {
+            __syncthreads();                         // the barrier is initialised
+            FastShared &fs = *reinterpret_cast<FastShared *>(skey);
+            if (fast_select(fs, sh, &bar, scores + (int64_t)bh * score_stride, P, K, n_sink, n_local,
+                            idx + (int64_t)bh * idx_stride, budget, ghist + (int64_t)bh * kStepBins, range[bh],
+                            kv + (int64_t)bh * kv_head_bytes, page_bytes, n_prefetch))
+                return;
+            __syncthreads();
+            select_prepare(sh);                      // the scratch was used otherwise
+            __syncthreads();
+        }
+    }
     select_rows<ROWS, SMEM_KEYS>(sh, skey, scores + (int64_t)bh * score_stride, P, K, n_sink, n_local,
                                  idx + (int64_t)bh * idx_stride, budget, kv + (int64_t)bh * kv_head_bytes, page_bytes,
                                  n_prefetch);
@@ -366,7 +552,7 @@ __global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a
                                                                     const void *g_t, float *scores, int do_update, int K,
                                                                     int n_sink, int n_local, int32_t *idx, int idx_stride,
                                                                     int budget, int32_t *attend_ctr, int64_t kv_head_bytes,
-                                                                    int page_bytes, int n_prefetch)
+                                                                    int page_bytes, int n_prefetch, int32_t *ctr_other)
 {
     using G = ScoreGeom<T, D>;
     constexpr unsigned FULL = 0xffffffffu;
@@ -378,7 +564,11 @@ __global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a
     grid_dependency_wait();          // earlier kernels may still read what the update rewrites
     grid_launch_dependents();
     if (tid < 4) attend_ctr[bh * kCtrStride + tid] = 0;   // this head's ticket counters of the flash-decode kernel
-    if (do_update) update_head<T, D>(a, bh, q, k_t, v_t, g_t, scores, red);   // also scores the newest page
+    if (do_update) {
+        update_head<T, D>(a, bh, q, k_t, v_t, g_t, scores, red);   // also scores the newest page
+        // the one-launch step's counters of the next step (it may be the next to run on this cache)
+        if (ctr_other && tid < kStepCtrInts) ctr_other[bh * kStepCtrInts + tid] = 0;
+    }
 
     const int Ps = do_update ? P - 1 : P;            // pages whose records are read here
     float qs[G::VPL][G::CH];
@@ -424,8 +614,10 @@ __global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a
 
 }  // namespace
 
+bool topk_uses_hist(int64_t pages) { return pages <= kTopkFastPages; }
+
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
-                        int idx_stride, int32_t *attend_ctr, int prefetch, cudaStream_t s)
+                        int idx_stride, int32_t *attend_ctr, int prefetch, const ScoreHist &hs, cudaStream_t s)
 {
     const int P = (int)((a.len + a.S - 1) / a.S);
     const int K = budget < P ? budget : P;
@@ -436,6 +628,8 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     int nl = a.n_local < K - ns ? a.n_local : K - ns;
     if (nl > P - ns) nl = P - ns;
     if (P > kTopkThreads * kTopkMaxPerThread) return cudaErrorInvalidValue;
+    using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
+                            int, int, uint32_t *, const float2 *);
     // the keys of a large head live in dynamic shared memory: allow it once per device
     constexpr int kMidRows = 16, kBigRows = kTopkMaxPerThread;
     constexpr int kMidSmem = kMidRows * kTopkThreads * (int)sizeof(uint32_t);
@@ -446,6 +640,12 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
+        const Kernel regs[5] = {topk_kernel<2, false>, topk_kernel<4, false>, topk_kernel<6, false>, topk_kernel<8, false>,
+                                topk_kernel<10, false>};
+        for (int i = 0; i < 5; ++i) {
+            e = cudaFuncSetAttribute(regs[i], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FastShared));
+            if (e != cudaSuccess) return e;
+        }
         e = cudaFuncSetAttribute(topk_kernel<kMidRows, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMidSmem);
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(topk_kernel<kBigRows, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBigSmem);
@@ -472,14 +672,13 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
     int n_prefetch = prefetch ? (int)(kTopkPrefetchBytes / BH / page_bytes) : 0;
     if (n_prefetch > K / 8) n_prefetch = K / 8;      // the head of the list only: the kernel waits for its prefetches
     const int rows = (P + kTopkThreads - 1) / kTopkThreads;
-    using Kernel = void (*)(const float *, int64_t, int, int, int, int, int32_t *, int, int, int32_t *, const char *, int64_t,
-                            int, int);
+    uint32_t *ghist = hs.hist && topk_uses_hist(P) ? hs.hist : nullptr;
     Kernel kern;
     if (rows <= 10) {                                // the keys of a head fit in registers (more rows would spill)
         static const Kernel by_rows[5] = {topk_kernel<2, false>, topk_kernel<4, false>, topk_kernel<6, false>,
                                           topk_kernel<8, false>, topk_kernel<10, false>};
         kern = by_rows[(rows - 1) / 2];
-        cfg.dynamicSmemBytes = 0;
+        cfg.dynamicSmemBytes = ghist ? sizeof(FastShared) : 0;
     } else if (rows <= kMidRows) {
         kern = topk_kernel<kMidRows, true>;
         cfg.dynamicSmemBytes = kMidSmem;
@@ -488,12 +687,12 @@ cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, in
         cfg.dynamicSmemBytes = kBigSmem;
     }
     return cudaLaunchKernelEx(&cfg, kern, scores, stride, P, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv,
-                              kv_head_bytes, page_bytes, n_prefetch);
+                              kv_head_bytes, page_bytes, n_prefetch, ghist, hs.range);
 }
 
 cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *k_t, const void *v_t, const void *g_t,
                                 float *scores, int do_update, int budget, int32_t *idx, int idx_stride,
-                                int32_t *attend_ctr, int prefetch, cudaStream_t s)
+                                int32_t *attend_ctr, int prefetch, int32_t *ctr_other, cudaStream_t s)
 {
     const int P = (int)((a.len + a.S - 1) / a.S);
     const int K = budget < P ? budget : P;
@@ -523,7 +722,7 @@ cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *
 #define RQ_LAUNCH_SMALL(T, D)                                                                                          \
     return cudaLaunchKernelEx(&cfg, score_select_kernel<T, D, ROWS>, a, (const T *)q, (const T *)k_t, (const T *)v_t,  \
                               g_t, scores, do_update, K, ns, nl, idx, idx_stride, budget, attend_ctr, kv_head_bytes,   \
-                              page_bytes, n_prefetch)
+                              page_bytes, n_prefetch, ctr_other)
     if (a.dtype == RQ_BF16) {
         if (a.D == 128) RQ_LAUNCH_SMALL(bf16, 128);
         if (a.D == 64) RQ_LAUNCH_SMALL(bf16, 64);
