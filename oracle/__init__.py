@@ -25,9 +25,10 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile ``rqo.c`` into ``librqo.so`` next to it (gcc, -O2, strict IEEE)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    srcs = [_SRC, os.path.join(_HERE, "rqo_snapkv.c")]
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in srcs):
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
-               "-fno-fast-math", "-o", _LIB, _SRC, "-lm"]
+               "-fno-fast-math", "-o", _LIB, *srcs, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -82,6 +83,12 @@ def lib():
         L.rqo_head_export.restype = None
         L.rqo_head_load.argtypes = [C.c_void_p, C.c_int64, _dp, _dp, _dp, _dp]
         L.rqo_head_load.restype = C.c_int
+        L.rqo_snapkv_importance.argtypes = [C.c_int64, C.c_int, C.c_int, _dp, C.c_double, _dp, _dp]
+        L.rqo_snapkv_importance.restype = None
+        L.rqo_snapkv_select.argtypes = [C.c_int64, C.c_int, _dp, C.c_int64, _ip, C.POINTER(C.c_int)]
+        L.rqo_snapkv_select.restype = C.c_int64
+        L.rqo_token_attention.argtypes = [C.c_int64, _ip, C.c_int, _dp, C.c_double, _dp, _dp, _dp]
+        L.rqo_token_attention.restype = None
         _lib = L
     return _lib
 
@@ -148,6 +155,35 @@ def sparse_attention(q, scale, kst, vst, idx, S):
 
 
 # ---------------------------------------------------------------- head object
+def snapkv_importance(qw, scale, kst):
+    """App. A.1 (SnapKV): importance of every position under the window's queries.  qw [W, D], kst [T, D]."""
+    qw, kst = _f64(qw), _f64(kst)
+    W, D = qw.shape
+    T = kst.shape[0]
+    imp = np.empty(T, np.float64)
+    lib().rqo_snapkv_importance(T, W, D, _d(qw), float(scale), _d(kst), _d(imp))
+    return imp
+
+
+def snapkv_select(imp, W, keep):
+    """Retained positions (ascending) and the near-tie flag."""
+    imp = _f64(imp)
+    T = imp.shape[0]
+    idx = np.empty(max(min(keep, T), 1), np.int64)
+    near = C.c_int(0)
+    n = lib().rqo_snapkv_select(T, W, _d(imp), keep, idx.ctypes.data_as(_ip), C.byref(near))
+    return idx[:n].copy(), bool(near.value)
+
+
+def token_attention(q, scale, kst, vst, tok):
+    """Eq. 4 over an explicit token list."""
+    q, kst, vst = _f64(q), _f64(kst), _f64(vst)
+    tok = np.ascontiguousarray(tok, dtype=np.int64)
+    y = np.empty(q.shape[0], np.float64)
+    lib().rqo_token_attention(len(tok), tok.ctypes.data_as(_ip), q.shape[0], _d(q), float(scale), _d(kst), _d(vst), _d(y))
+    return y
+
+
 class Head:
     """fp64 cache of one (batch, head) pair: prefill = append(T tokens),
     decode step = append(1 token) then query."""
