@@ -242,6 +242,35 @@ RQ_API int rq_attend_pages_noalloc(const rq_config *cfg, const void *kv, int64_t
                                    const int32_t *idx, int32_t n_idx, float scale, void *o,
                                    void *stream);
 
+/* SnapKV-style reduction of the cache [App. A.1, "Sparse inference settings", SnapKV paragraph;
+ * Sec. 2.2, Table 1]: after the prompt, the queries of its last `window` positions (the
+ * observation window, at most 64; the paper uses 64) rate every position by the attention they pay
+ * to it, importance[j] = sum_i softmax_j(scale * q_i . k~_j) with query i (at position len - window
+ * + i) seeing the positions up to its own; the `keep` most important entries are retained: the
+ * window's own positions always (they count inside keep), then the most important earlier
+ * positions, equal importance to the lower position.
+ *   q_window       : [B][window][H][D] of cfg.dtype (device)
+ *   idx_out        : int32 [B][H][keep] (device): retained positions, ascending; -1 beyond len
+ *   importance_out : NULL or fp32 [B][H][len] (device)
+ *   scratch        : device memory of rq_snapkv_scratch_bytes() bytes for the cache's current
+ *                    length, 256-byte aligned, free again when the call's work has run
+ *   scale          : softmax scale; <= 0 selects 1/sqrt(D)
+ * Errors: INVALID_ARG (NULL, window outside 1..64 or longer than the cache, keep < 1), CUDA. */
+RQ_API int rq_snapkv_scratch_bytes(const rq_cache *cache, size_t *bytes);
+RQ_API int rq_snapkv_select(rq_cache *cache, const void *q_window, int32_t window, int32_t keep, float scale,
+                            int32_t *idx_out, float *importance_out, void *scratch, void *stream);
+
+/* The second half of the reduction [same passage: only the selected entries stay in the cache and
+ * later attention runs over them alone]: copies the `keep` positions idx[b][h][0..keep)
+ * (ascending, all < len) of every head of `src` into `dst`, an initialised cache of the same shape
+ * and types with capacity_tokens >= keep (plus the tokens to be decoded), as its positions
+ * 0..keep-1; rebuilds the page bounds of dst from the copied keys and carries the recurrence state
+ * over, so that rq_decode_step on dst continues Eq. 1 and attends over the retained entries and
+ * the tokens appended since (with budget_pages >= its pages: over all of them).  Whatever dst held
+ * is dropped.
+ * Errors: INVALID_ARG (shapes differ, dst is src, keep outside 1..len), CAPACITY, CUDA. */
+RQ_API int rq_snapkv_compact(const rq_cache *src, const int32_t *idx, int32_t keep, rq_cache *dst, void *stream);
+
 /* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
 RQ_API int64_t rq_cache_len(const rq_cache *cache);
 

@@ -49,6 +49,9 @@ SIGNATURES = {
     "rq_attend_pages": (C.c_int, [_cachep, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_attend_pages_noalloc": (C.c_int, [_cfgp, _vp, _i64, _vp, _vp, _i32, _f, _vp, _vp]),
     "rq_probe_read": (C.c_int, [_vp, C.c_size_t, _vp, _vp]),
+    "rq_snapkv_scratch_bytes": (C.c_int, [_cachep, _szp]),
+    "rq_snapkv_select": (C.c_int, [_cachep, _vp, _i32, _i32, _f, _vp, _vp, _vp, _vp]),
+    "rq_snapkv_compact": (C.c_int, [_cachep, _vp, _i32, _cachep, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
     "rq_decode_step_launches": (C.c_int, [_cachep, _i32]),
     "rq_device_status": (C.c_int, [_cachep, C.POINTER(C.c_int32), _vp]),
@@ -168,6 +171,21 @@ def rq_attend_pages_noalloc(cfg: rq_config, kv, length, q, idx, n_idx, scale, o,
 def rq_probe_read(buf, nbytes, sink, stream=None):
     """One launch that reads nbytes of the device tensor `buf` once (benchmarking aid)."""
     _check(lib().rq_probe_read(_ptr(buf), nbytes, _ptr(sink), _stream(stream)), "rq_probe_read")
+
+
+def rq_snapkv_scratch_bytes(cache: rq_cache) -> int:
+    n = C.c_size_t()
+    _check(lib().rq_snapkv_scratch_bytes(C.byref(cache), C.byref(n)), "rq_snapkv_scratch_bytes")
+    return n.value
+
+
+def rq_snapkv_select(cache: rq_cache, q_window, window, keep, scale, idx_out, importance_out, scratch, stream=None):
+    _check(lib().rq_snapkv_select(C.byref(cache), _ptr(q_window), window, keep, scale, _ptr(idx_out),
+                                  _ptr(importance_out), _ptr(scratch), _stream(stream)), "rq_snapkv_select")
+
+
+def rq_snapkv_compact(src: rq_cache, idx, keep, dst: rq_cache, stream=None):
+    _check(lib().rq_snapkv_compact(C.byref(src), _ptr(idx), keep, C.byref(dst), _stream(stream)), "rq_snapkv_compact")
 
 
 def rq_cache_len(cache: rq_cache) -> int:

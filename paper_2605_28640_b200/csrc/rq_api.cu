@@ -554,6 +554,66 @@ int rq_probe_read(const void *buf, size_t bytes, void *sink, void *stream)
     return cudaGetLastError() == cudaSuccess ? RQ_OK : RQ_ERR_CUDA;
 }
 
+int rq_snapkv_scratch_bytes(const rq_cache *cache, size_t *bytes)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!bytes) return RQ_ERR_INVALID_ARG;
+    *bytes = snap_scratch_bytes(cache->cfg.batch * cache->cfg.heads, cache->len > 0 ? cache->len : 1);
+    return RQ_OK;
+}
+
+int rq_snapkv_select(rq_cache *cache, const void *q_window, int32_t window, int32_t keep, float scale,
+                     int32_t *idx_out, float *importance_out, void *scratch, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q_window || !idx_out || !scratch || !aligned(scratch, 256)) return RQ_ERR_INVALID_ARG;
+    if (window < 1 || window > 64 || keep < 1 || cache->len < window) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    cudaStream_t s = (cudaStream_t)stream;
+    SnapArgs a;
+    a.kv = cache->kv; a.page_cap = cache->page_capacity; a.len = cache->len;
+    a.B = c.batch; a.H = c.heads; a.D = c.head_dim; a.S = c.page_size; a.dtype = c.dtype;
+    a.qw = q_window; a.W = window;
+    a.scale = scale > 0.0f ? scale : 1.0f / sqrtf((float)c.head_dim);
+    const int BH = c.batch * c.heads;
+    snap_carve(scratch, BH, cache->len, &a.imp, &a.stats, &a.rowstat);
+    if (launch_snap_scores(a, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (launch_snap_select(a.imp, BH, cache->len, window, keep, idx_out, s) != cudaSuccess) return RQ_ERR_CUDA;
+    if (importance_out && cudaMemcpyAsync(importance_out, a.imp, (size_t)BH * cache->len * sizeof(float),
+                                          cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    return RQ_OK;
+}
+
+int rq_snapkv_compact(const rq_cache *src, const int32_t *idx, int32_t keep, rq_cache *dst, void *stream)
+{
+    int rc = check_cache(src);
+    if (rc != RQ_OK) return rc;
+    rc = check_cache(dst);
+    if (rc != RQ_OK) return rc;
+    if (!idx || keep < 1 || keep > src->len) return RQ_ERR_INVALID_ARG;
+    const rq_config &a = src->cfg, &b = dst->cfg;
+    if (a.batch != b.batch || a.heads != b.heads || a.head_dim != b.head_dim || a.page_size != b.page_size ||
+        a.dtype != b.dtype || a.gate_dtype != b.gate_dtype || dst->kv == src->kv)
+        return RQ_ERR_INVALID_ARG;
+    if (keep > b.capacity_tokens) return RQ_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    rc = rq_cache_reset(dst, stream);                    // empties dst, clears its bookkeeping
+    if (rc != RQ_OK) return rc;
+    const int BH = a.batch * a.heads;
+    if (launch_snap_compact(src->kv, src->page_capacity, dst->kv, dst->meta, dst->page_capacity, a.page_size, a.head_dim,
+                            a.dtype, idx, keep, absmax_of(dst), BH, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    // the recurrence goes on from where the prompt ended
+    if (cudaMemcpyAsync(dst->state, src->state, (size_t)BH * 2 * a.head_dim * sizeof(float), cudaMemcpyDeviceToDevice, s) !=
+        cudaSuccess)
+        return RQ_ERR_CUDA;
+    dst->len = keep;
+    return RQ_OK;
+}
+
 int64_t rq_cache_len(const rq_cache *cache) { return cache ? cache->len : -1; }
 
 int rq_decode_step_launches(const rq_cache *cache, int32_t budget_pages)

@@ -136,6 +136,25 @@ cudaError_t launch_sort_list32(const int32_t *sel, int sel_stride, int K, int P,
 cudaError_t launch_sort_list(const int2 *sel, int sel_stride, int K, int P, int BH, int32_t *out, int out_stride,
                              cudaStream_t s);
 
+// ---- SnapKV-style cache reduction (rq_snapkv.cu) ----
+struct SnapArgs {
+    const void *kv;     // the source cache
+    int64_t page_cap, len;
+    int B, H, D, S, dtype;
+    const void *qw;     // [B][W][H][D] queries of the observation window
+    int W;
+    float scale;
+    float *imp;         // [BH][len] importance of every position
+    float2 *stats;      // [BH][tiles][64] per-tile row statistics
+    float2 *rowstat;    // [BH][64] final row statistics
+};
+size_t snap_scratch_bytes(int BH, int64_t len);
+void snap_carve(void *scratch, int BH, int64_t len, float **imp, float2 **stats, float2 **rowstat);
+cudaError_t launch_snap_scores(const SnapArgs &a, cudaStream_t s);
+cudaError_t launch_snap_select(const float *imp, int BH, int64_t len, int window, int keep, int32_t *idx, cudaStream_t s);
+cudaError_t launch_snap_compact(const void *skv, int64_t s_page_cap, void *dkv, void *dmeta, int64_t d_page_cap, int S, int D,
+                                int dtype, const int32_t *idx, int keep, float *absmax, int BH, cudaStream_t s);
+
 // Grid of a streaming kernel for a number of work units spread evenly over `heads` heads: at
 // most what the device holds at once, at least two units per warp, and a whole number of CTAs per
 // head if that keeps at least 85 % of the CTAs (heads served by more CTAs than others would

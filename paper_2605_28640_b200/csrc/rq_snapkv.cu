@@ -1,0 +1,426 @@
+// SnapKV-style reduction of the cache of decayed keys and values (App. A.1, "Sparse inference
+// settings", SnapKV paragraph; Table 1, row SnapKV): the queries of the last W prompt positions
+// (the observation window) rate every earlier position by the attention they pay to it, the keep
+// most important entries are retained (the window itself always, inside keep) and copied into a
+// new, smaller cache on which decoding then runs.
+//
+//   importance[j] = sum_i softmax_j(scale * q_i . k~_j),  query i at position T - W + i sees j <= T - W + i
+//
+// Kernels (plain fp32 ALU work; the window is at most 64 queries, so the score pass is a thin
+// 64 x T x D contraction per head):
+//   snap_tile_kernel<PASS 1>  per (head, tile of 128 keys): the 64 x 128 block of scores in registers
+//                             (8 rows x 4 keys per thread, operands from shared memory), per row the
+//                             block's maximum and sum of exponentials -> partial statistics
+//   snap_rows_kernel          per (head, query): merges the partial statistics of all tiles
+//   snap_tile_kernel<PASS 2>  the same block of scores again, turned into weights with the final
+//                             statistics and summed over the queries -> importance of the tile's keys
+//   snap_select_kernel        per head: the keep - W most important positions before the window
+//                             (most-significant-digit radix select on the order-preserving image of the
+//                             importance, equal importance to the lower position) plus the window,
+//                             written in ascending order
+//   snap_compact_kernel       per (head, page of the new cache): gathers the retained rows, rebuilds
+//                             the page's min/max bounds, tracks the head's largest |key|
+// The keys are read twice (statistics, then weights): the 64 x T scores of a head are never stored.
+#include <math.h>
+#include <math_constants.h>
+
+#include "rq_async.cuh"
+#include "rq_device.cuh"
+#include "rq_internal.h"
+
+namespace rq {
+
+namespace {
+
+constexpr int kSnapRows = 64;                  // queries of the window (fewer: the rest is masked)
+constexpr int kSnapKeys = 128;                 // keys per tile
+constexpr int kSnapThreads = 256;              // 8 row groups x 32 key groups
+constexpr int kSnapBins = 2048;
+
+template <int D>
+struct SnapGeom {
+    static constexpr int LD = D + 4;           // floats per row in shared memory (16-byte aligned rows, few bank conflicts)
+    // queries | keys | row max | row 1/l | reduction scratch (8 x 128 floats)
+    static constexpr int SMEM_BYTES = (kSnapRows + kSnapKeys) * LD * 4 + 2 * kSnapRows * 4 + 8 * kSnapKeys * 4;
+};
+
+// PASS 1: stats[bh][tile][row] = (max, sum exp) of the tile's visible scores.
+// PASS 2: imp[bh][key] = sum_rows exp(s - m_row) / l_row  with rowstat[bh][row] = (m, l).
+template <typename T, int D, int PASS>
+__global__ void __launch_bounds__(kSnapThreads) snap_tile_kernel(const T *kv, int64_t page_cap, int S, int64_t len,
+                                                                 const T *qw, int W, int H, float scale_log2,
+                                                                 float2 *stats, const float2 *rowstat, float *imp,
+                                                                 int ntiles)
+{
+    using G = SnapGeom<D>;
+    constexpr int LD = G::LD;
+    extern __shared__ __align__(16) float sm[];
+    float *qs = sm;                              // [64][LD]
+    float *ks = qs + kSnapRows * LD;             // [128][LD]
+    float *rm = ks + kSnapKeys * LD;             // [64] final row maximum (pass 2)
+    float *rl = rm + kSnapRows;                  // [64] 1 / final row sum  (pass 2)
+    float *red = rl + kSnapRows;                 // [8][128] column sums of the row groups (pass 2)
+
+    const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+    const int tile = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int64_t j0 = (int64_t)tile * kSnapKeys;
+    const int64_t first_q = len - W;             // position of query 0
+
+    // the window's queries of this head, scaled: qw is [B][W][H][D]
+    for (int i = tid; i < kSnapRows * (D / 4); i += kSnapThreads) {
+        const int r = i / (D / 4), c4 = i % (D / 4);
+        float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (r < W) {
+            const T *src = qw + (((int64_t)b * W + r) * H + h) * D + c4 * 4;
+            v = make_float4(load1<T>(src) * scale_log2, load1<T>(src + 1) * scale_log2, load1<T>(src + 2) * scale_log2,
+                            load1<T>(src + 3) * scale_log2);
+        }
+        *reinterpret_cast<float4 *>(qs + r * LD + c4 * 4) = v;
+    }
+    // the tile's keys: position j lives in page j / S, slot j % S of the head's cache
+    for (int i = tid; i < kSnapKeys * (D / 4); i += kSnapThreads) {
+        const int r = i / (D / 4), c4 = i % (D / 4);
+        const int64_t j = j0 + r;
+        float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (j < len) {
+            const T *src = kv + ((((int64_t)bh * page_cap + j / S) * 2) * S + j % S) * D + c4 * 4;
+            v = make_float4(load1<T>(src), load1<T>(src + 1), load1<T>(src + 2), load1<T>(src + 3));
+        }
+        *reinterpret_cast<float4 *>(ks + r * LD + c4 * 4) = v;
+    }
+    if (PASS == 2 && tid < kSnapRows) {
+        const float2 f = tid < W ? rowstat[(int64_t)bh * kSnapRows + tid] : make_float2(0.0f, 1.0f);
+        rm[tid] = f.x;
+        rl[tid] = 1.0f / f.y;
+    }
+    __syncthreads();
+
+    // scores: rows ty * 8 .. + 7, keys tx * 4 .. + 3
+    float acc[8][4];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[r][c] = 0.0f;
+#pragma unroll 2
+    for (int d = 0; d < D; d += 4) {
+        float4 kq[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) kq[c] = *reinterpret_cast<const float4 *>(ks + (tx * 4 + c) * LD + d);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const float4 q4 = *reinterpret_cast<const float4 *>(qs + (ty * 8 + r) * LD + d);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                acc[r][c] = fmaf(q4.x, kq[c].x, acc[r][c]);
+                acc[r][c] = fmaf(q4.y, kq[c].y, acc[r][c]);
+                acc[r][c] = fmaf(q4.z, kq[c].z, acc[r][c]);
+                acc[r][c] = fmaf(q4.w, kq[c].w, acc[r][c]);
+            }
+        }
+    }
+    // query `row` sees key j iff row < W and j <= first_q + row (which is < len)
+    auto visible = [&](int row, int c) { return row < W && j0 + tx * 4 + c <= first_q + row; };
+
+    if (PASS == 1) {
+        // per row: maximum over the tile, then sum of exponentials (exp2 domain); the lanes of a warp share the rows
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int row = ty * 8 + r;
+            float m = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (visible(row, c)) m = fmaxf(m, acc[r][c]);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+            float l = 0.0f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (visible(row, c)) l += exp2f(acc[r][c] - m);
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+            if (tx == 0) stats[((int64_t)bh * ntiles + tile) * kSnapRows + row] = make_float2(m, l);
+        }
+    } else {
+        // weights, summed over this thread's 8 rows, then over the 8 row groups through shared memory
+        float col[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int row = ty * 8 + r;
+            const float m = rm[row], il = rl[row];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (visible(row, c)) col[c] = fmaf(exp2f(acc[r][c] - m), il, col[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) red[ty * kSnapKeys + tx * 4 + c] = col[c];
+        __syncthreads();
+        if (tid < kSnapKeys) {
+            float s = 0.0f;
+#pragma unroll
+            for (int g = 0; g < 8; ++g) s += red[g * kSnapKeys + tid];
+            if (j0 + tid < len) imp[(int64_t)bh * len + j0 + tid] = s;
+        }
+    }
+}
+
+// Final statistics of a row: merge of its tiles' (max, sum exp).  One warp per (head, row).
+__global__ void __launch_bounds__(128) snap_rows_kernel(const float2 *stats, float2 *rowstat, int ntiles, int n_rows_total)
+{
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (w >= n_rows_total) return;
+    const int bh = w / kSnapRows, row = w % kSnapRows;
+    float m = -CUDART_INF_F, l = 0.0f;
+    for (int t = lane; t < ntiles; t += 32) {
+        const float2 f = stats[((int64_t)bh * ntiles + t) * kSnapRows + row];
+        if (f.x > -CUDART_INF_F) {
+            const float mn = fmaxf(m, f.x);
+            l = l * exp2f(m - mn) + f.y * exp2f(f.x - mn);     // exp2f(-inf) = 0 on the first merge
+            m = mn;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float mo = __shfl_xor_sync(0xffffffffu, m, off), lo = __shfl_xor_sync(0xffffffffu, l, off);
+        const float mn = fmaxf(m, mo);
+        const float fa = m > -CUDART_INF_F ? exp2f(m - mn) : 0.0f, fb = mo > -CUDART_INF_F ? exp2f(mo - mn) : 0.0f;
+        l = l * fa + lo * fb;
+        m = mn;
+    }
+    if (lane == 0) rowstat[w] = make_float2(m, l > 0.0f ? l : 1.0f);
+}
+
+// ---------------------------------------------------------------- token-level selection
+// One CTA of 1024 threads per head.  Candidates: positions 0 .. C-1 (C = len - w, w = window
+// positions kept outright); `want` of them are taken: those with the largest importance, equal
+// importance to the lower position.  Radix select over the order-preserving keys, 11 bits per pass,
+// reading the importances from global memory (L2) each pass; then every warp walks its own
+// contiguous range twice (count, write), so the list comes out ascending.
+__global__ void __launch_bounds__(1024) snap_select_kernel(const float *imp, int64_t len, int w, int keep, int32_t *idx)
+{
+    constexpr unsigned FULL = 0xffffffffu;
+    __shared__ uint32_t hist[kSnapBins];
+    __shared__ uint32_t red[32], red2[32];
+    __shared__ uint32_t s_digit, s_krem, s_cnt;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.x;
+    const float *x = imp + (int64_t)bh * len;
+    int32_t *out = idx + (int64_t)bh * keep;
+    const int C = (int)(len - w);
+    const int want = keep - w;
+    if (want >= C) {                                 // everything is kept
+        for (int j = tid; j < keep; j += 1024) out[j] = j < len ? j : -1;
+        return;
+    }
+    uint32_t tau = 0xffffffffu;                      // want == 0: nothing but the window
+    int r_eq = 0;
+    if (want > 0) {
+        uint32_t prefix = 0u;
+        int k = want;
+        bool whole = false;
+#pragma unroll 1
+        for (int hi = 31; hi >= 0 && !whole; hi -= 11) {
+            const int lo = hi >= 10 ? hi - 10 : 0;   // this pass decides bits hi .. lo
+            const uint32_t dmask = (1u << (hi - lo + 1)) - 1u;
+            const uint32_t himask = hi == 31 ? 0u : ~0u << (hi + 1);
+            for (int i = tid; i < kSnapBins; i += 1024) hist[i] = 0u;
+            __syncthreads();
+            for (int j = tid; j < C; j += 1024) {
+                const uint32_t kx = order_key(__ldcg(x + j));
+                if ((kx & himask) == (prefix & himask)) atomicAdd(&hist[(kx >> lo) & dmask], 1u);
+            }
+            __syncthreads();
+            // walk the bins from the top until k keys are covered: thread t owns bins 2t, 2t+1
+            const uint32_t c0 = hist[2 * tid], c1 = hist[2 * tid + 1];
+            uint32_t suf = c0 + c1;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t t = __shfl_down_sync(FULL, suf, off);
+                if (lane + off < 32) suf += t;
+            }
+            if (lane == 0) red[warp] = suf;
+            __syncthreads();
+            const uint32_t wtot = red[lane];
+            uint32_t wsuf = wtot;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t t = __shfl_down_sync(FULL, wsuf, off);
+                if (lane + off < 32) wsuf += t;
+            }
+            const uint32_t above = __shfl_sync(FULL, wsuf - wtot, warp);
+            const uint32_t incl1 = above + suf - c0, excl1 = incl1 - c1, incl0 = incl1 + c0, kr = (uint32_t)k;
+            if (incl1 >= kr && excl1 < kr) { s_digit = 2u * tid + 1u; s_krem = kr - excl1; s_cnt = c1; }
+            if (incl0 >= kr && incl1 < kr) { s_digit = 2u * tid; s_krem = kr - incl1; s_cnt = c0; }
+            __syncthreads();
+            prefix |= s_digit << lo;
+            k = (int)s_krem;
+            whole = s_cnt == s_krem;                 // the whole bin is wanted: its lowest possible key is a threshold
+            __syncthreads();
+        }
+        tau = prefix;
+        r_eq = whole ? 0x7fffffff : k;               // keys equal to tau that are taken, lowest positions first
+    }
+    // every warp owns a contiguous range of the candidates: count, scan over the warps, write
+    const int per = (C + 31) / 32, lo_j = warp * per, hi_j = min(C, lo_j + per);
+    uint32_t wgt = 0, weq = 0;
+    for (int j0 = lo_j; j0 < hi_j; j0 += 32) {
+        const int j = j0 + lane;
+        const bool in = j < hi_j;
+        const uint32_t kx = in ? order_key(__ldcg(x + j)) : 0u;
+        wgt += __popc(__ballot_sync(FULL, in && kx > tau));
+        weq += __popc(__ballot_sync(FULL, in && kx == tau));
+    }
+    if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
+    __syncthreads();
+    uint32_t g_inc = red[lane], e_inc = red2[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t tg = __shfl_up_sync(FULL, g_inc, off), te = __shfl_up_sync(FULL, e_inc, off);
+        if (lane >= off) { g_inc += tg; e_inc += te; }
+    }
+    int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt), eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int j0 = lo_j; j0 < hi_j; j0 += 32) {
+        const int j = j0 + lane;
+        const bool in = j < hi_j;
+        const uint32_t kx = in ? order_key(__ldcg(x + j)) : 0u;
+        const bool is_gt = in && kx > tau, is_eq = in && kx == tau;
+        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
+        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
+        const int rank = is_gt ? gb + min(eb, r_eq) : (is_eq && eb < r_eq) ? gb + eb : -1;
+        if (rank >= 0 && rank < want) out[rank] = j;
+        gt_run += __popc(bg);
+        eq_run += __popc(be);
+    }
+    for (int i = tid; i < w; i += 1024) out[want + i] = C + i;       // the window, above every candidate
+}
+
+// ---------------------------------------------------------------- compaction into the new cache
+// One CTA per (head, page of the new cache), a thread per channel.
+template <typename T>
+__global__ void snap_compact_kernel(const T *skv, int64_t s_page_cap, T *dkv, T *dmeta, int64_t d_page_cap, int S, int D,
+                                    const int32_t *idx, int keep, float *absmax, int BH)
+{
+    const int bh = blockIdx.y, page = blockIdx.x, d = threadIdx.x;
+    const int32_t *list = idx + (int64_t)bh * keep;
+    T *dpage = dkv + (((int64_t)bh * d_page_cap + page) * 2) * S * D;
+    float mn = CUDART_INF_F, mx = -CUDART_INF_F;
+    for (int s = 0; s < S; ++s) {
+        const int r = page * S + s;
+        T kq, vq;
+        if (r < keep) {
+            const int64_t pos = list[r];
+            const T *src = skv + ((((int64_t)bh * s_page_cap + pos / S) * 2) * S + pos % S) * D + d;
+            kq = src[0];
+            vq = src[(int64_t)S * D];
+            const float kf = load1<T>(&kq);
+            mn = fminf(mn, kf);
+            mx = fmaxf(mx, kf);
+        } else {
+            store1<T>(&kq, 0.0f);                    // unused slots of the last page are defined
+            store1<T>(&vq, 0.0f);
+        }
+        dpage[(int64_t)s * D + d] = kq;
+        dpage[(int64_t)(S + s) * D + d] = vq;
+    }
+    T *m = dmeta + (((int64_t)bh * d_page_cap + page) * 2) * D;
+    store1<T>(m + d, mn);
+    store1<T>(m + D + d, mx);
+    if (absmax) {
+        float am = fmaxf(-mn, mx);                   // the page holds at least one retained row
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, off));
+        if ((d & 31) == 0) {
+            atomicMax(reinterpret_cast<unsigned *>(absmax) + bh, __float_as_uint(am));
+            atomicMax(reinterpret_cast<unsigned *>(absmax) + BH + bh, __float_as_uint(am));
+        }
+    }
+}
+
+template <typename T, int D>
+cudaError_t snap_scores_t(const SnapArgs &a, cudaStream_t s)
+{
+    using G = SnapGeom<D>;
+    static bool ready[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!ready[dev]) {
+        e = cudaFuncSetAttribute(snap_tile_kernel<T, D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(snap_tile_kernel<T, D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        ready[dev] = true;
+    }
+    const int BH = a.B * a.H;
+    const int ntiles = (int)((a.len + kSnapKeys - 1) / kSnapKeys);
+    const dim3 grid((unsigned)ntiles, (unsigned)BH);
+    const float sl2 = a.scale * 1.4426950408889634f;
+    snap_tile_kernel<T, D, 1><<<grid, kSnapThreads, G::SMEM_BYTES, s>>>((const T *)a.kv, a.page_cap, a.S, a.len, (const T *)a.qw,
+                                                                      a.W, a.H, sl2, a.stats, nullptr, nullptr, ntiles);
+    const int rows = BH * kSnapRows;
+    snap_rows_kernel<<<(rows * 32 + 127) / 128, 128, 0, s>>>(a.stats, a.rowstat, ntiles, rows);
+    snap_tile_kernel<T, D, 2><<<grid, kSnapThreads, G::SMEM_BYTES, s>>>((const T *)a.kv, a.page_cap, a.S, a.len, (const T *)a.qw,
+                                                                      a.W, a.H, sl2, nullptr, a.rowstat, a.imp, ntiles);
+    return cudaGetLastError();
+}
+
+size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+
+size_t snap_scratch_bytes(int BH, int64_t len)
+{
+    const size_t ntiles = (size_t)((len + kSnapKeys - 1) / kSnapKeys);
+    return round256((size_t)BH * len * sizeof(float))                         // importance
+           + round256((size_t)BH * ntiles * kSnapRows * sizeof(float2))       // per-tile statistics
+           + round256((size_t)BH * kSnapRows * sizeof(float2));               // final statistics
+}
+
+void snap_carve(void *scratch, int BH, int64_t len, float **imp, float2 **stats, float2 **rowstat)
+{
+    const size_t ntiles = (size_t)((len + kSnapKeys - 1) / kSnapKeys);
+    char *p = (char *)scratch;
+    *imp = (float *)p;
+    p += round256((size_t)BH * len * sizeof(float));
+    *stats = (float2 *)p;
+    p += round256((size_t)BH * ntiles * kSnapRows * sizeof(float2));
+    *rowstat = (float2 *)p;
+}
+
+cudaError_t launch_snap_scores(const SnapArgs &a, cudaStream_t s)
+{
+    if (a.W < 1 || a.W > kSnapRows || a.len < a.W) return cudaErrorInvalidValue;
+    if (a.B * a.H > 65535) return cudaErrorInvalidValue;
+    if (a.dtype == RQ_BF16) {
+        if (a.D == 128) return snap_scores_t<bf16, 128>(a, s);
+        if (a.D == 64) return snap_scores_t<bf16, 64>(a, s);
+    } else {
+        if (a.D == 128) return snap_scores_t<float, 128>(a, s);
+        if (a.D == 64) return snap_scores_t<float, 64>(a, s);
+    }
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_snap_select(const float *imp, int BH, int64_t len, int window, int keep, int32_t *idx, cudaStream_t s)
+{
+    int w = window < keep ? window : keep;
+    if ((int64_t)w > len) w = (int)len;
+    snap_select_kernel<<<(unsigned)BH, 1024, 0, s>>>(imp, len, w, keep, idx);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_snap_compact(const void *skv, int64_t s_page_cap, void *dkv, void *dmeta, int64_t d_page_cap, int S, int D,
+                                int dtype, const int32_t *idx, int keep, float *absmax, int BH, cudaStream_t s)
+{
+    const dim3 grid((unsigned)((keep + S - 1) / S), (unsigned)BH);
+    if (dtype == RQ_BF16)
+        snap_compact_kernel<bf16><<<grid, D, 0, s>>>((const bf16 *)skv, s_page_cap, (bf16 *)dkv, (bf16 *)dmeta, d_page_cap, S, D, idx,
+                                                     keep, absmax, BH);
+    else
+        snap_compact_kernel<float><<<grid, D, 0, s>>>((const float *)skv, s_page_cap, (float *)dkv, (float *)dmeta, d_page_cap, S, D,
+                                                      idx, keep, absmax, BH);
+    return cudaGetLastError();
+}
+
+}  // namespace rq

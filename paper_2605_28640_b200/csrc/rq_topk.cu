@@ -466,10 +466,7 @@ __device__ __forceinline__ bool fast_select(FastShared &fs, SelectScratch &sh, u
         const int i = __ffs(m_sure) - 1;
         m_sure &= m_sure - 1;
         const int p = ((i >> 2) * NTH + tid) * 4 - mis + (i & 3);
-        if (ps < K) {
-            out[ps] = p;
-            if (ps < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
-        }
+        if (ps < K) out[ps] = p;
         ++ps;
     }
     while (m_cand) {
@@ -493,11 +490,15 @@ __device__ __forceinline__ bool fast_select(FastShared &fs, SelectScratch &sh, u
             r += (ki > kj) || (ki == kj && fs.cpage[i] < pj);
         }
         r = __reduce_add_sync(FULL, r);
-        if (lane == 0 && r < k_in) {
-            const int pos = n_forced + n_sure + r;
-            out[pos] = pj;
-            if (pos < n_prefetch) bulk_prefetch_l2(kvh + (int64_t)pj * page_bytes, (uint32_t)page_bytes);
-        }
+        if (lane == 0 && r < k_in) out[n_forced + n_sure + r] = pj;
+    }
+    // the pages the flash-decode kernel reads first are on their way into L2 before it starts: one
+    // thread per page (issued by the few threads that happened to own the first ranks, the
+    // prefetches held the whole CTA up for two microseconds)
+    __syncthreads();
+    if (tid < n_prefetch && tid < K) {
+        const int p = out[tid];
+        if (p >= 0 && p < P) bulk_prefetch_l2(kvh + (int64_t)p * page_bytes, (uint32_t)page_bytes);
     }
     return true;
 }
