@@ -222,7 +222,7 @@ def event_ms(fn, stream=None):
     return e0.elapsed_time(e1)
 
 
-def parity_block(w, cache, sample_inputs, q, tok, K, T0, dev):
+def parity_block(w, cache, sample_inputs, q, tok, K, T0, dev, recall_cache=None, recall_w=None):
     """One decode step of the timed configuration checked against the fp64 oracle on a sample of
     heads (states, stored cache, page bounds, scores, page list, attention output), and the recall
     of the planted pages over all heads for the three budgets.  Runs before the timed region."""
@@ -263,16 +263,18 @@ def parity_block(w, cache, sample_inputs, q, tok, K, T0, dev):
                     "attention_max_abs_err": stats.get("att_max"), "attention_mean_abs_err": stats.get("att_mean")})
     except AssertionError as e:
         out.update({"passed": False, "failure": str(e)[:300]})
-    if w.needles:
-        planted = wl.needle_pages(w, T0)
-        P = w.pages(T0 + 1)
-        rec = {}
+    if w.needles and recall_cache is not None:
+        # pages planted to align with this query, in a cache of the metric's own recipe (copy 0 also
+        # carries the state resets of the prefill case, whose short averages outscore everything)
+        planted = wl.needle_pages(recall_w, T0)
+        P = w.pages(len(recall_cache))
+        rec = {"cache": "copy 1 (no resets), %d tokens" % len(recall_cache)}
         for den in (4, 8, 16):
             Kd = max(1, math.ceil(P / den))
-            if Kd > cache.cfg.max_budget_pages:
+            if Kd > recall_cache.cfg.max_budget_pages:
                 continue
             idd = torch.empty(w.B, w.H, Kd, dtype=torch.int32, device=dev)
-            rq.rq_select_pages(cache.handle, q, Kd, None, idd)
+            rq.rq_select_pages(recall_cache.handle, q, Kd, None, idd)
             sel = idd.cpu().numpy()
             hit = sum(len(set(planted[b, h].tolist()) & set(sel[b, h].tolist())) for b in range(w.B) for h in range(w.H))
             rec[f"1/{den}"] = hit / (w.B * w.H * w.needles)
@@ -288,6 +290,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="rq", choices=["rq", "reference"])
     ap.add_argument("--workload", default="metric")
+    ap.add_argument("--batch", type=int, default=0, help="the chosen workload at another batch size (context runs, not the metric)")
+    ap.add_argument("--context", type=int, default=0, help="the chosen workload at another context length (context runs, not the metric)")
     ap.add_argument("--copies", type=int, default=0, help="independent caches to rotate (0 = auto, at least 4)")
     ap.add_argument("--path", type=int, default=0, choices=[0, 1, 2, 4, 8],
                     help="how the step is launched: 0 the library chooses, 1 separate kernels, 2/4/8 one launch with that many groups of heads")
@@ -297,7 +301,11 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rq" else args.warmup
 
+    import dataclasses
     w = pick_workload(args.workload)
+    if args.batch or args.context:
+        w = dataclasses.replace(w, name=f"{w.name}-b{args.batch or w.B}-t{args.context or w.T}", B=args.batch or w.B,
+                                T=args.context or w.T)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -369,7 +377,8 @@ def main():
 
     parity = None
     if first and not args.no_parity:
-        parity = parity_block(w, caches[0], sample_inputs, qs[0], toks[0], K, T0, dev)
+        parity = parity_block(w, caches[0], sample_inputs, qs[0], toks[0], K, T0, dev, recall_cache=caches[1 % ncopies],
+                              recall_w=dataclasses.replace(w, seed=w.seed + 17 * (1 % ncopies)))
 
     stream = torch.cuda.current_stream()
 

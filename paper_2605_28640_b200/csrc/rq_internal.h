@@ -32,7 +32,8 @@ constexpr int kTargetSMs = 148;        // B200
 constexpr int kStepMaxHeads = 256;     // the one-launch step serves at most this many (batch, head) pairs
 constexpr int kStepBins = 2048;        // value buckets of a head's score histogram
 constexpr int kStepCtrInts = 16;       // int32 per head and counter set (64 bytes)
-constexpr int kTopkFastPages = 10240;  // heads of up to this many pages are selected from the scoring kernel's histogram
+constexpr int kTopkFastPages = 10240;  // heads of up to this many pages are selected from the scoring kernel's histogram,
+constexpr int kTopkHistMinPages = 6144; // and of at least this many: below, counting the pages while scoring costs more than the selection saves
 
 // ---- workspace carving (byte offsets, every region 256-byte aligned) ----
 struct WorkspaceLayout {
@@ -97,8 +98,8 @@ cudaError_t launch_score_select(const DecodeArgs &a, const void *q, const void *
                                 float *scores, int do_update, int budget, int32_t *idx, int idx_stride,
                                 int32_t *attend_ctr, int prefetch, int32_t *ctr_other, cudaStream_t s);
 // prefetch: the flash-decode kernel runs next, start moving the first selected pages into L2
-// sh: the histogram the scoring kernel filled (NULL members: none).  With it, and at most
-// kTopkFastPages pages, the list comes out in no particular order; otherwise ascending.
+// sh: the histogram the scoring kernel filled (NULL members: none).  With it, and
+// kTopkHistMinPages to kTopkFastPages pages, the list comes out in no particular order; otherwise ascending.
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
                         int idx_stride, int32_t *attend_ctr, int prefetch, const ScoreHist &sh, cudaStream_t s);
 // does launch_topk take the histogram path for this many pages per head?

@@ -1,6 +1,11 @@
 // Second kernel of a decode step: per (b,h) selection of the budget's pages from
 // the page scores (the TopK of Eq. 3), forced first/local pages inside the
-// budget (App. A.1), ties to the lower page index, output ascending.
+// budget (App. A.1), ties to the lower page index.  Two routines give the same set:
+// select_rows works from the scores alone (range, value histogram, direct ranking or
+// radix passes; ascending list); fast_select starts from the histogram that the scoring
+// kernel filled while it scored (no pass for the range, no keys; list in no particular
+// order) and hands over to select_rows whenever it cannot finish.  Also here: the
+// short-context kernel that scores and selects a head in one CTA.
 #include <math_constants.h>
 
 #include "rq_async.cuh"
@@ -615,7 +620,7 @@ __global__ void __launch_bounds__(kTopkThreads) score_select_kernel(DecodeArgs a
 
 }  // namespace
 
-bool topk_uses_hist(int64_t pages) { return pages <= kTopkFastPages; }
+bool topk_uses_hist(int64_t pages) { return pages >= kTopkHistMinPages && pages <= kTopkFastPages; }
 
 cudaError_t launch_topk(const DecodeArgs &a, const float *scores, int budget, int32_t *idx,
                         int idx_stride, int32_t *attend_ctr, int prefetch, const ScoreHist &hs, cudaStream_t s)
