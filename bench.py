@@ -37,10 +37,10 @@ METRIC = "sparse decode us/step at 128K ctx, 1/16 budget"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu captures
-# (profiles/*_64k_b1.md: captured on the 64K-context case, scaled by two to the launches of the
+# (profiles/*_96k_b1.md: captured on a 96K-context case, scaled by 4/3 to the launches of the
 # default workload, traffic being proportional to the pages processed): kernel -> bytes, or None
 # when the kernel has changed since the capture.
-NCU_TRAFFIC = {"score": 2 * (67.23e6 + 0.57e6), "attend": 2 * (67.24e6 + 1.05e6), "step": None}
+NCU_TRAFFIC = {"score": 4 / 3 * (100.83e6 + 3.83e6), "attend": 4 / 3 * (100.81e6 + 2.82e6), "step": 4 / 3 * (201.73e6 + 5.03e6)}
 
 
 def measured_peak():
