@@ -579,6 +579,7 @@ int rq_snapkv_select(rq_cache *cache, const void *q_window, int32_t window, int3
     a.scale = scale > 0.0f ? scale : 1.0f / sqrtf((float)c.head_dim);
     const int BH = c.batch * c.heads;
     snap_carve(scratch, BH, cache->len, &a.imp, &a.stats, &a.rowstat);
+    a.status = (int32_t *)((char *)cache->workspace + workspace_layout(c).status);
     if (launch_snap_scores(a, s) != cudaSuccess) return RQ_ERR_CUDA;
     if (launch_snap_select(a.imp, BH, cache->len, window, keep, idx_out, s) != cudaSuccess) return RQ_ERR_CUDA;
     if (importance_out && cudaMemcpyAsync(importance_out, a.imp, (size_t)BH * cache->len * sizeof(float),

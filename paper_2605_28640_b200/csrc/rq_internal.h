@@ -148,6 +148,7 @@ struct SnapArgs {
     float *imp;         // [BH][len] importance of every position
     float2 *stats;      // [BH][tiles][64] per-tile row statistics
     float2 *rowstat;    // [BH][64] final row statistics
+    int32_t *status;    // the cache's device status word (a wait that runs out is reported there)
 };
 size_t snap_scratch_bytes(int BH, int64_t len);
 void snap_carve(void *scratch, int BH, int64_t len, float **imp, float2 **stats, float2 **rowstat);

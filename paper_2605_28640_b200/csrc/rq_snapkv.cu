@@ -6,27 +6,36 @@
 //
 //   importance[j] = sum_i softmax_j(scale * q_i . k~_j),  query i at position T - W + i sees j <= T - W + i
 //
-// Kernels (plain fp32 ALU work; the window is at most 64 queries, so the score pass is a thin
-// 64 x T x D contraction per head):
-//   snap_tile_kernel<PASS 1>  per (head, tile of 128 keys): the 64 x 128 block of scores in registers
-//                             (8 rows x 4 keys per thread, operands from shared memory), per row the
-//                             block's maximum and sum of exponentials -> partial statistics
-//   snap_rows_kernel          per (head, query): merges the partial statistics of all tiles
-//   snap_tile_kernel<PASS 2>  the same block of scores again, turned into weights with the final
-//                             statistics and summed over the queries -> importance of the tile's keys
+// Kernels.  The importance is a dense contraction (W x D x T per head) followed by a softmax over T
+// and a sum over the window.  The 64 x T scores of a head are never stored: the keys are read twice,
+// once for the row statistics (maximum and sum of exponentials of every query) and once for the
+// weights.
+//   snap_mma_kernel<PASS 1>   bf16 caches.  Per (head, run of 128-key tiles): the scores of a tile on the
+//                             tensor cores (tcgen05.mma, operands in shared memory, fp32 accumulator
+//                             in tensor memory): D[query][key] with the window's queries as the M
+//                             side (both halves of the 128 rows hold the same 64 queries, so that all
+//                             four warps have rows to work on: the upper half takes the tile's upper 64
+//                             keys), a thread per (query, half of the keys) keeps a running maximum
+//                             and sum of exponentials -> partial statistics per run
+//   snap_rows_kernel          per (head, query): merges the partial statistics
+//   snap_mma_kernel<PASS 2>   the same products with the roles swapped, D[key][query] (keys as the M
+//                             side), so that a thread owns a key and sums its weights over the
+//                             queries without any exchange -> importance of the tile's keys
+//   snap_tile_kernel<1 / 2>   fp32 caches: the same two passes as plain fp32 FMA code (64 x 128
+//                             score tiles in registers, 8 rows x 4 keys per thread)
 //   snap_select_kernel        per head: the keep - W most important positions before the window
 //                             (most-significant-digit radix select on the order-preserving image of the
 //                             importance, equal importance to the lower position) plus the window,
 //                             written in ascending order
 //   snap_compact_kernel       per (head, page of the new cache): gathers the retained rows, rebuilds
 //                             the page's min/max bounds, tracks the head's largest |key|
-// The keys are read twice (statistics, then weights): the 64 x T scores of a head are never stored.
 #include <math.h>
 #include <math_constants.h>
 
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
+#include "rq_umma.cuh"
 
 namespace rq {
 
@@ -161,6 +170,184 @@ __global__ void __launch_bounds__(kSnapThreads) snap_tile_kernel(const T *kv, in
             if (j0 + tid < len) imp[(int64_t)bh * len + j0 + tid] = s;
         }
     }
+}
+
+// ---------------------------------------------------------------- the two passes on the tensor cores (bf16)
+constexpr int kMmaKeys = 128;                  // keys per tile
+constexpr int kMmaThreads = 128;               // one thread per accumulator lane
+constexpr int kMmaStages = 2;                  // key tiles in shared memory (two CTAs per SM)
+constexpr int kMmaMaxTiles = 8;                // tiles per CTA at most
+
+template <int D>
+struct SnapMmaGeom {
+    static constexpr int PIECES = D / 8;                       // 16-byte pieces of a row
+    static constexpr int SBO = PIECES * 128;                   // bytes from one group of 8 rows to the next
+    static constexpr int Q_BYTES = 128 * D * 2;                // the window's queries, twice
+    static constexpr int TILE_BYTES = kMmaKeys * D * 2;
+    static constexpr int SMEM_BYTES = Q_BYTES + kMmaStages * TILE_BYTES;
+};
+
+__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Grid (runs of tiles, heads).  stats: [bh][runs][64]; rowstat: [bh][64]; imp: [bh][len].
+template <int D, int PASS>
+__global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const bf16 *kv, int64_t page_cap, int S, int64_t len,
+                                                               const bf16 *qw, int W, int H, float scale_log2,
+                                                               float2 *stats, const float2 *rowstat, float *imp,
+                                                               int ntiles, int tiles_per_cta, int32_t *status)
+{
+    using G = SnapMmaGeom<D>;
+    constexpr int PIECES = G::PIECES;
+    constexpr int NST = kMmaStages;
+    constexpr uint32_t TCOLS = PASS == 1 ? 128 : 64;           // accumulator columns
+    extern __shared__ __align__(128) unsigned char dsm[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t tbase;
+    __shared__ float2 qst[kSnapRows];                          // pass 1: merge of the two halves; pass 2: (max, 1 / sum) per query
+    unsigned char *qs = dsm, *ks = dsm + G::Q_BYTES;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int t0 = blockIdx.x * tiles_per_cta, n = min(tiles_per_cta, ntiles - t0);
+    const int64_t first_q = len - W;                           // position of query 0
+
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        mbar_init_fence();
+    }
+    if (warp == 0) tmem_alloc(&tbase, TCOLS);
+    // the window's queries of this head (qw is [B][W][H][D]) in rows r and r + 64; rows beyond the window are zero
+    for (int i = tid; i < 128 * PIECES; i += kMmaThreads) {
+        const int r = i / PIECES, c = i % PIECES, qr = r & (kSnapRows - 1);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (qr < W) v = *reinterpret_cast<const uint4 *>(qw + (((int64_t)b * W + qr) * H + h) * D + c * 8);
+        *reinterpret_cast<uint4 *>(qs + umma_tile_offset(r, c, PIECES)) = v;
+    }
+    if (PASS == 2 && tid < kSnapRows) {
+        const float2 f = tid < W ? rowstat[(int64_t)bh * kSnapRows + tid] : make_float2(0.0f, 1.0f);
+        qst[tid] = make_float2(f.x, 1.0f / f.y);
+    }
+    // a tile's keys: position j lives in page j / S, slot j % S of the head's cache.  A warp-wide copy
+    // takes 8 rows x 4 pieces: 64 consecutive bytes per row from global memory, 512 consecutive bytes in
+    // shared memory
+    auto issue = [&](int t, int stage) {
+        unsigned char *dst = ks + (size_t)stage * G::TILE_BYTES;
+        const int64_t j0 = (int64_t)t * kMmaKeys;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int r = (warp + 4 * g) * 8 + (lane & 7);
+            const int64_t j = j0 + r;
+            if (j < len) {
+                const bf16 *src = kv + ((((int64_t)bh * page_cap + j / S) * 2) * S + j % S) * D;
+#pragma unroll
+                for (int cg = 0; cg < PIECES / 4; ++cg) {
+                    const int c = cg * 4 + (lane >> 3);
+                    cp_async16(dst + umma_tile_offset(r, c, PIECES), src + c * 8);
+                }
+            }
+        }
+    };
+#pragma unroll 1
+    for (int s = 0; s < NST - 1; ++s) {
+        if (s < n) issue(t0 + s, s);
+        cp_async_commit();
+    }
+
+    const int row = tid & (kSnapRows - 1), half = tid >> 6;    // pass 1: this thread's query and half of the tile's keys
+    float m = -CUDART_INF_F, l = 0.0f;                         // pass 1: running statistics
+    bool ok = true;
+    uint32_t tb = 0;
+#pragma unroll 1
+    for (int i = 0; i < n; ++i) {
+        cp_async_wait<NST - 2>();                              // this thread's pieces of tile i have landed
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ... and are visible to the tensor core's reads
+        tcgen05_before_sync();
+        if (!__syncthreads_and(ok)) break;                     // everybody's pieces; the accumulator of tile i - 1 has been read
+        tcgen05_after_sync();
+        tb = tbase;
+        if (tid == 0) {
+            constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
+            const uint32_t qa = smem_addr(qs), ka = smem_addr(ks + (size_t)(i % NST) * G::TILE_BYTES);
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+                const uint64_t dq = umma_desc(qa + k * 256, G::SBO), dk = umma_desc(ka + k * 256, G::SBO);
+                if (PASS == 1) umma_bf16(tb, dq, dk, idesc, k > 0);
+                else umma_bf16(tb, dk, dq, idesc, k > 0);
+            }
+            umma_commit(&bar);
+        }
+        // the stage of tile i - 1 is free: its product completed before the accumulator was read
+        if (i + NST - 1 < n) issue(t0 + i + NST - 1, (i + NST - 1) % NST);
+        cp_async_commit();
+        ok = mbar_wait(&bar, (uint32_t)(i & 1));
+        tcgen05_after_sync();
+        const int64_t j0 = (int64_t)(t0 + i) * kMmaKeys;
+        const uint32_t tl = tb + ((uint32_t)(warp * 32) << 16);    // this warp's lanes
+        if (PASS == 1) {
+            // lane = query (both halves of the lanes hold the same 64 queries), column = key
+            const int64_t pq = first_q + row;                  // query `row` sees keys up to its own position
+#pragma unroll 1
+            for (int cb = 0; cb < 64; cb += 32) {
+                float v[32];
+                tmem_ld32(tl + (uint32_t)(half * 64 + cb), v);
+                const int64_t jb = j0 + half * 64 + cb;
+                if (row < W && jb <= pq) {
+                    const int nv = (int)min((int64_t)32, pq - jb + 1);   // visible keys among these 32
+                    float tm = -CUDART_INF_F;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        v[c] = c < nv ? v[c] * scale_log2 : -CUDART_INF_F;
+                        tm = fmaxf(tm, v[c]);
+                    }
+                    const float mn = fmaxf(m, tm);             // finite: at least one key is visible
+                    float sum = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) sum += exp2f(v[c] - mn);
+                    l = l * exp2f(m - mn) + sum;               // exp2f(-inf) = 0 the first time
+                    m = mn;
+                }
+            }
+        } else {
+            // lane = key, column = query: the key's weights summed over the queries that see it
+            const int64_t j = j0 + tid;
+            const int q_lo = (int)max((int64_t)0, j - first_q);
+            float acc = 0.0f;
+#pragma unroll 1
+            for (int cb = 0; cb < kSnapRows; cb += 32) {
+                float v[32];
+                tmem_ld32(tl + (uint32_t)cb, v);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const int q = cb + c;
+                    const float2 st = qst[q];
+                    if (q < W && q >= q_lo) acc = fmaf(exp2f(fmaf(v[c], scale_log2, -st.x)), st.y, acc);
+                }
+            }
+            if (j < len) imp[(int64_t)bh * len + j] = acc;
+        }
+    }
+    cp_async_wait<0>();
+    if (__any_sync(0xffffffffu, !ok) && lane == 0) atomicCAS(status, RQ_OK, RQ_ERR_TIMEOUT);
+    if (PASS == 1) {
+        // the two halves of a query's keys, merged through shared memory
+        if (half == 1) qst[row] = make_float2(m, l);
+        __syncthreads();
+        if (half == 0) {
+            const float2 o = qst[row];
+            const float mn = fmaxf(m, o.x);
+            float lt = 0.0f;
+            if (mn > -CUDART_INF_F) lt = l * exp2f(m - mn) + o.y * exp2f(o.x - mn);
+            stats[((int64_t)bh * gridDim.x + blockIdx.x) * kSnapRows + row] = make_float2(mn, lt);
+        }
+    }
+    tcgen05_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, TCOLS);
 }
 
 // Final statistics of a row: merge of its tiles' (max, sum exp).  One warp per (head, row).
@@ -365,6 +552,39 @@ cudaError_t snap_scores_t(const SnapArgs &a, cudaStream_t s)
     return cudaGetLastError();
 }
 
+template <int D>
+cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
+{
+    using G = SnapMmaGeom<D>;
+    static bool ready[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!ready[dev]) {
+        e = cudaFuncSetAttribute(snap_mma_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(snap_mma_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        ready[dev] = true;
+    }
+    const int BH = a.B * a.H;
+    const int ntiles = (int)((a.len + kMmaKeys - 1) / kMmaKeys);
+    // tiles per CTA: as many as leave a few CTAs for every SM
+    int tpc = kMmaMaxTiles;
+    while (tpc > 1 && (int64_t)BH * ((ntiles + tpc - 1) / tpc) < 4 * (int64_t)sm_count()) tpc >>= 1;
+    const int runs = (ntiles + tpc - 1) / tpc;
+    const dim3 grid((unsigned)runs, (unsigned)BH);
+    const float sl2 = a.scale * 1.4426950408889634f;
+    snap_mma_kernel<D, 1><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>((const bf16 *)a.kv, a.page_cap, a.S, a.len, (const bf16 *)a.qw,
+                                                                 a.W, a.H, sl2, a.stats, nullptr, nullptr, ntiles, tpc, a.status);
+    const int rows = BH * kSnapRows;
+    snap_rows_kernel<<<(rows * 32 + 127) / 128, 128, 0, s>>>(a.stats, a.rowstat, runs, rows);
+    snap_mma_kernel<D, 2><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>((const bf16 *)a.kv, a.page_cap, a.S, a.len, (const bf16 *)a.qw,
+                                                                 a.W, a.H, sl2, nullptr, a.rowstat, a.imp, ntiles, tpc, a.status);
+    return cudaGetLastError();
+}
+
 size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 }  // namespace
@@ -393,8 +613,8 @@ cudaError_t launch_snap_scores(const SnapArgs &a, cudaStream_t s)
     if (a.W < 1 || a.W > kSnapRows || a.len < a.W) return cudaErrorInvalidValue;
     if (a.B * a.H > 65535) return cudaErrorInvalidValue;
     if (a.dtype == RQ_BF16) {
-        if (a.D == 128) return snap_scores_t<bf16, 128>(a, s);
-        if (a.D == 64) return snap_scores_t<bf16, 64>(a, s);
+        if (a.D == 128) return snap_scores_mma<128>(a, s);
+        if (a.D == 64) return snap_scores_mma<64>(a, s);
     } else {
         if (a.D == 128) return snap_scores_t<float, 128>(a, s);
         if (a.D == 64) return snap_scores_t<float, 64>(a, s);
