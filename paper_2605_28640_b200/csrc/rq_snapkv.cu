@@ -29,6 +29,7 @@
 //                             written in ascending order
 //   snap_compact_kernel       per (head, page of the new cache): gathers the retained rows, rebuilds
 //                             the page's min/max bounds, tracks the head's largest |key|
+#include <cuda.h>
 #include <math.h>
 #include <math_constants.h>
 
@@ -175,119 +176,132 @@ __global__ void __launch_bounds__(kSnapThreads) snap_tile_kernel(const T *kv, in
 // ---------------------------------------------------------------- the two passes on the tensor cores (bf16)
 constexpr int kMmaKeys = 128;                  // keys per tile
 constexpr int kMmaThreads = 128;               // one thread per accumulator lane
-constexpr int kMmaStages = 2;                  // key tiles in shared memory (two CTAs per SM)
-constexpr int kMmaMaxTiles = 8;                // tiles per CTA at most
+constexpr int kMmaStages = 5;                  // key tiles in shared memory: four in flight while one is multiplied
+constexpr int kMmaMaxTiles = 32;               // tiles per CTA at most
 
 template <int D>
 struct SnapMmaGeom {
-    static constexpr int PIECES = D / 8;                       // 16-byte pieces of a row
-    static constexpr int SBO = PIECES * 128;                   // bytes from one group of 8 rows to the next
-    static constexpr int Q_BYTES = 128 * D * 2;                // the window's queries, twice
-    static constexpr int TILE_BYTES = kMmaKeys * D * 2;
-    static constexpr int SMEM_BYTES = Q_BYTES + kMmaStages * TILE_BYTES;
+    static constexpr int HALVES = D / 64;                      // 64-element (128-byte) halves of a row
+    static constexpr int HALF_BYTES = 128 * 128;               // 128 rows of one half
+    static constexpr int Q_BYTES = HALVES * HALF_BYTES;        // the window's queries, twice (128 rows)
+    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;     // 128 keys
+    static constexpr int SMEM_BYTES = Q_BYTES + kMmaStages * TILE_BYTES + 1024;   // + room to align the base to 1024 bytes
 };
 
-__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src)
+// 2^x for x <= 0 (and -inf): the hardware approximation, relative error about 2^-22
+__device__ __forceinline__ float exp2_fast(float x)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src) : "memory");
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Grid (runs of tiles, heads).  stats: [bh][runs][64]; rowstat: [bh][64]; imp: [bh][len].
+// tmap: the cache as a rank-4 tensor (channel, slot, key / value, page over all heads), box = 64 channels
+// x the slots of a page x keys only x the pages of 128 positions, 128-byte swizzle: one copy brings one
+// 64-channel half of a tile's keys into shared memory in the layout the tensor core reads.
 template <int D, int PASS>
-__global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const bf16 *kv, int64_t page_cap, int S, int64_t len,
-                                                               const bf16 *qw, int W, int H, float scale_log2,
+__global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_constant__ CUtensorMap tmap, int64_t page_cap, int S,
+                                                               int64_t len, const bf16 *qw, int W, int H, float scale_log2,
                                                                float2 *stats, const float2 *rowstat, float *imp,
                                                                int ntiles, int tiles_per_cta, int32_t *status)
 {
     using G = SnapMmaGeom<D>;
-    constexpr int PIECES = G::PIECES;
     constexpr int NST = kMmaStages;
-    constexpr uint32_t TCOLS = PASS == 1 ? 128 : 64;           // accumulator columns
-    extern __shared__ __align__(128) unsigned char dsm[];
-    __shared__ __align__(8) uint64_t bar;
+    constexpr uint32_t ACC = PASS == 1 ? 128 : 64;             // columns of one accumulator
+    constexpr uint32_t TCOLS = 2 * ACC;                        // two accumulators: one is filled while the other is read
+    extern __shared__ __align__(1024) unsigned char dsm_raw[];
+    __shared__ __align__(8) uint64_t bar[2];                   // an accumulator's product is complete
+    __shared__ __align__(8) uint64_t full[NST];                // a stage's keys have landed
     __shared__ uint32_t tbase;
     __shared__ float2 qst[kSnapRows];                          // pass 1: merge of the two halves; pass 2: (max, 1 / sum) per query
+    unsigned char *dsm = dsm_raw + ((1024u - (smem_addr(dsm_raw) & 1023u)) & 1023u);
     unsigned char *qs = dsm, *ks = dsm + G::Q_BYTES;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int t0 = blockIdx.x * tiles_per_cta, n = min(tiles_per_cta, ntiles - t0);
     const int64_t first_q = len - W;                           // position of query 0
+    const int ppt = kMmaKeys / S;                              // pages per tile
+    int n_issued = 0, n_landed = 0;                            // thread 0: tiles whose copies were started / seen complete
 
     if (tid == 0) {
-        mbar_init(&bar, 1);
+        mbar_init(&bar[0], 1);
+        mbar_init(&bar[1], 1);
+        for (int s = 0; s < NST; ++s) mbar_init(&full[s], 1);
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(&tbase, TCOLS);
     // the window's queries of this head (qw is [B][W][H][D]) in rows r and r + 64; rows beyond the window are zero
-    for (int i = tid; i < 128 * PIECES; i += kMmaThreads) {
-        const int r = i / PIECES, c = i % PIECES, qr = r & (kSnapRows - 1);
+    for (int i = tid; i < 128 * (D / 8); i += kMmaThreads) {
+        const int r = i / (D / 8), c = i % (D / 8), qr = r & (kSnapRows - 1);
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (qr < W) v = *reinterpret_cast<const uint4 *>(qw + (((int64_t)b * W + qr) * H + h) * D + c * 8);
-        *reinterpret_cast<uint4 *>(qs + umma_tile_offset(r, c, PIECES)) = v;
+        *reinterpret_cast<uint4 *>(qs + (c >> 3) * G::HALF_BYTES + umma_sw128_offset(r, c & 7)) = v;
     }
     if (PASS == 2 && tid < kSnapRows) {
         const float2 f = tid < W ? rowstat[(int64_t)bh * kSnapRows + tid] : make_float2(0.0f, 1.0f);
         qst[tid] = make_float2(f.x, 1.0f / f.y);
     }
-    // a tile's keys: position j lives in page j / S, slot j % S of the head's cache.  A warp-wide copy
-    // takes 8 rows x 4 pieces: 64 consecutive bytes per row from global memory, 512 consecutive bytes in
-    // shared memory
-    auto issue = [&](int t, int stage) {
+    // the keys of tile t (relative to t0) into its stage: position j lives in page j / S, slot j % S of the
+    // head's cache; pages past the head's last one hold somebody else's rows or nothing, and every key at
+    // or beyond `len` is masked where the scores are used.  One thread.
+    auto issue = [&](int i) {
+        const int stage = i % NST;
         unsigned char *dst = ks + (size_t)stage * G::TILE_BYTES;
-        const int64_t j0 = (int64_t)t * kMmaKeys;
+        const int page = (int)((int64_t)bh * page_cap + (int64_t)(t0 + i) * ppt);
+        mbar_arrive_expect_tx(&full[stage], G::TILE_BYTES);
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const int r = (warp + 4 * g) * 8 + (lane & 7);
-            const int64_t j = j0 + r;
-            if (j < len) {
-                const bf16 *src = kv + ((((int64_t)bh * page_cap + j / S) * 2) * S + j % S) * D;
-#pragma unroll
-                for (int cg = 0; cg < PIECES / 4; ++cg) {
-                    const int c = cg * 4 + (lane >> 3);
-                    cp_async16(dst + umma_tile_offset(r, c, PIECES), src + c * 8);
-                }
-            }
-        }
+        for (int hh = 0; hh < G::HALVES; ++hh) tma_load_4d(dst + hh * G::HALF_BYTES, &tmap, hh * 64, 0, 0, page, &full[stage]);
+        n_issued = i + 1;
     };
-#pragma unroll 1
-    for (int s = 0; s < NST - 1; ++s) {
-        if (s < n) issue(t0 + s, s);
-        cp_async_commit();
-    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the queries, written with ordinary stores, are read by the tensor core
+    tcgen05_before_sync();
+    __syncthreads();
+    tcgen05_after_sync();
+    const uint32_t tb = tbase;
 
     const int row = tid & (kSnapRows - 1), half = tid >> 6;    // pass 1: this thread's query and half of the tile's keys
     float m = -CUDART_INF_F, l = 0.0f;                         // pass 1: running statistics
     bool ok = true;
-    uint32_t tb = 0;
+    // the product of tile i (relative to t0) into accumulator i & 1, once the tile's keys have landed; the
+    // barrier of that accumulator gets one arrival when it is complete.  One thread.
+    auto product = [&](int i) -> bool {
+        constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
+        if (!mbar_wait(&full[i % NST], (uint32_t)((i / NST) & 1))) return false;
+        n_landed = i + 1;
+        tcgen05_after_sync();
+        const uint32_t qa = smem_addr(qs), ka = smem_addr(ks + (size_t)(i % NST) * G::TILE_BYTES);
+        const uint32_t acc = tb + (uint32_t)(i & 1) * ACC;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) {
+            const uint32_t off = (uint32_t)(k >> 2) * G::HALF_BYTES + (uint32_t)(k & 3) * 32u;
+            const uint64_t dq = umma_desc_sw128(qa + off), dk = umma_desc_sw128(ka + off);
+            if (PASS == 1) umma_bf16(acc, dq, dk, idesc, k > 0);
+            else umma_bf16(acc, dk, dq, idesc, k > 0);
+        }
+        umma_commit(&bar[i & 1]);
+        return true;
+    };
+    if (tid == 0) {
+        for (int s = 0; s < NST - 1 && s < n; ++s) issue(s);
+        if (n > 0) ok = product(0);
+    }
 #pragma unroll 1
     for (int i = 0; i < n; ++i) {
-        cp_async_wait<NST - 2>();                              // this thread's pieces of tile i have landed
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ... and are visible to the tensor core's reads
         tcgen05_before_sync();
-        if (!__syncthreads_and(ok)) break;                     // everybody's pieces; the accumulator of tile i - 1 has been read
+        if (!__syncthreads_and(ok)) break;                     // accumulator (i + 1) & 1 has been read by everybody (tile i - 1)
         tcgen05_after_sync();
-        tb = tbase;
         if (tid == 0) {
-            constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
-            const uint32_t qa = smem_addr(qs), ka = smem_addr(ks + (size_t)(i % NST) * G::TILE_BYTES);
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-                const uint64_t dq = umma_desc(qa + k * 256, G::SBO), dk = umma_desc(ka + k * 256, G::SBO);
-                if (PASS == 1) umma_bf16(tb, dq, dk, idesc, k > 0);
-                else umma_bf16(tb, dk, dq, idesc, k > 0);
-            }
-            umma_commit(&bar);
+            // the next tile's product runs while this tile's accumulator is worked on; the stage of tile
+            // i - 1 is free (its product completed before its accumulator was read) and takes tile i + NST - 1
+            if (i + 1 < n) ok = product(i + 1);
+            if (i + NST - 1 < n) issue(i + NST - 1);
         }
-        // the stage of tile i - 1 is free: its product completed before the accumulator was read
-        if (i + NST - 1 < n) issue(t0 + i + NST - 1, (i + NST - 1) % NST);
-        cp_async_commit();
-        ok = mbar_wait(&bar, (uint32_t)(i & 1));
+        ok = mbar_wait(&bar[i & 1], (uint32_t)((i >> 1) & 1)) && ok;
         tcgen05_after_sync();
         const int64_t j0 = (int64_t)(t0 + i) * kMmaKeys;
-        const uint32_t tl = tb + ((uint32_t)(warp * 32) << 16);    // this warp's lanes
+        const uint32_t tl = tb + (uint32_t)(i & 1) * ACC + ((uint32_t)(warp * 32) << 16);    // this warp's lanes of the accumulator
         if (PASS == 1) {
             // lane = query (both halves of the lanes hold the same 64 queries), column = key
             const int64_t pq = first_q + row;                  // query `row` sees keys up to its own position
@@ -307,8 +321,8 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const bf16 *kv, i
                     const float mn = fmaxf(m, tm);             // finite: at least one key is visible
                     float sum = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) sum += exp2f(v[c] - mn);
-                    l = l * exp2f(m - mn) + sum;               // exp2f(-inf) = 0 the first time
+                    for (int c = 0; c < 32; ++c) sum += exp2_fast(v[c] - mn);
+                    l = l * exp2_fast(m - mn) + sum;           // 2^(-inf) = 0 the first time
                     m = mn;
                 }
             }
@@ -325,13 +339,15 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const bf16 *kv, i
                 for (int c = 0; c < 32; ++c) {
                     const int q = cb + c;
                     const float2 st = qst[q];
-                    if (q < W && q >= q_lo) acc = fmaf(exp2f(fmaf(v[c], scale_log2, -st.x)), st.y, acc);
+                    if (q < W && q >= q_lo) acc = fmaf(exp2_fast(fmaf(v[c], scale_log2, -st.x)), st.y, acc);
                 }
             }
             if (j < len) imp[(int64_t)bh * len + j] = acc;
         }
     }
-    cp_async_wait<0>();
+    // after a wait that ran out: no copy may still be on its way into this CTA's shared memory when it exits
+    if (tid == 0)
+        for (int k = n_landed; k < n_issued; ++k) mbar_wait(&full[k % NST], (uint32_t)((k / NST) & 1));
     if (__any_sync(0xffffffffu, !ok) && lane == 0) atomicCAS(status, RQ_OK, RQ_ERR_TIMEOUT);
     if (PASS == 1) {
         // the two halves of a query's keys, merged through shared memory
@@ -552,6 +568,23 @@ cudaError_t snap_scores_t(const SnapArgs &a, cudaStream_t s)
     return cudaGetLastError();
 }
 
+// The driver's tensor-map encoder, looked up once through the runtime (the library does not link the driver).
+typedef CUresult (*TensorMapEncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                         const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                         CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+TensorMapEncodeTiled tensor_map_encoder()
+{
+    static TensorMapEncodeTiled fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = (TensorMapEncodeTiled)p;
+    }
+    return fn;
+}
+
 template <int D>
 cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
 {
@@ -569,19 +602,31 @@ cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
         ready[dev] = true;
     }
     const int BH = a.B * a.H;
+    if (kMmaKeys % a.S != 0) return cudaErrorInvalidValue;
+    // the cache [BH][page][key / value][slot][channel] as a rank-4 tensor, pages of all heads in one dimension
+    const TensorMapEncodeTiled encode = tensor_map_encoder();
+    if (!encode) return cudaErrorNotSupported;
+    alignas(64) CUtensorMap tmap;
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)a.S, 2, (cuuint64_t)BH * (cuuint64_t)a.page_cap};
+    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)a.S * D * 2, (cuuint64_t)2 * a.S * D * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)a.S, 1, (cuuint32_t)(kMmaKeys / a.S)}, steps[4] = {1, 1, 1, 1};
+    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(a.kv), dims, strides, box, steps,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
     const int ntiles = (int)((a.len + kMmaKeys - 1) / kMmaKeys);
-    // tiles per CTA: as many as leave a few CTAs for every SM
+    // tiles per CTA: as many as leave a couple of CTAs for every SM
     int tpc = kMmaMaxTiles;
-    while (tpc > 1 && (int64_t)BH * ((ntiles + tpc - 1) / tpc) < 4 * (int64_t)sm_count()) tpc >>= 1;
+    while (tpc > 1 && (int64_t)BH * ((ntiles + tpc - 1) / tpc) < 2 * (int64_t)sm_count()) tpc >>= 1;
     const int runs = (ntiles + tpc - 1) / tpc;
     const dim3 grid((unsigned)runs, (unsigned)BH);
     const float sl2 = a.scale * 1.4426950408889634f;
-    snap_mma_kernel<D, 1><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>((const bf16 *)a.kv, a.page_cap, a.S, a.len, (const bf16 *)a.qw,
-                                                                 a.W, a.H, sl2, a.stats, nullptr, nullptr, ntiles, tpc, a.status);
+    snap_mma_kernel<D, 1><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>(tmap, a.page_cap, a.S, a.len, (const bf16 *)a.qw, a.W, a.H, sl2,
+                                                                 a.stats, nullptr, nullptr, ntiles, tpc, a.status);
     const int rows = BH * kSnapRows;
     snap_rows_kernel<<<(rows * 32 + 127) / 128, 128, 0, s>>>(a.stats, a.rowstat, runs, rows);
-    snap_mma_kernel<D, 2><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>((const bf16 *)a.kv, a.page_cap, a.S, a.len, (const bf16 *)a.qw,
-                                                                 a.W, a.H, sl2, nullptr, a.rowstat, a.imp, ntiles, tpc, a.status);
+    snap_mma_kernel<D, 2><<<grid, kMmaThreads, G::SMEM_BYTES, s>>>(tmap, a.page_cap, a.S, a.len, (const bf16 *)a.qw, a.W, a.H, sl2,
+                                                                 nullptr, a.rowstat, a.imp, ntiles, tpc, a.status);
     return cudaGetLastError();
 }
 

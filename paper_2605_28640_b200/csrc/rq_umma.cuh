@@ -31,6 +31,31 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo_bytes
            (1ull << 46);
 }
 
+// The same tiles with the 128-byte swizzle, which is what a tiled bulk-tensor copy (TMA) with
+// CU_TENSOR_MAP_SWIZZLE_128B writes: the K extent is cut into halves of 64 elements (128 bytes); a half
+// holds its rows 128 bytes apart, groups of 8 rows 1024 bytes apart, and inside a row the 16-byte piece p
+// sits at ((p ^ (row % 8)) * 16).  Tile bases are 1024-byte aligned.  A K step of 16 elements is 32 bytes
+// further on inside the half.
+__device__ __forceinline__ uint32_t umma_sw128_offset(int row, int piece)   // piece: 0..7 inside the half
+{
+    return (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u + (uint32_t)((piece ^ (row & 7)) * 16);
+}
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Tiled bulk-tensor copy of one box of a rank-4 tensor map into shared memory; completion (the box's
+// bytes) is counted on the barrier.  One thread.
+__device__ __forceinline__ void tma_load_4d(void *dst_smem, const void *tmap, int c0, int c1, int c2, int c3, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(
+            smem_addr(dst_smem)),
+        "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_addr(bar))
+        : "memory");
+}
+
 // instruction descriptor of D[M x N] (fp32) = A[M x 16] (bf16, K-major) * B[N x 16]^T (bf16, K-major)
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N)
 {
