@@ -27,6 +27,12 @@ __device__ __forceinline__ void mbar_init_fence()
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// One plain arrival.
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 // One arrival that also announces `bytes` of copy traffic to wait for.
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
 {

@@ -175,7 +175,8 @@ __global__ void __launch_bounds__(kSnapThreads) snap_tile_kernel(const T *kv, in
 
 // ---------------------------------------------------------------- the two passes on the tensor cores (bf16)
 constexpr int kMmaKeys = 128;                  // keys per tile
-constexpr int kMmaThreads = 128;               // one thread per accumulator lane
+constexpr int kMmaWarps = 4;                   // warps that read the accumulator: one thread per lane of it
+constexpr int kMmaThreads = (kMmaWarps + 1) * 32;   // and one warp that starts the copies and the products
 constexpr int kMmaStages = 5;                  // key tiles in shared memory: four in flight while one is multiplied
 constexpr int kMmaMaxTiles = 32;               // tiles per CTA at most
 
@@ -213,6 +214,7 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
     extern __shared__ __align__(1024) unsigned char dsm_raw[];
     __shared__ __align__(8) uint64_t bar[2];                   // an accumulator's product is complete
     __shared__ __align__(8) uint64_t full[NST];                // a stage's keys have landed
+    __shared__ __align__(8) uint64_t acc_free[2];              // an accumulator has been read by all four warps
     __shared__ uint32_t tbase;
     __shared__ float2 qst[kSnapRows];                          // pass 1: merge of the two halves; pass 2: (max, 1 / sum) per query
     unsigned char *dsm = dsm_raw + ((1024u - (smem_addr(dsm_raw) & 1023u)) & 1023u);
@@ -229,6 +231,8 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
         mbar_init(&bar[0], 1);
         mbar_init(&bar[1], 1);
         for (int s = 0; s < NST; ++s) mbar_init(&full[s], 1);
+        mbar_init(&acc_free[0], kMmaWarps * 32);
+        mbar_init(&acc_free[1], kMmaWarps * 32);
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(&tbase, TCOLS);
@@ -261,44 +265,48 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
     tcgen05_after_sync();
     const uint32_t tb = tbase;
 
-    const int row = tid & (kSnapRows - 1), half = tid >> 6;    // pass 1: this thread's query and half of the tile's keys
+    const int row = tid & (kSnapRows - 1), half = (tid >> 6) & 1;   // pass 1: this thread's query and half of the tile's keys
     float m = -CUDART_INF_F, l = 0.0f;                         // pass 1: running statistics
     bool ok = true;
-    // the product of tile i (relative to t0) into accumulator i & 1, once the tile's keys have landed; the
-    // barrier of that accumulator gets one arrival when it is complete.  One thread.
-    auto product = [&](int i) -> bool {
-        constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
-        if (!mbar_wait(&full[i % NST], (uint32_t)((i / NST) & 1))) return false;
-        n_landed = i + 1;
-        tcgen05_after_sync();
-        const uint32_t qa = smem_addr(qs), ka = smem_addr(ks + (size_t)(i % NST) * G::TILE_BYTES);
-        const uint32_t acc = tb + (uint32_t)(i & 1) * ACC;
+    if (warp == kMmaWarps) {
+        // ---- the producing warp: one thread starts the copies and the products; nobody else waits for it
+        // except through the barriers
+        if (lane == 0) {
+            for (int s = 0; s < NST && s < n; ++s) issue(s);
+            constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
+            const uint32_t qa = smem_addr(qs);
+#pragma unroll 1
+            for (int i = 0; i < n && ok; ++i) {
+                // accumulator i & 1 has been read (tile i - 2), the tile's keys have landed
+                if (i >= 2) ok = mbar_wait(&acc_free[i & 1], (uint32_t)(((i >> 1) - 1) & 1));
+                ok = ok && mbar_wait(&full[i % NST], (uint32_t)((i / NST) & 1));
+                if (!ok) break;
+                n_landed = i + 1;
+                tcgen05_after_sync();
+                const uint32_t ka = smem_addr(ks + (size_t)(i % NST) * G::TILE_BYTES);
+                const uint32_t acc = tb + (uint32_t)(i & 1) * ACC;
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-            const uint32_t off = (uint32_t)(k >> 2) * G::HALF_BYTES + (uint32_t)(k & 3) * 32u;
-            const uint64_t dq = umma_desc_sw128(qa + off), dk = umma_desc_sw128(ka + off);
-            if (PASS == 1) umma_bf16(acc, dq, dk, idesc, k > 0);
-            else umma_bf16(acc, dk, dq, idesc, k > 0);
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (uint32_t)(k >> 2) * G::HALF_BYTES + (uint32_t)(k & 3) * 32u;
+                    const uint64_t dq = umma_desc_sw128(qa + off), dk = umma_desc_sw128(ka + off);
+                    if (PASS == 1) umma_bf16(acc, dq, dk, idesc, k > 0);
+                    else umma_bf16(acc, dk, dq, idesc, k > 0);
+                }
+                umma_commit(&bar[i & 1]);
+                // the stage of tile i - 1 is free once its product has completed; it takes tile i - 1 + NST
+                if (i >= 1 && i - 1 + NST < n) {
+                    ok = mbar_wait(&bar[(i - 1) & 1], (uint32_t)(((i - 1) >> 1) & 1));
+                    if (ok) issue(i - 1 + NST);
+                }
+            }
+            // after a wait that ran out: no copy may still be on its way into this CTA's shared memory when it exits
+            for (int k = n_landed; k < n_issued; ++k) mbar_wait(&full[k % NST], (uint32_t)((k / NST) & 1));
         }
-        umma_commit(&bar[i & 1]);
-        return true;
-    };
-    if (tid == 0) {
-        for (int s = 0; s < NST - 1 && s < n; ++s) issue(s);
-        if (n > 0) ok = product(0);
-    }
+    } else {
 #pragma unroll 1
     for (int i = 0; i < n; ++i) {
-        tcgen05_before_sync();
-        if (!__syncthreads_and(ok)) break;                     // accumulator (i + 1) & 1 has been read by everybody (tile i - 1)
-        tcgen05_after_sync();
-        if (tid == 0) {
-            // the next tile's product runs while this tile's accumulator is worked on; the stage of tile
-            // i - 1 is free (its product completed before its accumulator was read) and takes tile i + NST - 1
-            if (i + 1 < n) ok = product(i + 1);
-            if (i + NST - 1 < n) issue(i + NST - 1);
-        }
-        ok = mbar_wait(&bar[i & 1], (uint32_t)((i >> 1) & 1)) && ok;
+        ok = mbar_wait(&bar[i & 1], (uint32_t)((i >> 1) & 1));
+        if (!__all_sync(0xffffffffu, ok)) break;               // (a warp's lanes stay together: the accumulator loads are warp-wide)
         tcgen05_after_sync();
         const int64_t j0 = (int64_t)(t0 + i) * kMmaKeys;
         const uint32_t tl = tb + (uint32_t)(i & 1) * ACC + ((uint32_t)(warp * 32) << 16);    // this warp's lanes of the accumulator
@@ -344,16 +352,16 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
             }
             if (j < len) imp[(int64_t)bh * len + j] = acc;
         }
+        tcgen05_before_sync();
+        mbar_arrive(&acc_free[i & 1]);                         // this thread has read the accumulator
     }
-    // after a wait that ran out: no copy may still be on its way into this CTA's shared memory when it exits
-    if (tid == 0)
-        for (int k = n_landed; k < n_issued; ++k) mbar_wait(&full[k % NST], (uint32_t)((k / NST) & 1));
+    }
     if (__any_sync(0xffffffffu, !ok) && lane == 0) atomicCAS(status, RQ_OK, RQ_ERR_TIMEOUT);
     if (PASS == 1) {
         // the two halves of a query's keys, merged through shared memory
-        if (half == 1) qst[row] = make_float2(m, l);
+        if (warp < kMmaWarps && half == 1) qst[row] = make_float2(m, l);
         __syncthreads();
-        if (half == 0) {
+        if (warp < kMmaWarps && half == 0) {
             const float2 o = qst[row];
             const float mn = fmaxf(m, o.x);
             float lt = 0.0f;
