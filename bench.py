@@ -282,6 +282,36 @@ def parity_block(w, cache, sample_inputs, q, tok, K, T0, dev, recall_cache=None,
     return out
 
 
+def snapkv_block(w, cache, dev, peak):
+    """Times of the SnapKV-style reduction (App. A.1) of one of the timed caches, after the decode steps: window of
+    64 queries, 1/16 of the entries retained; median of five event-timed calls after two warm-up calls."""
+    import torch
+    import paper_2605_28640_b200 as rq
+    T = len(cache)
+    W, keep = 64, max(64, T // 16)
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed + 99)
+    qw = torch.randn(w.B, W, w.H, w.D, generator=g, device=dev, dtype=torch.float32).to(w.dtype)
+    idx = torch.empty(w.B, w.H, keep, dtype=torch.int32, device=dev)
+    scratch = torch.empty(rq.rq_snapkv_scratch_bytes(cache.handle), dtype=torch.uint8, device=dev)
+    small = rq.Cache(w.B, w.H, w.D, w.S, keep + 64, w.dtype, w.gdtype, device=dev)
+    sel = sorted(event_ms(lambda: rq.rq_snapkv_select(cache.handle, qw, W, keep, 0.0, idx, None, scratch)) for _ in range(7))[:5]
+    cmp_ = sorted(event_ms(lambda: rq.rq_snapkv_compact(cache.handle, idx, keep, small.handle)) for _ in range(7))[:5]
+    es = 2 if w.dtype == torch.bfloat16 else 4
+    key_bytes = 2 * w.B * w.H * T * w.D * es                   # the keys are read twice (statistics, then weights)
+    flops = 2 * 2.0 * W * w.D * T * w.B * w.H
+    move = 2 * 2 * w.B * w.H * keep * w.D * es                 # retained keys and values read and written
+    return {"window": W, "keep": keep, "tokens": T,
+            "select_ms": sel[2], "select_ms_min": sel[0], "select_key_bytes": key_bytes,
+            "select_gbs": key_bytes / (sel[2] * 1e-3) / 1e9, "select_frac_of_hbm_peak": key_bytes / (sel[2] * 1e-3) / 1e9 / peak,
+            "select_tflops": flops / (sel[2] * 1e-3) / 1e12,
+            "compact_ms": cmp_[2], "compact_ms_min": cmp_[0], "compact_bytes": move,
+            "compact_gbs": move / (cmp_[2] * 1e-3) / 1e9,
+            "status_ok": rq.rq_device_status(cache.handle) == rq.RQ_OK,
+            "note": "rq_snapkv_select = importance (two passes over the keys) + selection; rq_snapkv_compact = reset of the "
+                    "new cache + gather of the retained rows + page bounds + state"}
+
+
 # ------------------------------------------------------------------------- own arm
 def main():
     ap = argparse.ArgumentParser()
@@ -298,6 +328,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
     ap.add_argument("--no-parity", action="store_true")
+    ap.add_argument("--snapkv", action="store_true",
+                    help="also time the SnapKV-style reduction of the first cache (window 64, 1/16 of the entries retained)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "rq" else args.warmup
 
@@ -530,6 +562,8 @@ def main():
                            "gbs": pbytes / (pm * 1e-3) / 1e9, "frac_of_peak": pbytes / (pm * 1e-3) / 1e9 / peak,
                            "runs_ms": rebuild_ms[2:], "first_build_ms": first_build_ms,
                            "note": "median of five rebuilds (rq_cache_reset + rq_build_cache) after two warm-up rebuilds"}
+    if args.snapkv and first:
+        line["snapkv"] = snapkv_block(w, caches[0], dev, peak)
     if first and not args.no_cpu_baseline:
         nh = min(8, w.H)
         threads = min(os.cpu_count() or 1, nh)

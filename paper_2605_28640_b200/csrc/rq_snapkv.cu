@@ -506,41 +506,58 @@ __global__ void __launch_bounds__(1024) snap_select_kernel(const float *imp, int
 }
 
 // ---------------------------------------------------------------- compaction into the new cache
-// One CTA per (head, page of the new cache), a thread per channel.
+// One CTA of 256 threads per (head, page of the new cache).  The page's retained rows move in 16-byte
+// pieces, keys and values alike (a thread per piece, a row's pieces on neighbouring threads); the keys
+// also pass through shared memory, from which a thread per channel then takes the page's bounds.
+constexpr int kCompactThreads = 256;
+constexpr int kCompactSmem = 64 * 128 * 4;                 // the keys of one page at most: 64 slots x 128 channels x 4 bytes
+
 template <typename T>
-__global__ void snap_compact_kernel(const T *skv, int64_t s_page_cap, T *dkv, T *dmeta, int64_t d_page_cap, int S, int D,
-                                    const int32_t *idx, int keep, float *absmax, int BH)
+__global__ void __launch_bounds__(kCompactThreads) snap_compact_kernel(const T *skv, int64_t s_page_cap, T *dkv, T *dmeta,
+                                                                       int64_t d_page_cap, int S, int D, const int32_t *idx,
+                                                                       int keep, float *absmax, int BH)
 {
-    const int bh = blockIdx.y, page = blockIdx.x, d = threadIdx.x;
-    const int32_t *list = idx + (int64_t)bh * keep;
-    T *dpage = dkv + (((int64_t)bh * d_page_cap + page) * 2) * S * D;
-    float mn = CUDART_INF_F, mx = -CUDART_INF_F;
-    for (int s = 0; s < S; ++s) {
-        const int r = page * S + s;
-        T kq, vq;
-        if (r < keep) {
-            const int64_t pos = list[r];
-            const T *src = skv + ((((int64_t)bh * s_page_cap + pos / S) * 2) * S + pos % S) * D + d;
-            kq = src[0];
-            vq = src[(int64_t)S * D];
-            const float kf = load1<T>(&kq);
+    __shared__ __align__(16) unsigned char krows[kCompactSmem];
+    __shared__ int32_t src_pos[64];
+    const int bh = blockIdx.y, page = blockIdx.x, tid = threadIdx.x;
+    const int rb = D * (int)sizeof(T), ppr = rb / 16;        // bytes and 16-byte pieces of a row
+    const int rows = min(S, keep - page * S);                // retained rows of this page (at least one)
+    if (tid < S) src_pos[tid] = tid < rows ? idx[(int64_t)bh * keep + page * S + tid] : -1;
+    __syncthreads();
+    unsigned char *dpage = reinterpret_cast<unsigned char *>(dkv + (((int64_t)bh * d_page_cap + page) * 2) * S * D);
+    const unsigned char *shead = reinterpret_cast<const unsigned char *>(skv + (int64_t)bh * s_page_cap * 2 * S * D);
+    for (int i = tid; i < S * ppr; i += kCompactThreads) {
+        const int r = i / ppr, c = i % ppr;
+        uint4 kq = make_uint4(0u, 0u, 0u, 0u), vq = kq;      // unused slots of the last page are defined (zero)
+        if (r < rows) {
+            const int64_t pos = src_pos[r];
+            const unsigned char *src = shead + ((pos / S) * 2 * S + pos % S) * (int64_t)rb + c * 16;
+            kq = *reinterpret_cast<const uint4 *>(src);
+            vq = *reinterpret_cast<const uint4 *>(src + (int64_t)S * rb);
+        }
+        *reinterpret_cast<uint4 *>(dpage + (int64_t)r * rb + c * 16) = kq;
+        *reinterpret_cast<uint4 *>(dpage + (int64_t)(S + r) * rb + c * 16) = vq;
+        *reinterpret_cast<uint4 *>(krows + r * rb + c * 16) = kq;
+    }
+    __syncthreads();
+    float am = 0.0f;
+    if (tid < D) {
+        const T *kr = reinterpret_cast<const T *>(krows);
+        float mn = CUDART_INF_F, mx = -CUDART_INF_F;
+        for (int r = 0; r < rows; ++r) {
+            const float kf = load1<T>(kr + r * D + tid);
             mn = fminf(mn, kf);
             mx = fmaxf(mx, kf);
-        } else {
-            store1<T>(&kq, 0.0f);                    // unused slots of the last page are defined
-            store1<T>(&vq, 0.0f);
         }
-        dpage[(int64_t)s * D + d] = kq;
-        dpage[(int64_t)(S + s) * D + d] = vq;
+        T *mrow = dmeta + (((int64_t)bh * d_page_cap + page) * 2) * D;
+        store1<T>(mrow + tid, mn);
+        store1<T>(mrow + D + tid, mx);
+        am = fmaxf(-mn, mx);
     }
-    T *m = dmeta + (((int64_t)bh * d_page_cap + page) * 2) * D;
-    store1<T>(m + d, mn);
-    store1<T>(m + D + d, mx);
-    if (absmax) {
-        float am = fmaxf(-mn, mx);                   // the page holds at least one retained row
+    if (absmax && tid < D) {                                 // D is a multiple of 32: whole warps
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, off));
-        if ((d & 31) == 0) {
+        if ((tid & 31) == 0) {
             atomicMax(reinterpret_cast<unsigned *>(absmax) + bh, __float_as_uint(am));
             atomicMax(reinterpret_cast<unsigned *>(absmax) + BH + bh, __float_as_uint(am));
         }
@@ -688,10 +705,10 @@ cudaError_t launch_snap_compact(const void *skv, int64_t s_page_cap, void *dkv, 
 {
     const dim3 grid((unsigned)((keep + S - 1) / S), (unsigned)BH);
     if (dtype == RQ_BF16)
-        snap_compact_kernel<bf16><<<grid, D, 0, s>>>((const bf16 *)skv, s_page_cap, (bf16 *)dkv, (bf16 *)dmeta, d_page_cap, S, D, idx,
+        snap_compact_kernel<bf16><<<grid, kCompactThreads, 0, s>>>((const bf16 *)skv, s_page_cap, (bf16 *)dkv, (bf16 *)dmeta, d_page_cap, S, D, idx,
                                                      keep, absmax, BH);
     else
-        snap_compact_kernel<float><<<grid, D, 0, s>>>((const float *)skv, s_page_cap, (float *)dkv, (float *)dmeta, d_page_cap, S, D,
+        snap_compact_kernel<float><<<grid, kCompactThreads, 0, s>>>((const float *)skv, s_page_cap, (float *)dkv, (float *)dmeta, d_page_cap, S, D,
                                                       idx, keep, absmax, BH);
     return cudaGetLastError();
 }
