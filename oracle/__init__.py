@@ -25,7 +25,7 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile ``rqo.c`` into ``librqo.so`` next to it (gcc, -O2, strict IEEE)."""
-    srcs = [_SRC, os.path.join(_HERE, "rqo_snapkv.c")]
+    srcs = [_SRC, os.path.join(_HERE, "rqo_snapkv.c"), os.path.join(_HERE, "rqo_moba.c")]
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(f) for f in srcs):
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
                "-fno-fast-math", "-o", _LIB, *srcs, "-lm"]
@@ -89,6 +89,10 @@ def lib():
         L.rqo_snapkv_select.restype = C.c_int64
         L.rqo_token_attention.argtypes = [C.c_int64, _ip, C.c_int, _dp, C.c_double, _dp, _dp, _dp]
         L.rqo_token_attention.restype = None
+        L.rqo_block_means.argtypes = [C.c_int64, C.c_int, C.c_int64, _dp, _dp]
+        L.rqo_block_means.restype = None
+        L.rqo_moba_scores.argtypes = [C.c_int64, C.c_int, _dp, _dp, _dp]
+        L.rqo_moba_scores.restype = None
         _lib = L
     return _lib
 
@@ -182,6 +186,41 @@ def token_attention(q, scale, kst, vst, tok):
     y = np.empty(q.shape[0], np.float64)
     lib().rqo_token_attention(len(tok), tok.ctypes.data_as(_ip), q.shape[0], _d(q), float(scale), _d(kst), _d(vst), _d(y))
     return y
+
+
+def block_means(kst, block):
+    """App. A.1 (MoBA): mean-pooled representative of every block of `block` positions.  kst [T, D]."""
+    kst = _f64(kst)
+    T, D = kst.shape
+    means = np.empty(((T + block - 1) // block, D), np.float64)
+    lib().rqo_block_means(T, D, block, _d(kst), _d(means))
+    return means
+
+
+def moba_scores(q, means, n):
+    """Eq. 3's score of the first n blocks under query q: q . mean."""
+    q, means = _f64(q), _f64(means)
+    U = np.empty(n, np.float64)
+    lib().rqo_moba_scores(n, q.shape[0], _d(q), _d(means), _d(U))
+    return U
+
+
+def moba_route(q, means, t, block, K, n_sink=1, n_local=1):
+    """Blocks the query of position t attends (ascending) and the near-tie flag: the TopK of Eq. 3 over the
+    complete blocks before the query's own, the first block(s) and the own block always included, all inside K."""
+    bt = t // block
+    U = np.zeros(bt + 1)
+    if bt > 0:
+        U[:bt] = moba_scores(q, means, bt)
+    # the own block is the newest `page`: forced whatever its score (n_local >= 1), ranked last otherwise
+    U[bt] = -np.inf if n_local < 1 else 0.0
+    return select_pages(U, K, n_sink, n_local)
+
+
+def moba_attention(q, scale, kst, vst, blocks, t, block):
+    """Eq. 4 for the query of position t over the listed blocks: their tokens up to position t."""
+    tok = np.concatenate([np.arange(j * block, min((j + 1) * block, t + 1)) for j in blocks]) if len(blocks) else np.zeros(0, np.int64)
+    return token_attention(q, scale, kst, vst, tok)
 
 
 class Head:
