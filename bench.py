@@ -312,6 +312,39 @@ def snapkv_block(w, cache, dev, peak):
                     "new cache + gather of the retained rows + page bounds + state"}
 
 
+def moba_block(w, dev):
+    """Times of the MoBA-style block-sparse prefill attention (App. A.1) at the paper's setting: prompts of 4096 tokens,
+    block 64 and 128, budget 1/4 and 1/16, for the workload's batch, heads and head size; median of five event-timed calls."""
+    import dataclasses
+    import torch
+    import paper_2605_28640_b200 as rq
+    from paper_2605_28640_b200 import workloads as wl
+    T = 4096
+    wm = dataclasses.replace(w, T=T, needles=0, resets=False, name="moba-4k")
+    cache = rq.Cache(wm.B, wm.H, wm.D, wm.S, T, wm.dtype, wm.gdtype, device=dev)
+    k, v, g = wl.make_prefill(wm, dev, T)
+    rq.rq_build_cache(cache.handle, k, v, g)
+    del k, v, g
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed + 55)
+    q = torch.randn(wm.B, T, wm.H, wm.D, generator=gen, device=dev, dtype=torch.float32).to(wm.dtype)
+    o = torch.empty_like(q)
+    out = {"tokens": T, "batch": wm.B, "heads": wm.H, "runs": []}
+    for block, K in ((64, 16), (64, 4), (128, 8)):
+        scratch = torch.empty(rq.rq_moba_scratch_bytes(cache.handle, block, K), dtype=torch.uint8, device=dev)
+        ts = sorted(event_ms(lambda: rq.rq_moba_prefill(cache.handle, q, block, K, 0.0, o, None, None, scratch)) for _ in range(7))[:5]
+        # attended (query, key) pairs: K blocks per query (fewer for the first K blocks of queries), the own block half on average
+        nb = T // block
+        pairs = sum(min(K, t // block + 1) * block - (block - 1 - t % block) for t in range(T))
+        flops = 4.0 * pairs * wm.D * wm.B * wm.H
+        out["runs"].append({"block": block, "blocks_per_query": K, "ms": ts[2], "ms_min": ts[0],
+                            "attended_fraction": pairs / (T * (T + 1) / 2), "tflops_on_attended_pairs": flops / (ts[2] * 1e-3) / 1e12})
+        del scratch
+    out["status_ok"] = rq.rq_device_status(cache.handle) == rq.RQ_OK
+    out["note"] = "rq_moba_prefill = block means + routing of every query + attention over the chosen blocks (plain fp32 FMA kernels)"
+    return out
+
+
 # ------------------------------------------------------------------------- own arm
 def main():
     ap = argparse.ArgumentParser()
@@ -328,6 +361,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
     ap.add_argument("--no-parity", action="store_true")
+    ap.add_argument("--moba", action="store_true",
+                    help="also time the MoBA-style block-sparse prefill attention at the paper's setting (4K prompts, block 64, "
+                         "16 blocks per query) for the workload's batch and heads")
     ap.add_argument("--snapkv", action="store_true",
                     help="also time the SnapKV-style reduction of the first cache (window 64, 1/16 of the entries retained)")
     args = ap.parse_args()
@@ -564,6 +600,8 @@ def main():
                            "note": "median of five rebuilds (rq_cache_reset + rq_build_cache) after two warm-up rebuilds"}
     if args.snapkv and first:
         line["snapkv"] = snapkv_block(w, caches[0], dev, peak)
+    if args.moba and first:
+        line["moba"] = moba_block(w, dev)
     if first and not args.no_cpu_baseline:
         nh = min(8, w.H)
         threads = min(os.cpu_count() or 1, nh)

@@ -271,6 +271,26 @@ RQ_API int rq_snapkv_select(rq_cache *cache, const void *q_window, int32_t windo
  * Errors: INVALID_ARG (shapes differ, dst is src, keep outside 1..len), CAPACITY, CUDA. */
 RQ_API int rq_snapkv_compact(const rq_cache *src, const int32_t *idx, int32_t keep, rq_cache *dst, void *stream);
 
+/* MoBA-style block-sparse PREFILL attention over the cache the prompt was prefilled into [Sec. 2.2,
+ * Eq. 3 and Eq. 4, Table 1 row MoBA; App. A.1, "Sparse inference settings", MoBA paragraph]: the
+ * query of every prompt position t is routed to budget_blocks KV blocks of `block` positions: the
+ * complete blocks before its own are scored with their mean-pooled representatives (q . mean of the
+ * block's stored decayed keys) and the best are taken, equal scores to the lower block; the first
+ * block and the query's own block are always taken and count inside budget_blocks; with fewer
+ * blocks than that before it, a query attends everything before it.  Attention is softmax over the
+ * positions <= t of the chosen blocks, on the decayed keys and values as stored.
+ *   q          : [B][T][H][D] of cfg.dtype (device), T = the cache's current length
+ *   block      : 64, 128, ... (a multiple of 64 and of the page size); at most 2048 blocks per prompt
+ *   o          : [B][T][H][D] of cfg.dtype (device)
+ *   blocks_out : NULL or int32 [B][H][T][budget_blocks] (device): chosen blocks, ascending, -1 beyond
+ *   means_out  : NULL or fp32 [B][H][blocks][D] (device): the representatives
+ *   scratch    : device memory of rq_moba_scratch_bytes() bytes, 256-byte aligned
+ *   scale      : softmax scale; <= 0 selects 1/sqrt(D)
+ * Errors: INVALID_ARG (NULL, empty cache, block or budget_blocks < 2 out of range), CUDA. */
+RQ_API int rq_moba_scratch_bytes(const rq_cache *cache, int32_t block, int32_t budget_blocks, size_t *bytes);
+RQ_API int rq_moba_prefill(rq_cache *cache, const void *q, int32_t block, int32_t budget_blocks, float scale, void *o,
+                           int32_t *blocks_out, float *means_out, void *scratch, void *stream);
+
 /* Tokens in the cache (host bookkeeping; no CUDA call).  -1 for NULL. */
 RQ_API int64_t rq_cache_len(const rq_cache *cache);
 

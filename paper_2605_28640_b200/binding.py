@@ -52,6 +52,8 @@ SIGNATURES = {
     "rq_snapkv_scratch_bytes": (C.c_int, [_cachep, _szp]),
     "rq_snapkv_select": (C.c_int, [_cachep, _vp, _i32, _i32, _f, _vp, _vp, _vp, _vp]),
     "rq_snapkv_compact": (C.c_int, [_cachep, _vp, _i32, _cachep, _vp]),
+    "rq_moba_scratch_bytes": (C.c_int, [_cachep, _i32, _i32, _szp]),
+    "rq_moba_prefill": (C.c_int, [_cachep, _vp, _i32, _i32, _f, _vp, _vp, _vp, _vp, _vp]),
     "rq_cache_len": (C.c_int64, [_cachep]),
     "rq_decode_step_launches": (C.c_int, [_cachep, _i32]),
     "rq_device_status": (C.c_int, [_cachep, C.POINTER(C.c_int32), _vp]),
@@ -186,6 +188,17 @@ def rq_snapkv_select(cache: rq_cache, q_window, window, keep, scale, idx_out, im
 
 def rq_snapkv_compact(src: rq_cache, idx, keep, dst: rq_cache, stream=None):
     _check(lib().rq_snapkv_compact(C.byref(src), _ptr(idx), keep, C.byref(dst), _stream(stream)), "rq_snapkv_compact")
+
+
+def rq_moba_scratch_bytes(cache: rq_cache, block, budget_blocks) -> int:
+    n = C.c_size_t()
+    _check(lib().rq_moba_scratch_bytes(C.byref(cache), block, budget_blocks, C.byref(n)), "rq_moba_scratch_bytes")
+    return n.value
+
+
+def rq_moba_prefill(cache: rq_cache, q, block, budget_blocks, scale, o, blocks_out, means_out, scratch, stream=None):
+    _check(lib().rq_moba_prefill(C.byref(cache), _ptr(q), block, budget_blocks, scale, _ptr(o), _ptr(blocks_out),
+                                 _ptr(means_out), _ptr(scratch), _stream(stream)), "rq_moba_prefill")
 
 
 def rq_cache_len(cache: rq_cache) -> int:

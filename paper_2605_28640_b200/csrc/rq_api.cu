@@ -615,6 +615,48 @@ int rq_snapkv_compact(const rq_cache *src, const int32_t *idx, int32_t keep, rq_
     return RQ_OK;
 }
 
+static bool moba_shape_ok(const rq_cache *cache, int32_t block, int32_t budget_blocks)
+{
+    return cache->len >= 1 && block >= 64 && block % 64 == 0 && block % cache->cfg.page_size == 0 && budget_blocks >= 2 &&
+           (cache->len + block - 1) / block <= 2048;
+}
+
+int rq_moba_scratch_bytes(const rq_cache *cache, int32_t block, int32_t budget_blocks, size_t *bytes)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!bytes || !moba_shape_ok(cache, block, budget_blocks)) return RQ_ERR_INVALID_ARG;
+    *bytes = moba_scratch_bytes(cache->cfg.batch * cache->cfg.heads, cache->len, cache->cfg.head_dim, block, budget_blocks);
+    return RQ_OK;
+}
+
+int rq_moba_prefill(rq_cache *cache, const void *q, int32_t block, int32_t budget_blocks, float scale, void *o,
+                    int32_t *blocks_out, float *means_out, void *scratch, void *stream)
+{
+    const int rc = check_cache(cache);
+    if (rc != RQ_OK) return rc;
+    if (!q || !o || !scratch || !aligned(scratch, 256) || !aligned(q, 16) || !aligned(o, 16)) return RQ_ERR_INVALID_ARG;
+    if (!moba_shape_ok(cache, block, budget_blocks)) return RQ_ERR_INVALID_ARG;
+    const rq_config &c = cache->cfg;
+    cudaStream_t s = (cudaStream_t)stream;
+    MobaArgs a;
+    a.kv = cache->kv; a.page_cap = cache->page_capacity; a.len = cache->len;
+    a.B = c.batch; a.H = c.heads; a.D = c.head_dim; a.S = c.page_size; a.dtype = c.dtype;
+    a.q = q; a.block = block; a.K = budget_blocks; a.o = o;
+    a.scale = scale > 0.0f ? scale : 1.0f / sqrtf((float)c.head_dim);
+    const int BH = c.batch * c.heads;
+    moba_carve(scratch, BH, cache->len, c.head_dim, block, &a.means, &a.sel);
+    if (launch_moba(a, s) != cudaSuccess) return RQ_ERR_CUDA;
+    const size_t nb = (size_t)((cache->len + block - 1) / block);
+    if (blocks_out && cudaMemcpyAsync(blocks_out, a.sel, (size_t)BH * cache->len * budget_blocks * sizeof(int32_t),
+                                      cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    if (means_out && cudaMemcpyAsync(means_out, a.means, (size_t)BH * nb * c.head_dim * sizeof(float), cudaMemcpyDeviceToDevice,
+                                     s) != cudaSuccess)
+        return RQ_ERR_CUDA;
+    return RQ_OK;
+}
+
 int64_t rq_cache_len(const rq_cache *cache) { return cache ? cache->len : -1; }
 
 int rq_decode_step_launches(const rq_cache *cache, int32_t budget_pages)

@@ -157,6 +157,22 @@ cudaError_t launch_snap_select(const float *imp, int BH, int64_t len, int window
 cudaError_t launch_snap_compact(const void *skv, int64_t s_page_cap, void *dkv, void *dmeta, int64_t d_page_cap, int S, int D,
                                 int dtype, const int32_t *idx, int keep, float *absmax, int BH, cudaStream_t s);
 
+// ---- MoBA-style block-sparse prefill attention (rq_moba.cu) ----
+struct MobaArgs {
+    const void *kv;     // the cache the prompt was prefilled into
+    int64_t page_cap, len;
+    int B, H, D, S, dtype;
+    const void *q;      // [B][len][H][D] queries of all prompt positions
+    int block, K;       // block size in positions; blocks per query (first and own block included)
+    float scale;
+    float *means;       // [BH][blocks][D] block representatives
+    int32_t *sel;       // [BH][len][K] chosen blocks of every query, ascending, -1 beyond
+    void *o;            // [B][len][H][D]
+};
+size_t moba_scratch_bytes(int BH, int64_t len, int D, int block, int K);
+void moba_carve(void *scratch, int BH, int64_t len, int D, int block, float **means, int32_t **sel);
+cudaError_t launch_moba(const MobaArgs &a, cudaStream_t s);
+
 // Grid of a streaming kernel for a number of work units spread evenly over `heads` heads: at
 // most what the device holds at once, at least two units per warp, and a whole number of CTAs per
 // head if that keeps at least 85 % of the CTAs (heads served by more CTAs than others would
