@@ -646,6 +646,7 @@ int rq_moba_prefill(rq_cache *cache, const void *q, int32_t block, int32_t budge
     a.scale = scale > 0.0f ? scale : 1.0f / sqrtf((float)c.head_dim);
     const int BH = c.batch * c.heads;
     moba_carve(scratch, BH, cache->len, c.head_dim, block, &a.means, &a.sel);
+    a.status = (int32_t *)((char *)cache->workspace + workspace_layout(c).status);
     if (launch_moba(a, s) != cudaSuccess) return RQ_ERR_CUDA;
     const size_t nb = (size_t)((cache->len + block - 1) / block);
     if (blocks_out && cudaMemcpyAsync(blocks_out, a.sel, (size_t)BH * cache->len * budget_blocks * sizeof(int32_t),

@@ -168,6 +168,7 @@ struct MobaArgs {
     float *means;       // [BH][blocks][D] block representatives
     int32_t *sel;       // [BH][len][K] chosen blocks of every query, ascending, -1 beyond
     void *o;            // [B][len][H][D]
+    int32_t *status;    // the cache's device status word
 };
 size_t moba_scratch_bytes(int BH, int64_t len, int D, int block, int K);
 void moba_carve(void *scratch, int BH, int64_t len, int D, int block, float **means, int32_t **sel);

@@ -24,6 +24,8 @@
 #include "rq_device.cuh"
 #include "rq_internal.h"
 #include "rq_stream.cuh"
+#include "rq_tmap.h"
+#include "rq_umma.cuh"
 
 namespace rq {
 
@@ -259,6 +261,308 @@ __global__ void __launch_bounds__(kMobaQueries * 32) moba_attend_kernel(const T 
     }
 }
 
+// ---------------------------------------------------------------- attention on the tensor cores (bf16 caches)
+// Grid (ceil(T / 128), heads).  A CTA owns 128 consecutive queries of a head: they are the 128 lanes of the
+// accumulators, so everything per query (mask, running maximum, sum, weights) is per thread.  The chunks
+// (64 positions) of the blocks ANY of the 128 queries chose are walked twice:
+//   pass 1   S = Q K^T (tcgen05.mma, 128 x 64, fp32 in tensor memory); a thread masks the chunk for its query
+//            (block not chosen / positions after the query) and keeps the running maximum and sum of exponentials
+//   pass 2   S again; the thread turns its row into normalised weights, rounds them to bf16 and writes them
+//            into shared memory as the K-major operand of the second product, O += P V (128 x D, the values as an
+//            MN-major operand straight from the cache's rows), accumulated in tensor memory over all chunks
+// One thread of a fifth warp starts the tensor-map copies (keys and values of a chunk, four stages each) and the
+// products; the four other warps read the accumulators.  They meet only through mbarriers; every wait is bounded.
+constexpr int kMobaMmaQueries = 128;
+constexpr int kMobaMmaWarps = 4;
+constexpr int kMobaMmaThreads = (kMobaMmaWarps + 1) * 32;
+constexpr int kMobaMmaStages = 4;
+
+template <int D>
+struct MobaMmaGeom {
+    static constexpr int HALVES = D / 64;
+    static constexpr int Q_BYTES = HALVES * 128 * 128;             // 128 queries
+    static constexpr int KC_BYTES = HALVES * kMobaChunk * 128;     // the keys (or the values) of a chunk
+    static constexpr int P_BYTES = 128 * 128;                      // weights: 128 queries x 64 positions, bf16
+    static constexpr int OFF_K = Q_BYTES;
+    static constexpr int OFF_V = OFF_K + kMobaMmaStages * KC_BYTES;
+    static constexpr int OFF_P = OFF_V + kMobaMmaStages * KC_BYTES;
+    static constexpr int OFF_MASK = OFF_P + 2 * P_BYTES;
+    static constexpr int FIXED_BYTES = OFF_MASK + 1024;            // + room to align the base to 1024 bytes
+};
+
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t saddr, uint32_t lbo_bytes)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+__device__ __forceinline__ float exp2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float a, float b)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_constant__ CUtensorMap tmap, int64_t page_cap, int S,
+                                                                  int64_t len, const bf16 *q, int H, int block, int nb, int K,
+                                                                  const int32_t *sel, float scale_log2, bf16 *o, int32_t *status)
+{
+    using G = MobaMmaGeom<D>;
+    constexpr int NST = kMobaMmaStages;
+    constexpr uint32_t ACC_S = 64, OFF_O = 128, TCOLS = 256;   // two score accumulators of 64 columns, the output from column 128
+    extern __shared__ __align__(1024) unsigned char msm_raw[];
+    __shared__ __align__(8) uint64_t full_k[NST], full_v[NST], s_ready[2], s_free[2], p_ready[2], pv_done[2];
+    __shared__ uint32_t tbase;
+    unsigned char *msm = msm_raw + ((1024u - (smem_addr(msm_raw) & 1023u)) & 1023u);
+    unsigned char *qs = msm, *kst = msm + G::OFF_K, *vst = msm + G::OFF_V, *ps = msm + G::OFF_P;
+    const int words = (nb + 31) / 32;
+    uint32_t *umask = reinterpret_cast<uint32_t *>(msm + G::OFF_MASK);   // blocks chosen by any query of the CTA
+    uint32_t *qmask = umask + words;                                     // [128][words] blocks chosen by each query
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int64_t t0 = (int64_t)blockIdx.x * kMobaMmaQueries;
+    const int64_t tq = t0 + tid;                                         // this thread's query (threads 0 .. 127)
+    // chunks of 64 positions up to the CTA's last query; chunk c belongs to block c * 64 / block
+    const int n_chunks_all = (int)((min(t0 + kMobaMmaQueries, len) + kMobaChunk - 1) / kMobaChunk);
+
+    if (tid == 0) {
+        for (int s = 0; s < NST; ++s) { mbar_init(&full_k[s], 1); mbar_init(&full_v[s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&s_ready[s], 1);
+            mbar_init(&pv_done[s], 1);
+            mbar_init(&s_free[s], kMobaMmaWarps * 32);
+            mbar_init(&p_ready[s], kMobaMmaWarps * 32);
+        }
+        mbar_init_fence();
+    }
+    if (warp == 0) tmem_alloc(&tbase, TCOLS);
+    for (int i = tid; i < words * (kMobaMmaQueries + 1); i += kMobaMmaThreads) umask[i] = 0u;
+    // the queries (q is [B][T][H][D]) as the K-major operand; rows past the prompt are zero
+    for (int i = tid; i < 128 * (D / 8); i += kMobaMmaThreads) {
+        const int r = i / (D / 8), c = i % (D / 8);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (t0 + r < len) v = *reinterpret_cast<const uint4 *>(q + (((int64_t)b * len + t0 + r) * H + h) * D + c * 8);
+        *reinterpret_cast<uint4 *>(qs + (c >> 3) * (128 * 128) + umma_sw128_offset(r, c & 7)) = v;
+    }
+    __syncthreads();
+    if (tid < kMobaMmaQueries && tq < len) {
+        const int32_t *list = sel + ((int64_t)bh * len + tq) * K;
+        for (int i = 0; i < K; ++i) {
+            const int j = list[i];
+            if (j >= 0 && j < nb) {
+                qmask[tid * words + (j >> 5)] |= 1u << (j & 31);
+                atomicOr(&umask[j >> 5], 1u << (j & 31));
+            }
+        }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the queries, written with ordinary stores, are read by the tensor core
+    tcgen05_before_sync();
+    __syncthreads();
+    tcgen05_after_sync();
+    const uint32_t tb = tbase;
+    // number of chunks the CTA walks in one pass
+    int n = 0;
+    for (int c = 0; c < n_chunks_all; ++c) {
+        const int j = (int)(((int64_t)c * kMobaChunk) / block);
+        n += (umask[j >> 5] >> (j & 31)) & 1u;
+    }
+    // the chunk after `c` that belongs to a chosen block (the walk of both roles)
+    auto next_chunk = [&](int c) {
+        for (++c; c < n_chunks_all; ++c) {
+            const int j = (int)(((int64_t)c * kMobaChunk) / block);
+            if ((umask[j >> 5] >> (j & 31)) & 1u) break;
+        }
+        return c;
+    };
+    bool ok = true;
+
+    if (warp == kMobaMmaWarps) {
+        if (lane == 0) {
+            // ---- copies and products.  g counts the score products over both passes (0 .. 2n-1), hh the chunks of pass 2.
+            int ck_issue = -1, cv_issue = -1;        // chunk walk of the key copies (both passes) and of the value copies
+            int gk_issued = 0, hv_issued = 0, gk_landed = 0, hv_landed = 0;
+            auto issue_k = [&]() {                   // keys of the next chunk of the walk into stage gk_issued % NST
+                ck_issue = next_chunk(ck_issue);
+                if (ck_issue >= n_chunks_all) ck_issue = next_chunk(-1);      // pass 2 walks the same chunks again
+                const int st = gk_issued % NST;
+                const int page = (int)((int64_t)bh * page_cap + ((int64_t)ck_issue * kMobaChunk) / S);
+                mbar_arrive_expect_tx(&full_k[st], G::KC_BYTES);
+#pragma unroll
+                for (int hf = 0; hf < G::HALVES; ++hf)
+                    tma_load_4d(kst + (size_t)st * G::KC_BYTES + hf * (kMobaChunk * 128), &tmap, hf * 64, 0, 0, page, &full_k[st]);
+                ++gk_issued;
+            };
+            auto issue_v = [&]() {
+                cv_issue = next_chunk(cv_issue);
+                const int st = hv_issued % NST;
+                const int page = (int)((int64_t)bh * page_cap + ((int64_t)cv_issue * kMobaChunk) / S);
+                mbar_arrive_expect_tx(&full_v[st], G::KC_BYTES);
+#pragma unroll
+                for (int hf = 0; hf < G::HALVES; ++hf)
+                    tma_load_4d(vst + (size_t)st * G::KC_BYTES + hf * (kMobaChunk * 128), &tmap, hf * 64, 0, 1, page, &full_v[st]);
+                ++hv_issued;
+            };
+            auto product_pv = [&](int hh) -> bool {  // O += P(hh) V(hh)
+                if (!mbar_wait(&p_ready[hh & 1], (uint32_t)((hh >> 1) & 1))) return false;
+                if (!mbar_wait(&full_v[hh % NST], (uint32_t)((hh / NST) & 1))) return false;
+                hv_landed = hh + 1;
+                tcgen05_after_sync();
+                constexpr uint32_t idesc = umma_idesc_bf16(128, D) | (1u << 16);       // the values are MN-major
+                const uint32_t pa = smem_addr(ps + (size_t)(hh & 1) * G::P_BYTES), va = smem_addr(vst + (size_t)(hh % NST) * G::KC_BYTES);
+#pragma unroll
+                for (int k = 0; k < kMobaChunk / 16; ++k)
+                    umma_bf16(tb + OFF_O, umma_desc_sw128(pa + k * 32), umma_desc_sw128_mn(va + k * 2048, kMobaChunk * 128), idesc,
+                              (hh > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&pv_done[hh & 1]);
+                return true;
+            };
+            for (int s = 0; s < NST && s < 2 * n; ++s) issue_k();
+            for (int s = 0; s < NST && s < n; ++s) issue_v();
+            constexpr uint32_t idesc_s = umma_idesc_bf16(128, kMobaChunk);
+            const uint32_t qa = smem_addr(qs);
+#pragma unroll 1
+            for (int g = 0; g < 2 * n && ok; ++g) {
+                if (g >= 2) ok = mbar_wait(&s_free[g & 1], (uint32_t)(((g >> 1) - 1) & 1));
+                ok = ok && mbar_wait(&full_k[g % NST], (uint32_t)((g / NST) & 1));
+                if (!ok) break;
+                gk_landed = g + 1;
+                tcgen05_after_sync();
+                const uint32_t ka = smem_addr(kst + (size_t)(g % NST) * G::KC_BYTES);
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k)
+                    umma_bf16(tb + (uint32_t)(g & 1) * ACC_S, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
+                              umma_desc_sw128(ka + (k >> 2) * (kMobaChunk * 128) + (k & 3) * 32), idesc_s, k > 0);
+                umma_commit(&s_ready[g & 1]);
+                const int hh = g - n;                // pass 2: the chunk whose scores were just started
+                if (hh >= 1) ok = product_pv(hh - 1);
+                // refills: the key stage of product g - 1 once that product is complete, the value stage of chunk hh - 2 likewise
+                if (ok && g >= 1 && g - 1 + NST < 2 * n) {
+                    ok = mbar_wait(&s_ready[(g - 1) & 1], (uint32_t)(((g - 1) >> 1) & 1));
+                    if (ok) issue_k();
+                }
+                if (ok && hh >= 2 && hh - 2 + NST < n) {
+                    ok = mbar_wait(&pv_done[(hh - 2) & 1], (uint32_t)(((hh - 2) >> 1) & 1));
+                    if (ok) issue_v();
+                }
+            }
+            if (ok) ok = product_pv(n - 1);
+            // after a wait that ran out: no copy may still be on its way into this CTA's shared memory when it exits
+            for (int k = gk_landed; k < gk_issued; ++k) mbar_wait(&full_k[k % NST], (uint32_t)((k / NST) & 1));
+            for (int k = hv_landed; k < hv_issued; ++k) mbar_wait(&full_v[k % NST], (uint32_t)((k / NST) & 1));
+        }
+    } else {
+        // ---- the four warps that read the accumulators: thread = query
+        const uint32_t tl = tb + ((uint32_t)(warp * 32) << 16);
+        const uint32_t *mymask = qmask + tid * words;
+        float m = -CUDART_INF_F, l = 0.0f, inv_l = 0.0f;
+        int c = -1;
+#pragma unroll 1
+        for (int g = 0; g < 2 * n; ++g) {
+            if (g == n) {                            // pass 2 walks the same chunks again
+                c = -1;
+                inv_l = l > 0.0f ? 1.0f / l : 0.0f;
+            }
+            c = next_chunk(c);
+            const int64_t p0 = (int64_t)c * kMobaChunk;
+            const int j = (int)(p0 / block);
+            // positions of the chunk this query attends: none if it did not choose the block, else those up to its own
+            int nv = 0;
+            if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)kMobaChunk, tq - p0 + 1));
+            ok = mbar_wait(&s_ready[g & 1], (uint32_t)((g >> 1) & 1));
+            if (!__all_sync(FULLMASK, ok)) break;
+            tcgen05_after_sync();
+            const int hh = g - n;
+            if (hh >= 2) {                           // the weights buffer hh & 1 was read by the product of chunk hh - 2
+                ok = mbar_wait(&pv_done[hh & 1], (uint32_t)(((hh - 2) >> 1) & 1));
+                if (!__all_sync(FULLMASK, ok)) break;
+            }
+#pragma unroll 1
+            for (int cb = 0; cb < kMobaChunk; cb += 32) {
+                float v[32];
+                tmem_ld32(tl + (uint32_t)(g & 1) * ACC_S + (uint32_t)cb, v);
+                if (hh < 0) {
+                    if (cb < nv) {
+                        float tm = -CUDART_INF_F;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            v[i] = cb + i < nv ? v[i] * scale_log2 : -CUDART_INF_F;
+                            tm = fmaxf(tm, v[i]);
+                        }
+                        const float mn = fmaxf(m, tm);
+                        float sum = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) sum += exp2_fast(v[i] - mn);
+                        l = l * exp2_fast(m - mn) + sum;
+                        m = mn;
+                    }
+                } else {
+                    // normalised weights of 32 positions, rounded to bf16: four 16-byte pieces of this query's row
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float a = cb + i < nv ? exp2_fast(fmaf(v[i], scale_log2, -m)) * inv_l : 0.0f;
+                        const float bq = cb + i + 1 < nv ? exp2_fast(fmaf(v[i + 1], scale_log2, -m)) * inv_l : 0.0f;
+                        w[i >> 1] = pack2_bf16(a, bq);
+                    }
+                    unsigned char *prow = ps + (size_t)(hh & 1) * G::P_BYTES;
+#pragma unroll
+                    for (int pc = 0; pc < 4; ++pc)
+                        *reinterpret_cast<uint4 *>(prow + umma_sw128_offset(tid, cb / 8 + pc)) =
+                            make_uint4(w[4 * pc], w[4 * pc + 1], w[4 * pc + 2], w[4 * pc + 3]);
+                }
+            }
+            tcgen05_before_sync();
+            mbar_arrive(&s_free[g & 1]);             // this thread has read the scores
+            if (hh >= 0 && p0 + kMobaChunk > len) {
+                // the prompt ends inside this chunk: the value rows past its end hold whatever the cache's memory held;
+                // a weight of zero would not stop a NaN there, so those rows are cleared once they have landed
+                ok = mbar_wait(&full_v[hh % NST], (uint32_t)((hh / NST) & 1));
+                if (!__all_sync(FULLMASK, ok)) break;
+                const int r = tid & (kMobaChunk - 1), hf = tid >> 6;
+                if (hf < G::HALVES && p0 + r >= len) {
+                    uint4 *row = reinterpret_cast<uint4 *>(vst + (size_t)(hh % NST) * G::KC_BYTES + hf * (kMobaChunk * 128) + (r >> 3) * 1024 +
+                                                           (r & 7) * 128);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) row[i] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            if (hh >= 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the weights are read by the tensor core
+                mbar_arrive(&p_ready[hh & 1]);
+            }
+        }
+        // the output once the last product is complete
+        if (__all_sync(FULLMASK, ok)) {
+            ok = mbar_wait(&pv_done[(n - 1) & 1], (uint32_t)(((n - 1) >> 1) & 1));
+            if (__all_sync(FULLMASK, ok)) {
+                tcgen05_after_sync();
+#pragma unroll 1
+                for (int cb = 0; cb < D; cb += 32) {
+                    float v[32];
+                    tmem_ld32(tl + OFF_O + (uint32_t)cb, v);
+                    if (tq < len) {
+                        bf16 *orow = o + (((int64_t)b * len + tq) * H + h) * D + cb;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 8)
+                            *reinterpret_cast<uint4 *>(orow + i) = make_uint4(pack2_bf16(v[i], v[i + 1]), pack2_bf16(v[i + 2], v[i + 3]),
+                                                                              pack2_bf16(v[i + 4], v[i + 5]), pack2_bf16(v[i + 6], v[i + 7]));
+                    }
+                }
+            }
+        }
+    }
+    if (__any_sync(FULLMASK, !ok) && lane == 0) atomicCAS(status, RQ_OK, RQ_ERR_TIMEOUT);
+    tcgen05_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, TCOLS);
+}
+
 size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 template <typename T, int D>
@@ -289,8 +593,26 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
     moba_route_kernel<T, D><<<dim3((unsigned)((a.len + kMobaRouteWarps - 1) / kMobaRouteWarps), (unsigned)BH), kMobaRouteWarps * 32, rs,
                               s>>>((const T *)a.q, a.means, a.len, a.H, a.block, nb, a.K, a.sel);
     const float sl2 = a.scale * 1.4426950408889634f;
-    moba_attend_kernel<T, D><<<dim3((unsigned)((a.len + kMobaQueries - 1) / kMobaQueries), (unsigned)BH), kMobaQueries * 32, as, s>>>(
-        (const T *)a.kv, a.page_cap, a.S, a.len, (const T *)a.q, a.H, a.block, nb, a.K, a.sel, sl2, (T *)a.o);
+    if constexpr (sizeof(T) == 2) {
+        // bf16 caches: the attention on the tensor cores
+        using G = MobaMmaGeom<D>;
+        const size_t ms = (size_t)G::FIXED_BYTES + (size_t)words * (kMobaMmaQueries + 1) * sizeof(uint32_t);
+        static bool mready[64];
+        if (!mready[dev]) {
+            e = cudaFuncSetAttribute(moba_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)((size_t)G::FIXED_BYTES + (size_t)(kMobaMaxBlocks / 32) * (kMobaMmaQueries + 1) * sizeof(uint32_t)));
+            if (e != cudaSuccess) return e;
+            mready[dev] = true;
+        }
+        alignas(64) CUtensorMap tmap;
+        e = cache_tensor_map(&tmap, a.kv, D, a.S, (int64_t)BH * a.page_cap, kMobaChunk);
+        if (e != cudaSuccess) return e;
+        moba_mma_kernel<D><<<dim3((unsigned)((a.len + kMobaMmaQueries - 1) / kMobaMmaQueries), (unsigned)BH), kMobaMmaThreads, ms, s>>>(
+            tmap, a.page_cap, a.S, a.len, (const bf16 *)a.q, a.H, a.block, nb, a.K, a.sel, sl2, (bf16 *)a.o, a.status);
+    } else {
+        moba_attend_kernel<T, D><<<dim3((unsigned)((a.len + kMobaQueries - 1) / kMobaQueries), (unsigned)BH), kMobaQueries * 32, as, s>>>(
+            (const T *)a.kv, a.page_cap, a.S, a.len, (const T *)a.q, a.H, a.block, nb, a.K, a.sel, sl2, (T *)a.o);
+    }
     return cudaGetLastError();
 }
 

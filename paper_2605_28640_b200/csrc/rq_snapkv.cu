@@ -29,13 +29,13 @@
 //                             written in ascending order
 //   snap_compact_kernel       per (head, page of the new cache): gathers the retained rows, rebuilds
 //                             the page's min/max bounds, tracks the head's largest |key|
-#include <cuda.h>
 #include <math.h>
 #include <math_constants.h>
 
 #include "rq_async.cuh"
 #include "rq_device.cuh"
 #include "rq_internal.h"
+#include "rq_tmap.h"
 #include "rq_umma.cuh"
 
 namespace rq {
@@ -593,23 +593,6 @@ cudaError_t snap_scores_t(const SnapArgs &a, cudaStream_t s)
     return cudaGetLastError();
 }
 
-// The driver's tensor-map encoder, looked up once through the runtime (the library does not link the driver).
-typedef CUresult (*TensorMapEncodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                         const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                         CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-TensorMapEncodeTiled tensor_map_encoder()
-{
-    static TensorMapEncodeTiled fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = (TensorMapEncodeTiled)p;
-    }
-    return fn;
-}
-
 template <int D>
 cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
 {
@@ -628,17 +611,9 @@ cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
     }
     const int BH = a.B * a.H;
     if (kMmaKeys % a.S != 0) return cudaErrorInvalidValue;
-    // the cache [BH][page][key / value][slot][channel] as a rank-4 tensor, pages of all heads in one dimension
-    const TensorMapEncodeTiled encode = tensor_map_encoder();
-    if (!encode) return cudaErrorNotSupported;
     alignas(64) CUtensorMap tmap;
-    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)a.S, 2, (cuuint64_t)BH * (cuuint64_t)a.page_cap};
-    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)a.S * D * 2, (cuuint64_t)2 * a.S * D * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)a.S, 1, (cuuint32_t)(kMmaKeys / a.S)}, steps[4] = {1, 1, 1, 1};
-    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(a.kv), dims, strides, box, steps,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
+    e = cache_tensor_map(&tmap, a.kv, D, a.S, (int64_t)BH * a.page_cap, kMmaKeys);
+    if (e != cudaSuccess) return e;
     const int ntiles = (int)((a.len + kMmaKeys - 1) / kMmaKeys);
     // tiles per CTA: as many as leave a couple of CTAs for every SM
     int tpc = kMmaMaxTiles;
