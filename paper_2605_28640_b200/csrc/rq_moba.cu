@@ -62,21 +62,40 @@ __global__ void moba_means_kernel(const T *kv, int64_t page_cap, int S, int D, i
 
 // ---------------------------------------------------------------- routing
 // Grid (ceil(T / 8), heads); a warp per query.  Shared memory per warp: the query (D floats), the
-// scores of the candidate blocks (nb floats), the chosen blocks as a bit mask (nb / 32 words).
+// scores of the candidate blocks (nb floats), the chosen blocks as a bit mask (nb / 32 words); and,
+// when they fit (STAGED), the head's representatives for the whole CTA, rows padded by four floats so
+// that the lanes of a quarter-warp, each reading its own row, hit different banks.
 // q: [B][T][H][D].  sel: [BH][T][K], ascending, -1 beyond the chosen blocks.
-template <typename T, int D>
+constexpr int kMobaStagedBlocks = 128;         // representatives of up to this many blocks are staged in shared memory
+
+template <typename T, int D, bool STAGED>
 __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const T *q, const float *means, int64_t len, int H,
                                                                          int block, int nb, int K, int32_t *sel)
 {
     extern __shared__ __align__(16) float rsm[];
+    constexpr int LDM = STAGED ? D + 4 : D;            // floats from one representative to the next
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int words = (nb + 31) / 32;
     float *qs = rsm + (size_t)warp * moba_route_floats(D, nb);
     float *sc = qs + D;
     uint32_t *mask = reinterpret_cast<uint32_t *>(sc + nb);
+    const int bh = blockIdx.y;
+    const float *mh = means + (int64_t)bh * nb * D;
+    if (STAGED) {
+        // the representatives the CTA's queries can need: blocks before the last query's own
+        float *ms = rsm + (size_t)kMobaRouteWarps * moba_route_floats(D, nb);
+        const int64_t t_last = min((int64_t)blockIdx.x * kMobaRouteWarps + kMobaRouteWarps - 1, len - 1);
+        const int need = (int)(t_last / block);
+        for (int i = threadIdx.x; i < need * (D / 4); i += kMobaRouteWarps * 32) {
+            const int j = i / (D / 4), c = i % (D / 4);
+            *reinterpret_cast<float4 *>(ms + j * LDM + 4 * c) = __ldg(reinterpret_cast<const float4 *>(mh + (int64_t)j * D) + c);
+        }
+        __syncthreads();
+        mh = ms;
+    }
     const int64_t t = (int64_t)blockIdx.x * kMobaRouteWarps + warp;
     if (t >= len) return;                              // (no CTA-wide barrier below)
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int b = bh / H, h = bh % H;
     int32_t *out = sel + ((int64_t)bh * len + t) * K;
     const int bt = (int)(t / block), P = bt + 1;       // the query's own block; blocks it may attend
     if (K >= P) {                                      // everything before the query
@@ -90,15 +109,14 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
     for (int i = lane; i < words; i += 32) mask[i] = 0u;
     __syncwarp();
     // scores: a lane per block, the block's representative read as 16-byte pieces
-    const float *mh = means + (int64_t)bh * nb * D;
     for (int j0 = c_lo; j0 < c_hi; j0 += 32) {
         const int j = j0 + lane;
         if (j < c_hi) {
-            const float4 *row = reinterpret_cast<const float4 *>(mh + (int64_t)j * D);
+            const float4 *row = reinterpret_cast<const float4 *>(mh + (int64_t)j * LDM);
             float s = 0.0f;
 #pragma unroll 8
             for (int i = 0; i < D / 4; ++i) {
-                const float4 m4 = __ldg(row + i);
+                const float4 m4 = STAGED ? row[i] : __ldg(row + i);
                 const float4 q4 = *reinterpret_cast<const float4 *>(qs + 4 * i);
                 s = fmaf(q4.x, m4.x, s);
                 s = fmaf(q4.y, m4.y, s);
@@ -268,12 +286,12 @@ __global__ void __launch_bounds__(kMobaQueries * 32) moba_attend_kernel(const T 
 //   pass 1   S = Q K^T (tcgen05.mma, 128 x 64, fp32 in tensor memory); a thread masks the chunk for its query
 //            (block not chosen / positions after the query) and keeps the running maximum and sum of exponentials
 //   pass 2   S again; the thread turns its row into normalised weights, rounds them to bf16 and writes them
-//            into shared memory as the K-major operand of the second product, O += P V (128 x D, the values as an
-//            MN-major operand straight from the cache's rows), accumulated in tensor memory over all chunks
-// One thread of a fifth warp starts the tensor-map copies (keys and values of a chunk, four stages each) and the
-// products; the four other warps read the accumulators.  They meet only through mbarriers; every wait is bounded.
+//            into tensor memory (tcgen05.st) as the A operand of the second product, O += P V (128 x D, the values
+//            as an MN-major operand straight from the cache's rows), accumulated in tensor memory over all chunks
+// One thread of a ninth warp starts the tensor-map copies (keys and values of a chunk, four stages each) and the
+// products; the eight other warps read the accumulators (two per query, half of a chunk's positions each).  They meet only through mbarriers; every wait is bounded.
 constexpr int kMobaMmaQueries = 128;
-constexpr int kMobaMmaWarps = 4;
+constexpr int kMobaMmaWarps = 8;               // warps that read the accumulators: two per 32 lanes, half of the columns each
 constexpr int kMobaMmaThreads = (kMobaMmaWarps + 1) * 32;
 constexpr int kMobaMmaStages = 4;
 
@@ -282,11 +300,9 @@ struct MobaMmaGeom {
     static constexpr int HALVES = D / 64;
     static constexpr int Q_BYTES = HALVES * 128 * 128;             // 128 queries
     static constexpr int KC_BYTES = HALVES * kMobaChunk * 128;     // the keys (or the values) of a chunk
-    static constexpr int P_BYTES = 128 * 128;                      // weights: 128 queries x 64 positions, bf16
     static constexpr int OFF_K = Q_BYTES;
     static constexpr int OFF_V = OFF_K + kMobaMmaStages * KC_BYTES;
-    static constexpr int OFF_P = OFF_V + kMobaMmaStages * KC_BYTES;
-    static constexpr int OFF_MASK = OFF_P + 2 * P_BYTES;
+    static constexpr int OFF_MASK = OFF_V + kMobaMmaStages * KC_BYTES;
     static constexpr int FIXED_BYTES = OFF_MASK + 1024;            // + room to align the base to 1024 bytes
 };
 
@@ -314,12 +330,15 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
 {
     using G = MobaMmaGeom<D>;
     constexpr int NST = kMobaMmaStages;
-    constexpr uint32_t ACC_S = 64, OFF_O = 128, TCOLS = 256;   // two score accumulators of 64 columns, the output from column 128
+    // tensor memory: two score accumulators of 64 columns, the output (D columns) from column 128, then two weight
+    // buffers of 32 columns (64 positions as bf16 pairs); allocations are powers of two
+    constexpr uint32_t ACC_S = 64, OFF_O = 128, OFF_P = 128 + D, P_COLS = 32, TCOLS = D == 128 ? 512 : 256;
     extern __shared__ __align__(1024) unsigned char msm_raw[];
-    __shared__ __align__(8) uint64_t full_k[NST], full_v[NST], s_ready[2], s_free[2], p_ready[2], pv_done[2];
+    __shared__ __align__(8) uint64_t full_k[NST], full_v[NST], s_ready[2], s_free[2], p_ready[2], pv_done[2], stat_ready;
+    __shared__ float2 stat[2][kMobaMmaQueries];                          // pass 1: a query's statistics from its two threads
     __shared__ uint32_t tbase;
     unsigned char *msm = msm_raw + ((1024u - (smem_addr(msm_raw) & 1023u)) & 1023u);
-    unsigned char *qs = msm, *kst = msm + G::OFF_K, *vst = msm + G::OFF_V, *ps = msm + G::OFF_P;
+    unsigned char *qs = msm, *kst = msm + G::OFF_K, *vst = msm + G::OFF_V;
     const int words = (nb + 31) / 32;
     uint32_t *umask = reinterpret_cast<uint32_t *>(msm + G::OFF_MASK);   // blocks chosen by any query of the CTA
     uint32_t *qmask = umask + words;                                     // [128][words] blocks chosen by each query
@@ -327,7 +346,6 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int64_t t0 = (int64_t)blockIdx.x * kMobaMmaQueries;
-    const int64_t tq = t0 + tid;                                         // this thread's query (threads 0 .. 127)
     // chunks of 64 positions up to the CTA's last query; chunk c belongs to block c * 64 / block
     const int n_chunks_all = (int)((min(t0 + kMobaMmaQueries, len) + kMobaChunk - 1) / kMobaChunk);
 
@@ -339,6 +357,7 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             mbar_init(&s_free[s], kMobaMmaWarps * 32);
             mbar_init(&p_ready[s], kMobaMmaWarps * 32);
         }
+        mbar_init(&stat_ready, kMobaMmaWarps * 32);
         mbar_init_fence();
     }
     if (warp == 0) tmem_alloc(&tbase, TCOLS);
@@ -351,8 +370,8 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
         *reinterpret_cast<uint4 *>(qs + (c >> 3) * (128 * 128) + umma_sw128_offset(r, c & 7)) = v;
     }
     __syncthreads();
-    if (tid < kMobaMmaQueries && tq < len) {
-        const int32_t *list = sel + ((int64_t)bh * len + tq) * K;
+    if (tid < kMobaMmaQueries && t0 + tid < len) {
+        const int32_t *list = sel + ((int64_t)bh * len + t0 + tid) * K;
         for (int i = 0; i < K; ++i) {
             const int j = list[i];
             if (j >= 0 && j < nb) {
@@ -414,11 +433,11 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 hv_landed = hh + 1;
                 tcgen05_after_sync();
                 constexpr uint32_t idesc = umma_idesc_bf16(128, D) | (1u << 16);       // the values are MN-major
-                const uint32_t pa = smem_addr(ps + (size_t)(hh & 1) * G::P_BYTES), va = smem_addr(vst + (size_t)(hh % NST) * G::KC_BYTES);
+                const uint32_t pa = tb + OFF_P + (uint32_t)(hh & 1) * P_COLS, va = smem_addr(vst + (size_t)(hh % NST) * G::KC_BYTES);
 #pragma unroll
                 for (int k = 0; k < kMobaChunk / 16; ++k)
-                    umma_bf16(tb + OFF_O, umma_desc_sw128(pa + k * 32), umma_desc_sw128_mn(va + k * 2048, kMobaChunk * 128), idesc,
-                              (hh > 0 || k > 0) ? 1u : 0u);
+                    umma_bf16_ta(tb + OFF_O, pa + k * 8, umma_desc_sw128_mn(va + k * 2048, kMobaChunk * 128), idesc,
+                                 (hh > 0 || k > 0) ? 1u : 0u);
                 umma_commit(&pv_done[hh & 1]);
                 return true;
             };
@@ -457,23 +476,36 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             for (int k = hv_landed; k < hv_issued; ++k) mbar_wait(&full_v[k % NST], (uint32_t)((k / NST) & 1));
         }
     } else {
-        // ---- the four warps that read the accumulators: thread = query
-        const uint32_t tl = tb + ((uint32_t)(warp * 32) << 16);
-        const uint32_t *mymask = qmask + tid * words;
+        // ---- the eight warps that read the accumulators: warps w and w + 4 share the 32 lanes (queries) of tensor-memory
+        // subpartition w; the first takes the chunk's first 32 positions, the second the other 32
+        const int lq = (warp & 3) * 32 + lane;       // this thread's query inside the CTA
+        const int ch = warp >> 2;                    // which half of a chunk's positions
+        const int64_t tq = t0 + lq;
+        const uint32_t tl = tb + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t *mymask = qmask + lq * words;
         float m = -CUDART_INF_F, l = 0.0f, inv_l = 0.0f;
         int c = -1;
 #pragma unroll 1
         for (int g = 0; g < 2 * n; ++g) {
-            if (g == n) {                            // pass 2 walks the same chunks again
+            if (g == n) {
+                // pass 2 walks the same chunks again; first the two halves of a query's statistics are merged
                 c = -1;
+                stat[ch][lq] = make_float2(m, l);
+                mbar_arrive(&stat_ready);
+                ok = mbar_wait(&stat_ready, 0u);
+                if (!__all_sync(FULLMASK, ok)) break;
+                const float2 other = stat[ch ^ 1][lq];
+                const float mn = fmaxf(m, other.x);
+                if (mn > -CUDART_INF_F) l = l * exp2_fast(m - mn) + other.y * exp2_fast(other.x - mn);
+                m = mn;
                 inv_l = l > 0.0f ? 1.0f / l : 0.0f;
             }
             c = next_chunk(c);
-            const int64_t p0 = (int64_t)c * kMobaChunk;
-            const int j = (int)(p0 / block);
-            // positions of the chunk this query attends: none if it did not choose the block, else those up to its own
+            const int64_t p0 = (int64_t)c * kMobaChunk + ch * 32;    // first of this thread's 32 positions
+            const int j = (int)(((int64_t)c * kMobaChunk) / block);
+            // positions this query attends among them: none if it did not choose the block, else those up to its own
             int nv = 0;
-            if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)kMobaChunk, tq - p0 + 1));
+            if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)32, tq - p0 + 1));
             ok = mbar_wait(&s_ready[g & 1], (uint32_t)((g >> 1) & 1));
             if (!__all_sync(FULLMASK, ok)) break;
             tcgen05_after_sync();
@@ -482,68 +514,63 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 ok = mbar_wait(&pv_done[hh & 1], (uint32_t)(((hh - 2) >> 1) & 1));
                 if (!__all_sync(FULLMASK, ok)) break;
             }
-#pragma unroll 1
-            for (int cb = 0; cb < kMobaChunk; cb += 32) {
-                float v[32];
-                tmem_ld32(tl + (uint32_t)(g & 1) * ACC_S + (uint32_t)cb, v);
-                if (hh < 0) {
-                    if (cb < nv) {
-                        float tm = -CUDART_INF_F;
+            float v[32];
+            tmem_ld32(tl + (uint32_t)(g & 1) * ACC_S + (uint32_t)(ch * 32), v);
+            if (hh < 0) {
+                if (nv > 0) {
+                    float tm = -CUDART_INF_F;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            v[i] = cb + i < nv ? v[i] * scale_log2 : -CUDART_INF_F;
-                            tm = fmaxf(tm, v[i]);
-                        }
-                        const float mn = fmaxf(m, tm);
-                        float sum = 0.0f;
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) sum += exp2_fast(v[i] - mn);
-                        l = l * exp2_fast(m - mn) + sum;
-                        m = mn;
+                    for (int i = 0; i < 32; ++i) {
+                        v[i] = i < nv ? v[i] * scale_log2 : -CUDART_INF_F;
+                        tm = fmaxf(tm, v[i]);
                     }
-                } else {
-                    // normalised weights of 32 positions, rounded to bf16: four 16-byte pieces of this query's row
-                    uint32_t w[16];
+                    const float mn = fmaxf(m, tm);
+                    float sum = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float a = cb + i < nv ? exp2_fast(fmaf(v[i], scale_log2, -m)) * inv_l : 0.0f;
-                        const float bq = cb + i + 1 < nv ? exp2_fast(fmaf(v[i + 1], scale_log2, -m)) * inv_l : 0.0f;
-                        w[i >> 1] = pack2_bf16(a, bq);
-                    }
-                    unsigned char *prow = ps + (size_t)(hh & 1) * G::P_BYTES;
-#pragma unroll
-                    for (int pc = 0; pc < 4; ++pc)
-                        *reinterpret_cast<uint4 *>(prow + umma_sw128_offset(tid, cb / 8 + pc)) =
-                            make_uint4(w[4 * pc], w[4 * pc + 1], w[4 * pc + 2], w[4 * pc + 3]);
+                    for (int i = 0; i < 32; ++i) sum += exp2_fast(v[i] - mn);
+                    l = l * exp2_fast(m - mn) + sum;
+                    m = mn;
                 }
+            } else {
+                // normalised weights of 32 positions, rounded to bf16: 16 columns of this query's lane
+                uint32_t w[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float a = i < nv ? exp2_fast(fmaf(v[i], scale_log2, -m)) * inv_l : 0.0f;
+                    const float bq = i + 1 < nv ? exp2_fast(fmaf(v[i + 1], scale_log2, -m)) * inv_l : 0.0f;
+                    w[i >> 1] = pack2_bf16(a, bq);
+                }
+                tmem_st16(tl + OFF_P + (uint32_t)(hh & 1) * P_COLS + (uint32_t)(ch * 16), w);
             }
             tcgen05_before_sync();
             mbar_arrive(&s_free[g & 1]);             // this thread has read the scores
-            if (hh >= 0 && p0 + kMobaChunk > len) {
+            if (hh >= 0 && (int64_t)c * kMobaChunk + kMobaChunk > len) {
                 // the prompt ends inside this chunk: the value rows past its end hold whatever the cache's memory held;
                 // a weight of zero would not stop a NaN there, so those rows are cleared once they have landed
                 ok = mbar_wait(&full_v[hh % NST], (uint32_t)((hh / NST) & 1));
                 if (!__all_sync(FULLMASK, ok)) break;
                 const int r = tid & (kMobaChunk - 1), hf = tid >> 6;
-                if (hf < G::HALVES && p0 + r >= len) {
+                if (hf < G::HALVES && (int64_t)c * kMobaChunk + r >= len) {
                     uint4 *row = reinterpret_cast<uint4 *>(vst + (size_t)(hh % NST) * G::KC_BYTES + hf * (kMobaChunk * 128) + (r >> 3) * 1024 +
                                                            (r & 7) * 128);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) row[i] = make_uint4(0u, 0u, 0u, 0u);
                 }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordinary stores, read by the tensor core
             }
             if (hh >= 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the weights are read by the tensor core
+                tmem_st_wait();                      // the weights are in tensor memory
+                tcgen05_before_sync();
                 mbar_arrive(&p_ready[hh & 1]);
             }
         }
-        // the output once the last product is complete
+        // the output once the last product is complete: each of a query's two threads writes half of the channels
         if (__all_sync(FULLMASK, ok)) {
             ok = mbar_wait(&pv_done[(n - 1) & 1], (uint32_t)(((n - 1) >> 1) & 1));
             if (__all_sync(FULLMASK, ok)) {
                 tcgen05_after_sync();
 #pragma unroll 1
-                for (int cb = 0; cb < D; cb += 32) {
+                for (int cb = ch * (D / 2); cb < (ch + 1) * (D / 2); cb += 32) {
                     float v[32];
                     tmem_ld32(tl + OFF_O + (uint32_t)cb, v);
                     if (tq < len) {
@@ -573,7 +600,8 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
     const int words = (nb + 31) / 32;
     moba_means_kernel<T><<<dim3((unsigned)nb, (unsigned)BH), D, 0, s>>>((const T *)a.kv, a.page_cap, a.S, D, a.len, a.block,
                                                                       a.means, nb);
-    const size_t rs = (size_t)kMobaRouteWarps * moba_route_floats(D, nb) * sizeof(float);
+    const bool staged = nb <= kMobaStagedBlocks;
+    const size_t rs = (size_t)kMobaRouteWarps * moba_route_floats(D, nb) * sizeof(float) + (staged ? (size_t)nb * (D + 4) * sizeof(float) : 0);
     constexpr int CHUNK_BYTES = 2 * kMobaChunk * D * (int)sizeof(T);
     const size_t as = 2 * (size_t)CHUNK_BYTES + (size_t)words * (kMobaQueries + 1) * sizeof(uint32_t);
     static bool ready[64];
@@ -582,16 +610,23 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
-        e = cudaFuncSetAttribute(moba_route_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(moba_route_kernel<T, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)((size_t)kMobaRouteWarps * moba_route_floats(D, kMobaMaxBlocks) * sizeof(float)));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(moba_route_kernel<T, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)((size_t)kMobaRouteWarps * moba_route_floats(D, kMobaStagedBlocks) * sizeof(float) +
+                                       (size_t)kMobaStagedBlocks * (D + 4) * sizeof(float)));
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(moba_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)(2 * (size_t)CHUNK_BYTES + (size_t)(kMobaMaxBlocks / 32) * (kMobaQueries + 1) * sizeof(uint32_t)));
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
-    moba_route_kernel<T, D><<<dim3((unsigned)((a.len + kMobaRouteWarps - 1) / kMobaRouteWarps), (unsigned)BH), kMobaRouteWarps * 32, rs,
-                              s>>>((const T *)a.q, a.means, a.len, a.H, a.block, nb, a.K, a.sel);
+    const dim3 rgrid((unsigned)((a.len + kMobaRouteWarps - 1) / kMobaRouteWarps), (unsigned)BH);
+    if (staged)
+        moba_route_kernel<T, D, true><<<rgrid, kMobaRouteWarps * 32, rs, s>>>((const T *)a.q, a.means, a.len, a.H, a.block, nb, a.K, a.sel);
+    else
+        moba_route_kernel<T, D, false><<<rgrid, kMobaRouteWarps * 32, rs, s>>>((const T *)a.q, a.means, a.len, a.H, a.block, nb, a.K, a.sel);
     const float sl2 = a.scale * 1.4426950408889634f;
     if constexpr (sizeof(T) == 2) {
         // bf16 caches: the attention on the tensor cores
