@@ -288,12 +288,12 @@ __global__ void __launch_bounds__(kMobaQueries * 32) moba_attend_kernel(const T 
 //   pass 2   S again; the thread turns its row into normalised weights, rounds them to bf16 and writes them
 //            into tensor memory (tcgen05.st) as the A operand of the second product, O += P V (128 x D, the values
 //            as an MN-major operand straight from the cache's rows), accumulated in tensor memory over all chunks
-// One thread of a ninth warp starts the tensor-map copies (keys and values of a chunk, four stages each) and the
+// One thread of a ninth warp starts the tensor-map copies (keys and values of a chunk, two stages each) and the
 // products; the eight other warps read the accumulators (two per query, half of a chunk's positions each).  They meet only through mbarriers; every wait is bounded.
 constexpr int kMobaMmaQueries = 128;
 constexpr int kMobaMmaWarps = 8;               // warps that read the accumulators: two per 32 lanes, half of the columns each
 constexpr int kMobaMmaThreads = (kMobaMmaWarps + 1) * 32;
-constexpr int kMobaMmaStages = 4;
+constexpr int kMobaMmaStages = 2;
 
 template <int D>
 struct MobaMmaGeom {
@@ -330,9 +330,11 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
 {
     using G = MobaMmaGeom<D>;
     constexpr int NST = kMobaMmaStages;
-    // tensor memory: two score accumulators of 64 columns, the output (D columns) from column 128, then two weight
-    // buffers of 32 columns (64 positions as bf16 pairs); allocations are powers of two
-    constexpr uint32_t ACC_S = 64, OFF_O = 128, OFF_P = 128 + D, P_COLS = 32, TCOLS = D == 128 ? 512 : 256;
+    // tensor memory: one score accumulator of 64 columns, the output (D columns), two weight buffers of 32 columns
+    // (64 positions as bf16 pairs): 256 columns, and with two key and two value stages 97 KB of shared memory, so
+    // that TWO CTAs share an SM: each CTA's chunk is a chain of dependent steps, and the two chains overlap
+    constexpr int NSB = 1;                                       // score accumulators
+    constexpr uint32_t ACC_S = 64, OFF_O = 64, OFF_P = 64 + D, P_COLS = 32, TCOLS = 256;
     extern __shared__ __align__(1024) unsigned char msm_raw[];
     __shared__ __align__(8) uint64_t full_k[NST], full_v[NST], s_ready[2], s_free[2], p_ready[2], pv_done[2], stat_ready;
     __shared__ float2 stat[2][kMobaMmaQueries];                          // pass 1: a query's statistics from its two threads
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             const uint32_t qa = smem_addr(qs);
 #pragma unroll 1
             for (int g = 0; g < 2 * n && ok; ++g) {
-                if (g >= 2) ok = mbar_wait(&s_free[g & 1], (uint32_t)(((g >> 1) - 1) & 1));
+                if (g >= NSB) ok = mbar_wait(&s_free[g % NSB], (uint32_t)(((g / NSB) - 1) & 1));
                 ok = ok && mbar_wait(&full_k[g % NST], (uint32_t)((g / NST) & 1));
                 if (!ok) break;
                 gk_landed = g + 1;
@@ -455,14 +457,15 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 const uint32_t ka = smem_addr(kst + (size_t)(g % NST) * G::KC_BYTES);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    umma_bf16(tb + (uint32_t)(g & 1) * ACC_S, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
+                    umma_bf16(tb + (uint32_t)(g % NSB) * ACC_S, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
                               umma_desc_sw128(ka + (k >> 2) * (kMobaChunk * 128) + (k & 3) * 32), idesc_s, k > 0);
-                umma_commit(&s_ready[g & 1]);
+                umma_commit(&s_ready[g % NSB]);
                 const int hh = g - n;                // pass 2: the chunk whose scores were just started
                 if (hh >= 1) ok = product_pv(hh - 1);
-                // refills: the key stage of product g - 1 once that product is complete, the value stage of chunk hh - 2 likewise
+                // refills: the key stage of product g - 1 (complete: its scores were read), the value stage of chunk hh - 2
+                // once the second product of that chunk is complete
                 if (ok && g >= 1 && g - 1 + NST < 2 * n) {
-                    ok = mbar_wait(&s_ready[(g - 1) & 1], (uint32_t)(((g - 1) >> 1) & 1));
+                    ok = true;                       // (one score accumulator: product g - 1 is complete, its scores have been read)
                     if (ok) issue_k();
                 }
                 if (ok && hh >= 2 && hh - 2 + NST < n) {
@@ -506,7 +509,7 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             // positions this query attends among them: none if it did not choose the block, else those up to its own
             int nv = 0;
             if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)32, tq - p0 + 1));
-            ok = mbar_wait(&s_ready[g & 1], (uint32_t)((g >> 1) & 1));
+            ok = mbar_wait(&s_ready[g % NSB], (uint32_t)((g / NSB) & 1));
             if (!__all_sync(FULLMASK, ok)) break;
             tcgen05_after_sync();
             const int hh = g - n;
@@ -515,7 +518,7 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 if (!__all_sync(FULLMASK, ok)) break;
             }
             float v[32];
-            tmem_ld32(tl + (uint32_t)(g & 1) * ACC_S + (uint32_t)(ch * 32), v);
+            tmem_ld32(tl + (uint32_t)(g % NSB) * ACC_S + (uint32_t)(ch * 32), v);
             if (hh < 0) {
                 if (nv > 0) {
                     float tm = -CUDART_INF_F;
@@ -543,7 +546,7 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 tmem_st16(tl + OFF_P + (uint32_t)(hh & 1) * P_COLS + (uint32_t)(ch * 16), w);
             }
             tcgen05_before_sync();
-            mbar_arrive(&s_free[g & 1]);             // this thread has read the scores
+            mbar_arrive(&s_free[g % NSB]);
             if (hh >= 0 && (int64_t)c * kMobaChunk + kMobaChunk > len) {
                 // the prompt ends inside this chunk: the value rows past its end hold whatever the cache's memory held;
                 // a weight of zero would not stop a NaN there, so those rows are cleared once they have landed
