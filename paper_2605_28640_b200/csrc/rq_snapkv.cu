@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(kSnapThreads) snap_tile_kernel(const T *kv, in
 constexpr int kMmaKeys = 128;                  // keys per tile
 constexpr int kMmaWarps = 4;                   // warps that read the accumulator: one thread per lane of it
 constexpr int kMmaThreads = (kMmaWarps + 1) * 32;   // and one warp that starts the copies and the products
-constexpr int kMmaStages = 5;                  // key tiles in shared memory: four in flight while one is multiplied
+constexpr int kMmaStages = 2;                  // key tiles in shared memory: 97 KB with the queries, so that two CTAs share an SM
 constexpr int kMmaMaxTiles = 32;               // tiles per CTA at most
 
 template <int D>
