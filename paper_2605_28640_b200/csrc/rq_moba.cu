@@ -127,6 +127,37 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
         }
     }
     __syncwarp();
+    if (c_hi - c_lo <= 4 * 32) {
+        // few candidates: a candidate's rank is the number of candidates that beat it (higher score, or the same
+        // score and a lower block); a lane ranks its own (at most four) against all of them, read as broadcasts
+        float mv[4];
+        int rank[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int j = c_lo + lane + 32 * r;
+            mv[r] = j < c_hi ? sc[j] : 0.0f;
+            rank[r] = 0;
+        }
+        for (int i = c_lo; i < c_hi; ++i) {
+            const float ov = sc[i];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int j = c_lo + lane + 32 * r;
+                rank[r] += (ov > mv[r] || (ov == mv[r] && i < j)) ? 1 : 0;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int j = c_lo + lane + 32 * r;
+            const unsigned take = __ballot_sync(FULLMASK, j < c_hi && rank[r] < want);   // blocks c_lo + 32 r + bit
+            if (lane == 0 && take) {
+                const int p = c_lo + 32 * r;
+                mask[p >> 5] |= take << (p & 31);
+                if (p & 31) mask[(p >> 5) + 1] |= take >> (32 - (p & 31));
+            }
+        }
+        __syncwarp();
+    } else {
     // the `want` best candidates, one per round: every lane's best of its blocks, then the warp's best;
     // equal scores go to the lower block
     for (int r = 0; r < want; ++r) {
@@ -145,6 +176,7 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
         }
         if (lane == 0 && bj != INT_MAX) mask[bj >> 5] |= 1u << (bj & 31);
         __syncwarp();
+    }
     }
     if (lane == 0) {
         for (int j = 0; j < ns; ++j) mask[j >> 5] |= 1u << (j & 31);

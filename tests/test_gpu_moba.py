@@ -101,6 +101,8 @@ def test_paper_settings_on_4k_prompts(block, K):
     (1, 2, 64, 2049, 64, 64, 6, torch.bfloat16),      # one position into a new block
     (1, 1, 128, 50, 16, 64, 4, torch.float32),        # a prompt shorter than one block
     (1, 2, 128, 1500, 16, 256, 3, torch.bfloat16),    # blocks of 256
+    (1, 2, 64, 12000, 16, 64, 9, torch.bfloat16),     # 188 blocks: representatives read from global memory, arg-max rounds
+    (1, 1, 128, 9000, 16, 64, 20, torch.float32),     # the same on an fp32 cache
 ])
 def test_shapes_blocks_and_ragged_sizes(B, H, D, T, S, block, K, dtype):
     w = wl.Workload("moba-small", B=B, H=H, D=D, T=T, S=S, dtype=dtype, seed=T + K)
