@@ -435,9 +435,16 @@ __global__ void __launch_bounds__(1024) snap_select_kernel(const float *imp, int
             const uint32_t himask = hi == 31 ? 0u : ~0u << (hi + 1);
             for (int i = tid; i < kSnapBins; i += 1024) hist[i] = 0u;
             __syncthreads();
-            for (int j = tid; j < C; j += 1024) {
-                const uint32_t kx = order_key(__ldcg(x + j));
-                if ((kx & himask) == (prefix & himask)) atomicAdd(&hist[(kx >> lo) & dmask], 1u);
+            // eight independent loads per thread are issued before the first is used
+            for (int j0 = tid; j0 < C; j0 += 8 * 1024) {
+                float f[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) f[u] = j0 + u * 1024 < C ? __ldcg(x + j0 + u * 1024) : 0.0f;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const uint32_t kx = order_key(f[u]);
+                    if (j0 + u * 1024 < C && (kx & himask) == (prefix & himask)) atomicAdd(&hist[(kx >> lo) & dmask], 1u);
+                }
             }
             __syncthreads();
             // walk the bins from the top until k keys are covered: thread t owns bins 2t, 2t+1
@@ -473,12 +480,17 @@ __global__ void __launch_bounds__(1024) snap_select_kernel(const float *imp, int
     // every warp owns a contiguous range of the candidates: count, scan over the warps, write
     const int per = (C + 31) / 32, lo_j = warp * per, hi_j = min(C, lo_j + per);
     uint32_t wgt = 0, weq = 0;
-    for (int j0 = lo_j; j0 < hi_j; j0 += 32) {
-        const int j = j0 + lane;
-        const bool in = j < hi_j;
-        const uint32_t kx = in ? order_key(__ldcg(x + j)) : 0u;
-        wgt += __popc(__ballot_sync(FULL, in && kx > tau));
-        weq += __popc(__ballot_sync(FULL, in && kx == tau));
+    for (int j0 = lo_j; j0 < hi_j; j0 += 8 * 32) {
+        float f[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) f[u] = j0 + u * 32 + lane < hi_j ? __ldcg(x + j0 + u * 32 + lane) : 0.0f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const bool in = j0 + u * 32 + lane < hi_j;
+            const uint32_t kx = order_key(f[u]);
+            wgt += __popc(__ballot_sync(FULL, in && kx > tau));
+            weq += __popc(__ballot_sync(FULL, in && kx == tau));
+        }
     }
     if (lane == 0) { red[warp] = wgt; red2[warp] = weq; }
     __syncthreads();
@@ -490,17 +502,23 @@ __global__ void __launch_bounds__(1024) snap_select_kernel(const float *imp, int
     }
     int gt_run = (int)(__shfl_sync(FULL, g_inc, warp) - wgt), eq_run = (int)(__shfl_sync(FULL, e_inc, warp) - weq);
     const uint32_t lt = (1u << lane) - 1u;
-    for (int j0 = lo_j; j0 < hi_j; j0 += 32) {
-        const int j = j0 + lane;
-        const bool in = j < hi_j;
-        const uint32_t kx = in ? order_key(__ldcg(x + j)) : 0u;
-        const bool is_gt = in && kx > tau, is_eq = in && kx == tau;
-        const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
-        const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
-        const int rank = is_gt ? gb + min(eb, r_eq) : (is_eq && eb < r_eq) ? gb + eb : -1;
-        if (rank >= 0 && rank < want) out[rank] = j;
-        gt_run += __popc(bg);
-        eq_run += __popc(be);
+    for (int j0 = lo_j; j0 < hi_j; j0 += 8 * 32) {
+        float f[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) f[u] = j0 + u * 32 + lane < hi_j ? __ldcg(x + j0 + u * 32 + lane) : 0.0f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * 32 + lane;
+            const bool in = j < hi_j;
+            const uint32_t kx = order_key(f[u]);
+            const bool is_gt = in && kx > tau, is_eq = in && kx == tau;
+            const uint32_t bg = __ballot_sync(FULL, is_gt), be = __ballot_sync(FULL, is_eq);
+            const int gb = gt_run + __popc(bg & lt), eb = eq_run + __popc(be & lt);
+            const int rank = is_gt ? gb + min(eb, r_eq) : (is_eq && eb < r_eq) ? gb + eb : -1;
+            if (rank >= 0 && rank < want) out[rank] = j;
+            gt_run += __popc(bg);
+            eq_run += __popc(be);
+        }
     }
     for (int i = tid; i < w; i += 1024) out[want + i] = C + i;       // the window, above every candidate
 }
