@@ -127,8 +127,9 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
         }
     }
     __syncwarp();
-    if (c_hi - c_lo <= 4 * 32) {
-        // few candidates: a candidate's rank is the number of candidates that beat it (higher score, or the same
+    if (c_hi - c_lo <= 4 * 32 && want >= 8) {
+        // few candidates and more than a handful to take (a round per taken block is cheaper otherwise): a
+        // candidate's rank is the number of candidates that beat it (higher score, or the same
         // score and a lower block); a lane ranks its own (at most four) against all of them, read as broadcasts
         float mv[4];
         int rank[4];
