@@ -204,6 +204,36 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def max_over_ranks(ms, world, device):
+    """The slowest rank's time: what a job of `world` replicas takes."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_us_per_step(max_ms, steps, world):
+    """Replicas only: `world` GPUs each take a step in max_ms / steps, so the job takes that time per `world` steps."""
+    return max_ms / steps * 1e3 / world
+
+
+def selftest_ranks():
+    """The rank plumbing on CPU (gloo): every rank contributes a time, rank 0 prints what the job would report."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = max_over_ranks(10.0 * (rank + 1), world, "cpu")
+    if rank == 0:
+        print(json.dumps({"max_ms": ms, "world": world, "us_per_step": whole_job_us_per_step(ms, 5, world)}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def workload_config(w):
     return {"workload": w.name, "batch": w.B, "heads": w.H, "head_dim": w.D, "context": w.T,
             "page_size": w.S, "budget": f"{w.budget_num}/{w.budget_den}", "budget_pages": w.budget_pages(),
@@ -341,7 +371,8 @@ def moba_block(w, dev):
                             "attended_fraction": pairs / (T * (T + 1) / 2), "tflops_on_attended_pairs": flops / (ts[2] * 1e-3) / 1e12})
         del scratch
     out["status_ok"] = rq.rq_device_status(cache.handle) == rq.RQ_OK
-    out["note"] = "rq_moba_prefill = block means + routing of every query + attention over the chosen blocks (plain fp32 FMA kernels)"
+    out["note"] = ("rq_moba_prefill = block means + routing of every query + attention over the chosen blocks "
+                   "(both products of the attention on the tensor cores for bf16 caches)")
     return out
 
 
@@ -361,6 +392,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
     ap.add_argument("--no-parity", action="store_true")
+    ap.add_argument("--selftest-ranks", action="store_true", help="CPU check of the multi-rank plumbing (gloo); used by the tests")
     ap.add_argument("--no-next", action="store_true", help="skip the SnapKV and MoBA timing blocks (they run by default)")
     ap.add_argument("--moba", action="store_true",
                     help="also time the MoBA-style block-sparse prefill attention at the paper's setting (4K prompts, block 64, "
@@ -368,6 +400,9 @@ def main():
     ap.add_argument("--snapkv", action="store_true",
                     help="also time the SnapKV-style reduction of the first cache (window 64, 1/16 of the entries retained)")
     args = ap.parse_args()
+    if args.selftest_ranks:
+        selftest_ranks()
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "rq" else args.warmup
 
     import dataclasses
@@ -484,10 +519,7 @@ def main():
             if j % 16 == 0:
                 torch.cuda.synchronize()
         torch.cuda.synchronize()
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = t.item() / args.steps
+    ms_per_step = max_over_ranks(ms, world, dev) / args.steps
     n_launches = args.steps * launches_per_step
 
     # ---- per-kernel times of the step run as separate kernels (a separate pass, same rotation):
@@ -542,10 +574,7 @@ def main():
         e2e_step(i)
     e1.record()
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_us = t.item() / n_e2e * 1e3
+    e2e_us = max_over_ranks(e0.elapsed_time(e1), world, dev) / n_e2e * 1e3
     in_bytes = w.B * w.H * w.D * (3 * es + (2 if w.gdtype == torch.bfloat16 else 4))
     out_bytes = w.B * w.H * w.D * es
 
@@ -575,7 +604,7 @@ def main():
     roof["as_separate_kernels_us"] = kernel_us
     roof["as_separate_kernels"] = separate
     line = {
-        "metric": METRIC, "value": us / world, "unit": "us/step", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": whole_job_us_per_step(ms_per_step * args.steps, args.steps, world), "unit": "us/step", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(w),
         "l2": f"inputs larger than L2: {ncopies} independent caches rotated, fresh q/k/v/g every step",
@@ -584,7 +613,7 @@ def main():
                      "frac_of_nominal_8tbs": step_gbs / 8000.0, "peak_gbs": peak, "peak_kind": peak_kind},
         "roofline": roof,
         "clocks": clocks.summary(),
-        "e2e": {"value": e2e_us / world, "unit": "us/step", "h2d_bytes_per_step": in_bytes,
+        "e2e": {"value": whole_job_us_per_step(e2e_us * n_e2e / 1e3, n_e2e, world), "unit": "us/step", "h2d_bytes_per_step": in_bytes,
                 "d2h_bytes_per_step": out_bytes},
         "gpu_launches": n_launches, "launches_per_step": launches_per_step,
     }

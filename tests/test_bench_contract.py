@@ -28,3 +28,19 @@ def test_reference_arm_two_ranks():
     assert line["cpu_baseline"]["value"] == line["value"] and line["cpu_baseline"]["sample"]
     assert line["e2e"] == {"value": line["value"], "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert line["config"]["workload"] == "7b-layer-16k" and line["vs_baseline"] is None
+
+
+def test_rank_plumbing_two_ranks_gloo():
+    """Two CPU ranks over gloo: the job's time is the slowest rank's, the whole-job value divides by the replicas,
+    and rank 0 alone prints."""
+    procs = []
+    for r in range(2):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT="29541",
+                   CUDA_VISIBLE_DEVICES="")
+        procs.append(subprocess.Popen([sys.executable, os.path.join(ROOT, "bench.py"), "--selftest-ranks"], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    outs = [p.communicate(timeout=300) for p in procs]
+    assert all(p.returncode == 0 for p in procs), [o[1][-500:] for o in outs]
+    assert outs[1][0].strip() == ""
+    line = json.loads(outs[0][0].strip().splitlines()[-1])
+    assert line == {"max_ms": 20.0, "world": 2, "us_per_step": 20.0 / 5 * 1e3 / 2}
