@@ -28,6 +28,22 @@ __device__ __forceinline__ uint4 ldg16(const void *p) { return __ldg(reinterpret
 __device__ __forceinline__ uint4 ldcs16(const void *p) { return __ldcs(reinterpret_cast<const uint4 *>(p)); }
 
 // Expand one 16-byte vector of T into floats.
+// Two fp32 operations in one instruction (packed pairs); each half is rounded like the scalar operation, so the
+// results are the same bits as two scalar instructions.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c)
+{
+    unsigned long long ra = *reinterpret_cast<unsigned long long *>(&a), rb = *reinterpret_cast<unsigned long long *>(&b),
+                       rc = *reinterpret_cast<unsigned long long *>(&c), rd;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(rd) : "l"(ra), "l"(rb), "l"(rc));
+    return *reinterpret_cast<float2 *>(&rd);
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b)
+{
+    unsigned long long ra = *reinterpret_cast<unsigned long long *>(&a), rb = *reinterpret_cast<unsigned long long *>(&b), rd;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    return *reinterpret_cast<float2 *>(&rd);
+}
+
 template <typename T> __device__ __forceinline__ void unpack16(const uint4 &r, float *out);
 template <> __device__ __forceinline__ void unpack16<bf16>(const uint4 &r, float *out)
 {

@@ -190,8 +190,8 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
         const int64_t tile_start = (tile0 + i) * TT;
 
         // ---- pass 1: this thread's run as a map from a zero state (identity outside the new range)
-        float g0[RT], g1[RT], k0[RT], k1[RT], v0[RT], v1[RT];    // g, (1-g) k, (1-g) v of the two channels
-        float A0 = 1.0f, A1 = 1.0f, Bk0 = 0.0f, Bk1 = 0.0f, Bv0 = 0.0f, Bv1 = 0.0f;
+        float2 g2[RT], k2[RT], v2[RT];                           // g, (1-g) k, (1-g) v of the two channels
+        float2 A2 = make_float2(1.0f, 1.0f), Bk2 = make_float2(0.0f, 0.0f), Bv2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
             const int e = row_slot<T>(row0 + r) * CG + ch2;
@@ -204,14 +204,15 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
                 ka = 0.0f; kb = 0.0f;
                 va = 0.0f; vb = 0.0f;
             }
-            const float oa = 1.0f - ga, ob = 1.0f - gb;
-            g0[r] = ga; g1[r] = gb;
-            k0[r] = oa * ka; k1[r] = ob * kb;
-            v0[r] = oa * va; v1[r] = ob * vb;
-            A0 *= ga; A1 *= gb;
-            Bk0 = fmaf(ga, Bk0, k0[r]); Bk1 = fmaf(gb, Bk1, k1[r]);
-            Bv0 = fmaf(ga, Bv0, v0[r]); Bv1 = fmaf(gb, Bv1, v1[r]);
+            g2[r] = make_float2(ga, gb);
+            const float2 o2 = fma2(g2[r], make_float2(-1.0f, -1.0f), make_float2(1.0f, 1.0f));   // 1 - g
+            k2[r] = mul2(o2, make_float2(ka, kb));
+            v2[r] = mul2(o2, make_float2(va, vb));
+            A2 = mul2(A2, g2[r]);
+            Bk2 = fma2(g2[r], Bk2, k2[r]);
+            Bv2 = fma2(g2[r], Bv2, v2[r]);
         }
+        const float A0 = A2.x, A1 = A2.y, Bk0 = Bk2.x, Bk1 = Bk2.y, Bv0 = Bv2.x, Bv1 = Bv2.y;
         // the map of the warp's first run, for the second run; the second run's lanes publish the warp's map
         const float LA0 = __shfl_sync(FULLMASK, A0, hl), LA1 = __shfl_sync(FULLMASK, A1, hl);
         const float LBk0 = __shfl_sync(FULLMASK, Bk0, hl), LBk1 = __shfl_sync(FULLMASK, Bk1, hl);
@@ -265,14 +266,15 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
                 sv0 = fmaf(LA0, sv0, LBv0); sv1 = fmaf(LA1, sv1, LBv1);
             }
         }
+        float2 sk2 = make_float2(sk0, sk1), sv2 = make_float2(sv0, sv1);
         float mn0 = INFINITY, mn1 = INFINITY, mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
             const int e = row_slot<T>(row0 + r) * CG + ch2;
             if (FULL || (row0 + r >= lo && row0 + r < hi)) {
-                sk0 = fmaf(g0[r], sk0, k0[r]); sk1 = fmaf(g1[r], sk1, k1[r]);
-                sv0 = fmaf(g0[r], sv0, v0[r]); sv1 = fmaf(g1[r], sv1, v1[r]);
-                float rk0 = sk0, rk1 = sk1, rv0 = sv0, rv1 = sv1;
+                sk2 = fma2(g2[r], sk2, k2[r]);
+                sv2 = fma2(g2[r], sv2, v2[r]);
+                float rk0 = sk2.x, rk1 = sk2.y, rv0 = sv2.x, rv1 = sv2.y;
                 store2(ks + e, rk0, rk1);
                 store2(vs + e, rv0, rv1);
                 mn0 = fminf(mn0, rk0); mx0 = fmaxf(mx0, rk0);

@@ -77,15 +77,15 @@ __device__ __forceinline__ void score_unit(const unsigned char *ub, const float 
 #pragma unroll
     for (int gi = 0; gi < NR; ++gi) {
         const unsigned char *rec = ub + (size_t)(gi * PPW + sub) * G::REC_BYTES;
-        float s = 0.0f;
+        float2 s2 = make_float2(0.0f, 0.0f);               // even and odd channels summed apart, then together
 #pragma unroll
         for (int v = 0; v < VPL; ++v) {
             float m[CH];
             unpack16<T>(lds16(rec + (c + v * LPP) * 16), m);
 #pragma unroll
-            for (int i = 0; i < CH; ++i) s = fmaf(qs[v][i], m[i], s);
+            for (int i = 0; i < CH; i += 2) s2 = fma2(make_float2(qs[v][i], qs[v][i + 1]), make_float2(m[i], m[i + 1]), s2);
         }
-        val[gi] = s;
+        val[gi] = s2.x + s2.y;
     }
     // sum over the LPP lanes of a record; while more than one value is left a step also
     // halves the values a lane carries, so the whole reduction costs about NR shuffles
@@ -183,10 +183,10 @@ __device__ __forceinline__ void attend_tile(AttendState<T> &st, const T *ks, con
     for (int n = 0; n < NI; ++n) {
         float kf[CH];
         unpack16<T>(lds16(ks + (n * 32 + lane) * CH), kf);
-        float d = 0.0f;
+        float2 d2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-        for (int c = 0; c < CH; ++c) d = fmaf(st.qf[c], kf[c], d);
-        s[n] = d;
+        for (int c = 0; c < CH; c += 2) d2 = fma2(make_float2(st.qf[c], st.qf[c + 1]), make_float2(kf[c], kf[c + 1]), d2);
+        s[n] = d2.x + d2.y;
     }
     int nv = NI;
 #pragma unroll
@@ -217,7 +217,11 @@ __device__ __forceinline__ void attend_tile(AttendState<T> &st, const T *ks, con
     st.m = m_new;
     st.l = fmaf(st.l, alpha, p_row);
 #pragma unroll
-    for (int c = 0; c < CH; ++c) st.acc[c] *= alpha;
+    for (int c = 0; c < CH; c += 2) {
+        const float2 a2 = mul2(make_float2(st.acc[c], st.acc[c + 1]), make_float2(alpha, alpha));
+        st.acc[c] = a2.x;
+        st.acc[c + 1] = a2.y;
+    }
     // V: row group n's weight comes from the lane that holds it
 #pragma unroll
     for (int n = 0; n < NI; ++n) {
@@ -225,7 +229,11 @@ __device__ __forceinline__ void attend_tile(AttendState<T> &st, const T *ks, con
         float vf[CH];
         unpack16<T>(lds16(vs + (n * 32 + lane) * CH), vf);
 #pragma unroll
-        for (int c = 0; c < CH; ++c) st.acc[c] = fmaf(p, vf[c], st.acc[c]);
+        for (int c = 0; c < CH; c += 2) {
+            const float2 a2 = fma2(make_float2(p, p), make_float2(vf[c], vf[c + 1]), make_float2(st.acc[c], st.acc[c + 1]));
+            st.acc[c] = a2.x;
+            st.acc[c + 1] = a2.y;
+        }
     }
 }
 
