@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/*_96k_b1.md: captured on a 96K-context case, scaled by 4/3 to the launches of the
 # default workload, traffic being proportional to the pages processed): kernel -> bytes, or None
 # when the kernel has changed since the capture.
-NCU_TRAFFIC = {"score": 4 / 3 * (100.83e6 + 3.83e6), "attend": 4 / 3 * (100.81e6 + 2.82e6), "step": 4 / 3 * (201.73e6 + 5.03e6)}
+NCU_TRAFFIC = {"score": 4 / 3 * (100.83e6 + 4.78e6), "attend": 4 / 3 * (100.81e6 + 3.64e6), "step": 4 / 3 * (201.73e6 + 5.97e6)}
 
 
 def measured_peak():
