@@ -47,6 +47,7 @@ WorkspaceLayout workspace_layout(const rq_config &c)
     const size_t slots = (size_t)attend_slots_per_head((int64_t)c.max_budget_pages * (c.page_size / 16));
     w.partial = off; off += align256(BH * slots * (size_t)(c.head_dim + 4) * sizeof(float));
     w.staging = off; off += align256(5 * BH * (size_t)c.head_dim * 4);
+    w.scan = off;    off += align256(kScanScratchBytes);
     w.total = off;
     return w;
 }
@@ -401,6 +402,7 @@ int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
     a.dtype = c.dtype; a.gate_dtype = c.gate_dtype;
     a.len0 = cache->len; a.T = T; a.page_cap = cache->page_capacity;
     a.absmax = absmax_of(cache);
+    a.chunk_scratch = (float *)((char *)cache->workspace + w.scan);
     if (launch_scan(a, (cudaStream_t)stream) != cudaSuccess) return RQ_ERR_CUDA;
     cache->len += T;
     return RQ_OK;

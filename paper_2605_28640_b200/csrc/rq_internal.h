@@ -43,6 +43,7 @@ struct WorkspaceLayout {
     size_t sel;       // int32 [BH][max_budget]
     size_t partial;   // float [BH][slots per head][D + 4]: flash-decode partials
     size_t staging;   // 5 * [BH][D] elements of 4 bytes (host-call staging)
+    size_t scan;      // kScanScratchBytes: the maps and entry states of the prefill's time chunks (few heads, long prompts)
     // the one-launch step (present when BH <= kStepMaxHeads, otherwise empty); everything from
     // `status` up to `scores` is cleared by rq_cache_reset, which is why these regions sit there
     size_t absmax;    // float [2][BH]: largest |stored key| of every head, two copies (read one, write the other)
@@ -64,7 +65,9 @@ struct ScanArgs {
     int B, H, D, S, dtype, gate_dtype;
     int64_t len0, T, page_cap;
     float *absmax;      // [2][BH] largest |stored key| per head, both copies brought up to date (NULL: not tracked)
+    float *chunk_scratch;   // kScanScratchBytes of device memory for the time-chunked form (NULL: one chunk always)
 };
+constexpr size_t kScanScratchBytes = (size_t)2 << 20;
 cudaError_t launch_scan(const ScanArgs &a, cudaStream_t s);
 
 struct DecodeArgs {

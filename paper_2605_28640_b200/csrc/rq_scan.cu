@@ -103,9 +103,22 @@ template <typename T, typename G> __host__ __device__ constexpr int scan_stages(
     return 192 * 1024 / scan_stage_bytes<T, G>() < 4 ? 192 * 1024 / scan_stage_bytes<T, G>() : 4;
 }
 
-template <typename T, typename G, int D, int S>
-__global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int ntiles)
+// MODE 0: the scan proper.  MODE 1: the affine map of a time chunk only (no output), for the time-chunked form.
+// Time chunks (chunks > 1; few heads and a long prompt, so that one CTA per channel group would leave most of the
+// chip idle): CTA x works on channel group x % units and the chunk_tiles tiles of chunk x / units.  First every
+// chunk but the last is reduced to its map s -> A s + B (MODE 1), a small kernel chains the maps into the state
+// that enters every chunk, then every chunk runs the scan proper from its own entry state.  The inputs of all
+// chunks but the last are read twice.
+//   maps   [units][chunks][3][CG]   A, B of the keys, B of the values
+//   entry  [units][chunks][2][CG]   state entering a chunk (chunk 0: the cache's state)
+template <typename T, typename G, int D, int S, int MODE>
+__global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int ntiles, int units, int chunks, int chunk_tiles,
+                                                  float *maps, const float *entry)
 {
+    const int unit = blockIdx.x % units, chunk = blockIdx.x / units;
+    if (MODE == 1 && chunk == chunks - 1) return;           // the last chunk's map is not needed
+    tile0 += (int64_t)chunk * chunk_tiles;
+    ntiles = min(chunk_tiles, ntiles - chunk * chunk_tiles);
     constexpr int NST = scan_stages<T, G>();
     constexpr int STAGE = scan_stage_bytes<T, G>();
     constexpr int EPC_T = 16 / (int)sizeof(T), EPC_G = 16 / (int)sizeof(G);   // elements per 16-byte piece
@@ -122,13 +135,14 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
     __shared__ __align__(8) float wmap[NW * kMapStride];    // the warps' maps of the current tile: [warp][A, Bk, Bv][channel]
     __shared__ __align__(8) float sin_[NW * kInStride];     // state entering every warp: [warp][k, v][channel]
     __shared__ float carry[2][2][CG];                       // state entering the tile (by tile parity): k, v
+    __shared__ float carry_a[2][CG];                        // MODE 1: product of the gates since the chunk began
     __shared__ float mm[NW][2][CG];                         // min / max of the warps (pages wider than a warp's 16 positions)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int hl = lane & 15, half = lane >> 4;  // channel pair of this lane; which of the warp's two runs
     const int ch2 = 2 * hl;                      // first of this lane's two channels inside the group
     constexpr int GPH = D / CG;                  // channel groups per head
-    const int bh = blockIdx.x / GPH, c0 = (blockIdx.x % GPH) * CG;
+    const int bh = unit / GPH, c0 = (unit % GPH) * CG;
     const int b = bh / a.H, h = bh % a.H;
     const int64_t end = a.len0 + a.T;
     const int64_t tail_end = (end + S - 1) / S * S;   // end of the last touched page
@@ -166,9 +180,19 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
         }
     };
 
-    if (tid < CG) {                              // the state the sequence starts from
-        carry[0][0][tid] = a.state[(int64_t)bh * 2 * D + c0 + tid];
-        carry[0][1][tid] = a.state[(int64_t)bh * 2 * D + D + c0 + tid];
+    if (tid < CG) {                              // the state the (chunk of the) sequence starts from
+        if (MODE == 1) {
+            carry[0][0][tid] = 0.0f;
+            carry[0][1][tid] = 0.0f;
+            carry_a[0][tid] = 1.0f;
+        } else if (chunk == 0) {
+            carry[0][0][tid] = a.state[(int64_t)bh * 2 * D + c0 + tid];
+            carry[0][1][tid] = a.state[(int64_t)bh * 2 * D + D + c0 + tid];
+        } else {
+            const float *e = entry + ((int64_t)unit * chunks + chunk) * 2 * CG;
+            carry[0][0][tid] = e[tid];
+            carry[0][1][tid] = e[CG + tid];
+        }
     }
 #pragma unroll 1
     for (int s = 0; s < NST - 1; ++s) {
@@ -251,8 +275,10 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
             if (m == LPC - 1) {                              // state entering the next tile
                 carry[(i + 1) & 1][0][ci] = fmaf(sa, ck, sbk);
                 carry[(i + 1) & 1][1][ci] = fmaf(sa, cv, sbv);
+                if (MODE == 1) carry_a[(i + 1) & 1][ci] = sa * carry_a[i & 1][ci];
             }
         }
+        if (MODE == 1) return;                               // the map needs no more of the tile (the lambda's caller goes on)
         __syncthreads();
 
         // ---- pass 2: token by token, rounded rows back into the stage, bounds of the rounded keys
@@ -355,7 +381,16 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
     }
     cp_async_wait<0>();
     __syncthreads();
-    if (tid < CG) {                              // the state after the last token
+    if (MODE == 1) {
+        if (tid < CG) {                          // the chunk's map
+            float *mp = maps + ((int64_t)unit * chunks + chunk) * 3 * CG;
+            mp[tid] = carry_a[ntiles & 1][tid];
+            mp[CG + tid] = carry[ntiles & 1][0][tid];
+            mp[2 * CG + tid] = carry[ntiles & 1][1][tid];
+        }
+        return;
+    }
+    if (tid < CG && chunk == chunks - 1) {       // the state after the last token
         a.state[(int64_t)bh * 2 * D + c0 + tid] = carry[ntiles & 1][0][tid];
         a.state[(int64_t)bh * 2 * D + D + c0 + tid] = carry[ntiles & 1][1][tid];
     }
@@ -366,6 +401,19 @@ __global__ void __launch_bounds__(NT) scan_kernel(ScanArgs a, int64_t tile0, int
             atomicMax(reinterpret_cast<unsigned *>(a.absmax) + bh, m);
             atomicMax(reinterpret_cast<unsigned *>(a.absmax) + (int64_t)a.B * a.H + bh, m);
         }
+    }
+}
+
+// The state entering every chunk from the chunks' maps, in order.  Grid: channel groups; a thread per (k or v, channel).
+__global__ void scan_chain_kernel(const float *state, int D, int gph, int chunks, const float *maps, float *entry)
+{
+    const int unit = blockIdx.x, kv = threadIdx.x / CG, ch = threadIdx.x % CG;
+    const int bh = unit / gph, c0 = (unit % gph) * CG;
+    float s = state[(int64_t)bh * 2 * D + kv * D + c0 + ch];
+    for (int c = 0; c + 1 < chunks; ++c) {
+        const float *mp = maps + ((int64_t)unit * chunks + c) * 3 * CG;
+        s = fmaf(mp[ch], s, mp[(1 + kv) * CG + ch]);
+        entry[(((int64_t)unit * chunks + c + 1) * 2 + kv) * CG + ch] = s;
     }
 }
 
@@ -386,11 +434,29 @@ cudaError_t run(const ScanArgs &a, cudaStream_t s)
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!ready[dev]) {
-        e = cudaFuncSetAttribute(scan_kernel<T, G, D, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, DSM);
+        e = cudaFuncSetAttribute(scan_kernel<T, G, D, S, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, DSM);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(scan_kernel<T, G, D, S, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, DSM);
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
-    scan_kernel<T, G, D, S><<<(unsigned)ctas, NT, DSM, s>>>(a, t0, (int)(t1 - t0));
+    // Time chunks: only where one CTA per channel group would fill less than half of the SMs and the prompt is long
+    // enough for chunks of at least 16 tiles; as many chunks as give every SM a CTA, within the scratch.
+    const int ntiles = (int)(t1 - t0), units = (int)ctas, sms = sm_count();
+    int chunks = 1;
+    if (a.chunk_scratch && 2 * units <= sms && ntiles >= 32) {
+        chunks = sms / units;
+        if (chunks > ntiles / 16) chunks = ntiles / 16;
+        while (chunks > 1 && (size_t)units * chunks * 5 * CG * sizeof(float) > kScanScratchBytes) --chunks;
+    }
+    int chunk_tiles = (ntiles + chunks - 1) / chunks;
+    chunks = (ntiles + chunk_tiles - 1) / chunk_tiles;
+    float *maps = a.chunk_scratch, *entry = a.chunk_scratch ? a.chunk_scratch + (size_t)units * chunks * 3 * CG : nullptr;
+    if (chunks > 1) {
+        scan_kernel<T, G, D, S, 1><<<(unsigned)(units * chunks), NT, DSM, s>>>(a, t0, ntiles, units, chunks, chunk_tiles, maps, entry);
+        scan_chain_kernel<<<(unsigned)units, 2 * CG, 0, s>>>(a.state, D, D / CG, chunks, maps, entry);
+    }
+    scan_kernel<T, G, D, S, 0><<<(unsigned)(units * chunks), NT, DSM, s>>>(a, t0, ntiles, units, chunks, chunk_tiles, maps, entry);
     return cudaGetLastError();
 }
 
