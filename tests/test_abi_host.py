@@ -123,6 +123,49 @@ def test_argument_checks_on_a_filled_in_handle(lib):
     assert lib.rq_select_pages(C.byref(cache), 256, 1, None, 256, None) == rq.RQ_ERR_INVALID_ARG   # empty cache
 
 
+def test_argument_checks_of_the_widened_rows(lib):
+    """SnapKV and MoBA entry points: everything that is decided on the host before a launch."""
+    c = cfg(capacity_tokens=8192, max_budget_pages=8)
+    cache = rq.rq_cache()
+    cache.cfg = c
+    cache.kv = cache.meta = cache.state = cache.workspace = 4096
+    cache.page_capacity = 8192 // c.page_size
+    cache.len = 5000
+    n = C.c_size_t()
+    BH = c.batch * c.heads
+    # SnapKV scratch: importance [BH][len] fp32 + statistics per 128-key tile and final, each rounded to 256 bytes
+    assert lib.rq_snapkv_scratch_bytes(C.byref(cache), C.byref(n)) == rq.RQ_OK
+    tiles = -(-5000 // 128)
+    r256 = lambda x: -(-x // 256) * 256
+    assert n.value == r256(BH * 5000 * 4) + r256(BH * tiles * 64 * 8) + r256(BH * 64 * 8)
+    assert lib.rq_snapkv_scratch_bytes(C.byref(cache), None) == rq.RQ_ERR_INVALID_ARG
+    for window, keep in ((0, 16), (65, 16), (64, 0), (5001, 16)):
+        assert lib.rq_snapkv_select(C.byref(cache), 256, window, keep, 0.0, 256, None, 256, None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_snapkv_select(C.byref(cache), None, 64, 16, 0.0, 256, None, 256, None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_snapkv_select(C.byref(cache), 256, 64, 16, 0.0, 256, None, 260, None) == rq.RQ_ERR_INVALID_ARG   # scratch alignment
+    other = rq.rq_cache()
+    other.cfg = cfg(capacity_tokens=64, max_budget_pages=2)
+    other.kv = other.meta = other.state = other.workspace = 8192
+    other.page_capacity = 4
+    assert lib.rq_snapkv_compact(C.byref(cache), 256, 65, C.byref(other), None) == rq.RQ_ERR_CAPACITY
+    assert lib.rq_snapkv_compact(C.byref(cache), 256, 0, C.byref(other), None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_snapkv_compact(C.byref(cache), 256, 5001, C.byref(other), None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_snapkv_compact(C.byref(cache), None, 16, C.byref(other), None) == rq.RQ_ERR_INVALID_ARG
+    other.kv = 4096                                                   # the same buffer as the source
+    assert lib.rq_snapkv_compact(C.byref(cache), 256, 16, C.byref(other), None) == rq.RQ_ERR_INVALID_ARG
+    # MoBA scratch: representatives [BH][blocks][D] fp32 + chosen blocks [BH][len][K] int32
+    assert lib.rq_moba_scratch_bytes(C.byref(cache), 64, 4, C.byref(n)) == rq.RQ_OK
+    nb = -(-5000 // 64)
+    assert n.value == r256(BH * nb * c.head_dim * 4) + r256(BH * 5000 * 4 * 4)
+    for block, K in ((32, 4), (96, 4), (64, 1), (72, 4)):
+        assert lib.rq_moba_scratch_bytes(C.byref(cache), block, K, C.byref(n)) == rq.RQ_ERR_INVALID_ARG
+        assert lib.rq_moba_prefill(C.byref(cache), 256, block, K, 0.0, 256, None, None, 256, None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_moba_prefill(C.byref(cache), None, 64, 4, 0.0, 256, None, None, 256, None) == rq.RQ_ERR_INVALID_ARG
+    assert lib.rq_moba_prefill(C.byref(cache), 256, 64, 4, 0.0, 256, None, None, 260, None) == rq.RQ_ERR_INVALID_ARG
+    cache.len = 0
+    assert lib.rq_moba_scratch_bytes(C.byref(cache), 64, 4, C.byref(n)) == rq.RQ_ERR_INVALID_ARG
+
+
 def _no_gpu():
     import torch
     return not torch.cuda.is_available()
