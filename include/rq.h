@@ -141,6 +141,9 @@ RQ_API int rq_cache_reset(rq_cache *cache, void *stream);
  *          multiples of 16 bytes; d contiguous; base 16-byte aligned)
  *   g    : same indexing, of cfg.gate_dtype, values in [0, 1]; the same gate
  *          drives k and v.
+ * The same call on the same inputs gives the same bits.  How a prompt is cut into calls, and how the
+ * library cuts a long prompt of few heads into time chunks that run side by side, changes the order of
+ * the fp32 operations: states agree within rounding (a few 1e-7 relative), not bit for bit.
  * Errors: INVALID_ARG (NULL, T < 0, misaligned), CAPACITY (len + T exceeds
  * capacity_tokens; nothing is enqueued), CUDA.  T == 0 is a no-op. */
 RQ_API int rq_build_cache(rq_cache *cache, const void *k, const void *v, const void *g,
