@@ -174,3 +174,26 @@ def test_argument_checks():
     with pytest.raises(rq.RqError) as e:
         rq.rq_moba_prefill(empty.handle, q, 64, 4, 0.0, o, None, None, scratch)
     assert e.value.status == rq.RQ_ERR_INVALID_ARG
+
+
+def test_unused_cache_memory_full_of_nans_does_not_leak():
+    """A cache much larger than the prompt whose memory holds NaN bit patterns everywhere the prefill did not write:
+    copies of whole chunks read some of it (the pages after the prompt's end); neither the routing nor the attention may
+    pick any of it up."""
+    w = wl.Workload("moba-nan", B=1, H=2, D=128, T=1000, seed=17)
+    block, K = 64, 4
+    cache = rq.Cache(w.B, w.H, w.D, w.S, 4096, w.dtype, w.gdtype)
+    cache.kv.fill_(0xFF)
+    cache.meta.fill_(0xFF)
+    k, v, g = wl.make_prefill(w, DEV, w.T)
+    rq.rq_build_cache(cache.handle, k, v, g)
+    q = prompt_queries(w, w.T, 3)
+    o = torch.full((w.B, w.T, w.H, w.D), float("nan"), dtype=w.dtype, device=DEV)
+    blocks = torch.empty(w.B, w.H, w.T, K, dtype=torch.int32, device=DEV)
+    means = torch.empty(w.B, w.H, (w.T + block - 1) // block, w.D, dtype=torch.float32, device=DEV)
+    scratch = torch.empty(rq.rq_moba_scratch_bytes(cache.handle, block, K), dtype=torch.uint8, device=DEV)
+    rq.rq_moba_prefill(cache.handle, q, block, K, 0.0, o, blocks, means, scratch)
+    torch.cuda.synchronize()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(means).all()
+    for h in range(w.H):
+        check_head(w, cache, q, o, blocks, means, 0, h, block, K, w.D ** -0.5, sample_positions(w.T, block, 8, h))

@@ -255,3 +255,20 @@ def test_128k_prompt_sampled_heads():
         src = check_head_selection(cache, b, h, qw, W, keep, idx, imp, w.D ** -0.5)
         sel = got[b, h].astype(np.int64)
         check_compaction(src, small, b, h, sel, parity.f64(cache.state_view()[b, h]))
+
+
+def test_unused_cache_memory_full_of_nans_does_not_leak():
+    """A cache much larger than the prompt whose memory holds NaN bit patterns everywhere the prefill did not write: the
+    tile copies of the last tiles read some of it; importances and the selection must not pick any of it up."""
+    w = wl.Workload("snapkv-nan", B=1, H=2, D=128, T=1000, seed=19)
+    cache = rq.Cache(w.B, w.H, w.D, w.S, 4096, w.dtype, w.gdtype)
+    cache.kv.fill_(0xFF)
+    cache.meta.fill_(0xFF)
+    k, v, g = wl.make_prefill(w, DEV, w.T)
+    rq.rq_build_cache(cache.handle, k, v, g)
+    W, keep = 64, 200
+    qw = window_queries(w, W, 5)
+    idx, imp = snap_select(cache, qw, W, keep)
+    assert torch.isfinite(imp).all()
+    for h in range(w.H):
+        check_head_selection(cache, 0, h, qw, W, keep, idx, imp, w.D ** -0.5)
