@@ -11,10 +11,9 @@
  *   rqo_block_means    rho(K~_j): the mean of the stored decayed keys of block j
  *   rqo_moba_scores    s(q_t, rho_j) = q_t . rho_j for the blocks before the query's own
  *
- * The TopK of Eq. 3 with the first block and the local block always included is
- * rqo_select_pages (the same rule as for Quest, App. A.1: "For both Quest and MoBA, we
- * always include the first block and local blocks"), and Eq. 4 over the chosen tokens is
- * rqo_token_attention; oracle/__init__.py chains them per query.
+ * The TopK of Eq. 3 with the first block and the local block always taken is
+ * rqo_select_pages (App. A.1 states that rule for Quest and MoBA alike), and Eq. 4 over
+ * the chosen tokens is rqo_token_attention; oracle/__init__.py chains them per query.
  *
  * Readings where the paper is silent: the candidates of the query at position t are the
  * COMPLETE blocks before its own (block j < t / B); the query's own block is the local
