@@ -103,6 +103,8 @@ def test_paper_settings_on_4k_prompts(block, K):
     (1, 2, 128, 1500, 16, 256, 3, torch.bfloat16),    # blocks of 256
     (1, 2, 64, 12000, 16, 64, 9, torch.bfloat16),     # 188 blocks: representatives read from global memory, arg-max rounds
     (1, 1, 128, 9000, 16, 64, 20, torch.float32),     # the same on an fp32 cache
+    (1, 2, 128, 65536, 16, 64, 64, torch.bfloat16),   # 1024 blocks, 64 per query: a long prompt at budget 1/16
+    (1, 1, 64, 131072, 64, 128, 16, torch.bfloat16),  # 1024 blocks of 128 on pages of 64
 ])
 def test_shapes_blocks_and_ragged_sizes(B, H, D, T, S, block, K, dtype):
     w = wl.Workload("moba-small", B=B, H=H, D=D, T=T, S=S, dtype=dtype, seed=T + K)
