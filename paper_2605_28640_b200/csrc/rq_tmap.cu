@@ -26,6 +26,7 @@ TensorMapEncodeTiled tensor_map_encoder()
 cudaError_t cache_tensor_map(CUtensorMap *out, const void *kv, int D, int S, int64_t pages_total, int positions)
 {
     if (positions % S != 0 || D % 64 != 0) return cudaErrorInvalidValue;
+    if (pages_total < 1 || pages_total >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;   // box coordinates are 32-bit
     const TensorMapEncodeTiled encode = tensor_map_encoder();
     if (!encode) return cudaErrorNotSupported;
     const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)S, 2, (cuuint64_t)pages_total};
