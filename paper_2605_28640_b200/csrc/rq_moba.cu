@@ -317,8 +317,9 @@ __global__ void __launch_bounds__(kMobaQueries * 32) moba_attend_kernel(const T 
 // accumulators, so everything per query (mask, running maximum, sum, weights) is per thread.  The chunks
 // (64 positions) of the blocks ANY of the 128 queries chose are walked twice:
 //   pass 1   S = Q K^T (tcgen05.mma, 128 x 64, fp32 in tensor memory); a thread masks the chunk for its query
-//            (block not chosen / positions after the query) and keeps the running maximum and sum of exponentials
-//   pass 2   S again; the thread turns its row into normalised weights, rounds them to bf16 and writes them
+//            (block not chosen / positions after the query) and keeps the running maximum
+//   pass 2   S again; the thread turns its row into weights relative to the query's maximum (summed in fp32 for
+//            the final division), rounds them to bf16 and writes them
 //            into tensor memory (tcgen05.st) as the A operand of the second product, O += P V (128 x D, the values
 //            as an MN-major operand straight from the cache's rows), accumulated in tensor memory over all chunks
 // One thread of a ninth warp starts the tensor-map copies (keys and values of a chunk, two stages each) and the
@@ -526,15 +527,11 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             if (g == n) {
                 // pass 2 walks the same chunks again; first the two halves of a query's statistics are merged
                 c = -1;
-                stat[ch][lq] = make_float2(m, l);
+                stat[ch][lq] = make_float2(m, 0.0f);
                 mbar_arrive(&stat_ready);
                 ok = mbar_wait(&stat_ready, 0u);
                 if (!__all_sync(FULLMASK, ok)) break;
-                const float2 other = stat[ch ^ 1][lq];
-                const float mn = fmaxf(m, other.x);
-                if (mn > -CUDART_INF_F) l = l * exp2_fast(m - mn) + other.y * exp2_fast(other.x - mn);
-                m = mn;
-                inv_l = l > 0.0f ? 1.0f / l : 0.0f;
+                m = fmaxf(m, stat[ch ^ 1][lq].x);    // the query's maximum over everything it attends
             }
             c = next_chunk(c);
             const int64_t p0 = (int64_t)c * kMobaChunk + ch * 32;    // first of this thread's 32 positions
@@ -553,27 +550,21 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             float v[32];
             tmem_ld32(tl + (uint32_t)(g % NSB) * ACC_S + (uint32_t)(ch * 32), v);
             if (hh < 0) {
-                if (nv > 0) {
+                if (nv > 0) {                        // pass 1 only needs the maximum: the weights are summed in pass 2
                     float tm = -CUDART_INF_F;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        v[i] = i < nv ? v[i] * scale_log2 : -CUDART_INF_F;
-                        tm = fmaxf(tm, v[i]);
-                    }
-                    const float mn = fmaxf(m, tm);
-                    float sum = 0.0f;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) sum += exp2_fast(v[i] - mn);
-                    l = l * exp2_fast(m - mn) + sum;
-                    m = mn;
+                    for (int i = 0; i < 32; ++i) tm = fmaxf(tm, i < nv ? v[i] : -CUDART_INF_F);
+                    m = fmaxf(m, tm * scale_log2);
                 }
             } else {
-                // normalised weights of 32 positions, rounded to bf16: 16 columns of this query's lane
+                // weights of 32 positions relative to the query's maximum (at most 1), rounded to bf16: 16 columns of
+                // this query's lane; their sum is kept in fp32 and divides the output at the end
                 uint32_t w[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float a = i < nv ? exp2_fast(fmaf(v[i], scale_log2, -m)) * inv_l : 0.0f;
-                    const float bq = i + 1 < nv ? exp2_fast(fmaf(v[i + 1], scale_log2, -m)) * inv_l : 0.0f;
+                    const float a = i < nv ? exp2_fast(fmaf(v[i], scale_log2, -m)) : 0.0f;
+                    const float bq = i + 1 < nv ? exp2_fast(fmaf(v[i + 1], scale_log2, -m)) : 0.0f;
+                    l += a + bq;
                     w[i >> 1] = pack2_bf16(a, bq);
                 }
                 tmem_st16(tl + OFF_P + (uint32_t)(hh & 1) * P_COLS + (uint32_t)(ch * 16), w);
@@ -600,8 +591,16 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 mbar_arrive(&p_ready[hh & 1]);
             }
         }
-        // the output once the last product is complete: each of a query's two threads writes half of the channels
+        // the output once the last product is complete: each of a query's two threads writes half of the channels,
+        // divided by the sum of the query's weights (the two threads' sums, exchanged through shared memory)
         if (__all_sync(FULLMASK, ok)) {
+            stat[ch][lq] = make_float2(l, 0.0f);
+            mbar_arrive(&stat_ready);
+            ok = mbar_wait(&stat_ready, 1u);
+        }
+        if (__all_sync(FULLMASK, ok)) {
+            l += stat[ch ^ 1][lq].x;
+            inv_l = l > 0.0f ? 1.0f / l : 0.0f;
             ok = mbar_wait(&pv_done[(n - 1) & 1], (uint32_t)(((n - 1) >> 1) & 1));
             if (__all_sync(FULLMASK, ok)) {
                 tcgen05_after_sync();
@@ -613,8 +612,9 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                         bf16 *orow = o + (((int64_t)b * len + tq) * H + h) * D + cb;
 #pragma unroll
                         for (int i = 0; i < 32; i += 8)
-                            *reinterpret_cast<uint4 *>(orow + i) = make_uint4(pack2_bf16(v[i], v[i + 1]), pack2_bf16(v[i + 2], v[i + 3]),
-                                                                              pack2_bf16(v[i + 4], v[i + 5]), pack2_bf16(v[i + 6], v[i + 7]));
+                            *reinterpret_cast<uint4 *>(orow + i) =
+                                make_uint4(pack2_bf16(v[i] * inv_l, v[i + 1] * inv_l), pack2_bf16(v[i + 2] * inv_l, v[i + 3] * inv_l),
+                                           pack2_bf16(v[i + 4] * inv_l, v[i + 5] * inv_l), pack2_bf16(v[i + 6] * inv_l, v[i + 7] * inv_l));
                     }
                 }
             }
