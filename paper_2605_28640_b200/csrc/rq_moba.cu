@@ -316,8 +316,9 @@ __global__ void __launch_bounds__(kMobaQueries * 32) moba_attend_kernel(const T 
 // Grid (ceil(T / 128), heads).  A CTA owns 128 consecutive queries of a head: they are the 128 lanes of the
 // accumulators, so everything per query (mask, running maximum, sum, weights) is per thread.  The chunks
 // (64 positions) of the blocks ANY of the 128 queries chose are walked twice:
-//   pass 1   S = Q K^T (tcgen05.mma, 128 x 64, fp32 in tensor memory); a thread masks the chunk for its query
-//            (block not chosen / positions after the query) and keeps the running maximum
+//   pass 1   S = Q K^T for two chunks at a time (tcgen05.mma, 128 x 128, fp32 in tensor memory, two accumulators);
+//            a thread masks its chunk for its query (block not chosen / positions after the query) and keeps the
+//            running maximum
 //   pass 2   S again; the thread turns its row into weights relative to the query's maximum (summed in fp32 for
 //            the final division), rounds them to bf16 and writes them
 //            into tensor memory (tcgen05.st) as the A operand of the second product, O += P V (128 x D, the values
@@ -364,13 +365,15 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
 {
     using G = MobaMmaGeom<D>;
     constexpr int NST = kMobaMmaStages;
-    // tensor memory: one score accumulator of 64 columns, the output (D columns), two weight buffers of 32 columns
-    // (64 positions as bf16 pairs): 256 columns, and with two key and two value stages 97 KB of shared memory, so
-    // that TWO CTAs share an SM: each CTA's chunk is a chain of dependent steps, and the two chains overlap
-    constexpr int NSB = 1;                                       // score accumulators
-    constexpr uint32_t ACC_S = 64, OFF_O = 64, OFF_P = 64 + D, P_COLS = 32, TCOLS = 256;
+    static_assert(NST == 2, "pass 1 uses the key region and the value region as its two stages of two chunks each");
+    // tensor memory, 256 columns.  Pass 1: two score accumulators of 128 columns.  Pass 2: one score accumulator of 64
+    // columns, the output (D columns), two weight buffers of 32 columns (64 positions as bf16 pairs).  With two key and
+    // two value stages a CTA needs 97 KB of shared memory, so that TWO CTAs share an SM: each CTA's chunk is a chain of
+    // dependent steps, and the two chains overlap
+    constexpr uint32_t OFF_O = 64, OFF_P = 64 + D, P_COLS = 32, TCOLS = 256;
     extern __shared__ __align__(1024) unsigned char msm_raw[];
     __shared__ __align__(8) uint64_t full_k[NST], full_v[NST], s_ready[2], s_free[2], p_ready[2], pv_done[2], stat_ready;
+    __shared__ __align__(8) uint64_t full1[2], s1_ready[2], s1_free[2];    // pass 1: stage landed, scores ready, scores read
     __shared__ float2 stat[2][kMobaMmaQueries];                          // pass 1: a query's statistics from its two threads
     __shared__ uint32_t tbase;
     unsigned char *msm = msm_raw + ((1024u - (smem_addr(msm_raw) & 1023u)) & 1023u);
@@ -392,6 +395,9 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             mbar_init(&pv_done[s], 1);
             mbar_init(&s_free[s], kMobaMmaWarps * 32);
             mbar_init(&p_ready[s], kMobaMmaWarps * 32);
+            mbar_init(&full1[s], 1);
+            mbar_init(&s1_ready[s], 1);
+            mbar_init(&s1_free[s], kMobaMmaWarps * 32);
         }
         mbar_init(&stat_ready, kMobaMmaWarps * 32);
         mbar_init_fence();
@@ -439,12 +445,11 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
 
     if (warp == kMobaMmaWarps) {
         if (lane == 0) {
-            // ---- copies and products.  g counts the score products over both passes (0 .. 2n-1), hh the chunks of pass 2.
-            int ck_issue = -1, cv_issue = -1;        // chunk walk of the key copies (both passes) and of the value copies
+            // ---- copies and products; hh counts the chunks of pass 2
+            int ck_issue = -1, cv_issue = -1;        // chunk walk of pass 2's key copies and value copies
             int gk_issued = 0, hv_issued = 0, gk_landed = 0, hv_landed = 0;
             auto issue_k = [&]() {                   // keys of the next chunk of the walk into stage gk_issued % NST
                 ck_issue = next_chunk(ck_issue);
-                if (ck_issue >= n_chunks_all) ck_issue = next_chunk(-1);      // pass 2 walks the same chunks again
                 const int st = gk_issued % NST;
                 const int page = (int)((int64_t)bh * page_cap + ((int64_t)ck_issue * kMobaChunk) / S);
                 mbar_arrive_expect_tx(&full_k[st], G::KC_BYTES);
@@ -477,31 +482,73 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 umma_commit(&pv_done[hh & 1]);
                 return true;
             };
-            for (int s = 0; s < NST && s < 2 * n; ++s) issue_k();
-            for (int s = 0; s < NST && s < n; ++s) issue_v();
-            constexpr uint32_t idesc_s = umma_idesc_bf16(128, kMobaChunk);
+            // ---- pass 1: the queries' maxima.  Two chunks (128 keys) per product; the key region and the value region
+            // are its two stages; two accumulators of 128 columns (the columns pass 2 uses for scores, output and weights)
             const uint32_t qa = smem_addr(qs);
+            const int n1 = (n + 1) / 2;
+            int c1 = -1, issued1 = 0, landed1 = 0;
+            auto issue1 = [&](int it) {
+                unsigned char *dst = (it & 1) ? vst : kst;
+                const int cnt = min(2, n - 2 * it);
+                mbar_arrive_expect_tx(&full1[it & 1], (uint32_t)cnt * G::KC_BYTES);
+                for (int u = 0; u < cnt; ++u) {
+                    c1 = next_chunk(c1);
+                    const int page = (int)((int64_t)bh * page_cap + ((int64_t)c1 * kMobaChunk) / S);
+#pragma unroll
+                    for (int hf = 0; hf < G::HALVES; ++hf)
+                        tma_load_4d(dst + hf * (128 * 128) + u * (kMobaChunk * 128), &tmap, hf * 64, 0, 0, page, &full1[it & 1]);
+                }
+                issued1 = it + 1;
+            };
+            issue1(0);
+            if (n1 > 1) issue1(1);
+            constexpr uint32_t idesc_1 = umma_idesc_bf16(128, 2 * kMobaChunk);
 #pragma unroll 1
-            for (int g = 0; g < 2 * n && ok; ++g) {
-                if (g >= NSB) ok = mbar_wait(&s_free[g % NSB], (uint32_t)(((g / NSB) - 1) & 1));
-                ok = ok && mbar_wait(&full_k[g % NST], (uint32_t)((g / NST) & 1));
+            for (int it = 0; it < n1 && ok; ++it) {
+                if (it >= 2) ok = mbar_wait(&s1_free[it & 1], (uint32_t)(((it >> 1) - 1) & 1));
+                ok = ok && mbar_wait(&full1[it & 1], (uint32_t)((it >> 1) & 1));
                 if (!ok) break;
-                gk_landed = g + 1;
+                landed1 = it + 1;
                 tcgen05_after_sync();
-                const uint32_t ka = smem_addr(kst + (size_t)(g % NST) * G::KC_BYTES);
+                const uint32_t sa = smem_addr((it & 1) ? vst : kst);
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    umma_bf16(tb + (uint32_t)(g % NSB) * ACC_S, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
-                              umma_desc_sw128(ka + (k >> 2) * (kMobaChunk * 128) + (k & 3) * 32), idesc_s, k > 0);
-                umma_commit(&s_ready[g % NSB]);
-                const int hh = g - n;                // pass 2: the chunk whose scores were just started
-                if (hh >= 1) ok = product_pv(hh - 1);
-                // refills: the key stage of product g - 1 (complete: its scores were read), the value stage of chunk hh - 2
-                // once the second product of that chunk is complete
-                if (ok && g >= 1 && g - 1 + NST < 2 * n) {
-                    ok = true;                       // (one score accumulator: product g - 1 is complete, its scores have been read)
-                    if (ok) issue_k();
+                    umma_bf16(tb + (uint32_t)(it & 1) * 128u, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
+                              umma_desc_sw128(sa + (k >> 2) * (128 * 128) + (k & 3) * 32), idesc_1, k > 0);
+                umma_commit(&s1_ready[it & 1]);
+                if (it >= 1 && it + 1 < n1) {        // the stage of product it - 1 takes the chunks of product it + 1
+                    ok = mbar_wait(&s1_ready[(it - 1) & 1], (uint32_t)(((it - 1) >> 1) & 1));
+                    if (ok) issue1(it + 1);
                 }
+            }
+            // pass 2 reuses the stages and the tensor memory: the last products are complete and their scores read
+            for (int it = max(0, n1 - 2); it < n1 && ok; ++it)
+                ok = mbar_wait(&s1_ready[it & 1], (uint32_t)((it >> 1) & 1)) && mbar_wait(&s1_free[it & 1], (uint32_t)((it >> 1) & 1));
+            for (int k = landed1; k < issued1; ++k) mbar_wait(&full1[k & 1], (uint32_t)((k >> 1) & 1));
+
+            // ---- pass 2: weights and output, a chunk per step
+            if (ok) {
+                for (int s = 0; s < NST && s < n; ++s) issue_k();
+                for (int s = 0; s < NST && s < n; ++s) issue_v();
+            }
+            constexpr uint32_t idesc_s = umma_idesc_bf16(128, kMobaChunk);
+#pragma unroll 1
+            for (int hh = 0; hh < n && ok; ++hh) {
+                if (hh >= 1) ok = mbar_wait(&s_free[0], (uint32_t)((hh - 1) & 1));
+                ok = ok && mbar_wait(&full_k[hh % NST], (uint32_t)((hh / NST) & 1));
+                if (!ok) break;
+                gk_landed = hh + 1;
+                tcgen05_after_sync();
+                const uint32_t ka = smem_addr(kst + (size_t)(hh % NST) * G::KC_BYTES);
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k)
+                    umma_bf16(tb, umma_desc_sw128(qa + (k >> 2) * (128 * 128) + (k & 3) * 32),
+                              umma_desc_sw128(ka + (k >> 2) * (kMobaChunk * 128) + (k & 3) * 32), idesc_s, k > 0);
+                umma_commit(&s_ready[0]);
+                if (hh >= 1) ok = product_pv(hh - 1);
+                // refills: the key stage of chunk hh - 1 (its scores have been read), the value stage of chunk hh - 2 once
+                // the second product of that chunk is complete
+                if (ok && hh >= 1 && hh - 1 + NST < n) issue_k();
                 if (ok && hh >= 2 && hh - 2 + NST < n) {
                     ok = mbar_wait(&pv_done[(hh - 2) & 1], (uint32_t)(((hh - 2) >> 1) & 1));
                     if (ok) issue_v();
@@ -522,41 +569,64 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
         const uint32_t *mymask = qmask + lq * words;
         float m = -CUDART_INF_F, l = 0.0f, inv_l = 0.0f;
         int c = -1;
+        // ---- pass 1: the maximum of the scores this query attends.  A product covers two chunks; of a query's two
+        // threads the first takes the first chunk, the second the other one.
+        const int n1 = (n + 1) / 2;
 #pragma unroll 1
-        for (int g = 0; g < 2 * n; ++g) {
-            if (g == n) {
-                // pass 2 walks the same chunks again; first the two halves of a query's statistics are merged
-                c = -1;
-                stat[ch][lq] = make_float2(m, 0.0f);
-                mbar_arrive(&stat_ready);
-                ok = mbar_wait(&stat_ready, 0u);
-                if (!__all_sync(FULLMASK, ok)) break;
-                m = fmaxf(m, stat[ch ^ 1][lq].x);    // the query's maximum over everything it attends
+        for (int it = 0; it < n1; ++it) {
+            const int ca = next_chunk(c), cb2 = 2 * it + 1 < n ? next_chunk(ca) : -1;
+            c = cb2 >= 0 ? cb2 : ca;
+            const int cm = ch == 0 ? ca : cb2;       // this thread's chunk (none: -1)
+            int nv = 0;
+            if (cm >= 0 && tq < len) {
+                const int j = (int)(((int64_t)cm * kMobaChunk) / block);
+                if ((mymask[j >> 5] >> (j & 31)) & 1u) nv = (int)max((int64_t)0, min((int64_t)kMobaChunk, tq - (int64_t)cm * kMobaChunk + 1));
             }
+            ok = mbar_wait(&s1_ready[it & 1], (uint32_t)((it >> 1) & 1));
+            if (!__all_sync(FULLMASK, ok)) break;
+            tcgen05_after_sync();
+#pragma unroll 1
+            for (int cb = 0; cb < kMobaChunk; cb += 32) {
+                float v[32];
+                tmem_ld32(tl + (uint32_t)(it & 1) * 128u + (uint32_t)(ch * kMobaChunk + cb), v);
+                if (cb < nv) {
+                    float tm = -CUDART_INF_F;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) tm = fmaxf(tm, cb + i < nv ? v[i] : -CUDART_INF_F);
+                    m = fmaxf(m, tm * scale_log2);
+                }
+            }
+            tcgen05_before_sync();
+            mbar_arrive(&s1_free[it & 1]);
+        }
+        // the query's maximum over everything it attends: its two threads exchange theirs
+        if (__all_sync(FULLMASK, ok)) {
+            stat[ch][lq] = make_float2(m, 0.0f);
+            mbar_arrive(&stat_ready);
+            ok = mbar_wait(&stat_ready, 0u);
+            if (__all_sync(FULLMASK, ok)) m = fmaxf(m, stat[ch ^ 1][lq].x);
+        }
+        // ---- pass 2: the same chunks one by one; of a query's two threads each takes 32 of a chunk's positions
+        c = -1;
+#pragma unroll 1
+        for (int hh = 0; hh < n; ++hh) {
+            if (!__all_sync(FULLMASK, ok)) break;
             c = next_chunk(c);
             const int64_t p0 = (int64_t)c * kMobaChunk + ch * 32;    // first of this thread's 32 positions
             const int j = (int)(((int64_t)c * kMobaChunk) / block);
             // positions this query attends among them: none if it did not choose the block, else those up to its own
             int nv = 0;
             if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)32, tq - p0 + 1));
-            ok = mbar_wait(&s_ready[g % NSB], (uint32_t)((g / NSB) & 1));
+            ok = mbar_wait(&s_ready[0], (uint32_t)(hh & 1));
             if (!__all_sync(FULLMASK, ok)) break;
             tcgen05_after_sync();
-            const int hh = g - n;
             if (hh >= 2) {                           // the weights buffer hh & 1 was read by the product of chunk hh - 2
                 ok = mbar_wait(&pv_done[hh & 1], (uint32_t)(((hh - 2) >> 1) & 1));
                 if (!__all_sync(FULLMASK, ok)) break;
             }
             float v[32];
-            tmem_ld32(tl + (uint32_t)(g % NSB) * ACC_S + (uint32_t)(ch * 32), v);
-            if (hh < 0) {
-                if (nv > 0) {                        // pass 1 only needs the maximum: the weights are summed in pass 2
-                    float tm = -CUDART_INF_F;
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) tm = fmaxf(tm, i < nv ? v[i] : -CUDART_INF_F);
-                    m = fmaxf(m, tm * scale_log2);
-                }
-            } else {
+            tmem_ld32(tl + (uint32_t)(ch * 32), v);
+            {
                 // weights of 32 positions relative to the query's maximum (at most 1), rounded to bf16: 16 columns of
                 // this query's lane; their sum is kept in fp32 and divides the output at the end
                 uint32_t w[16];
@@ -570,8 +640,8 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 tmem_st16(tl + OFF_P + (uint32_t)(hh & 1) * P_COLS + (uint32_t)(ch * 16), w);
             }
             tcgen05_before_sync();
-            mbar_arrive(&s_free[g % NSB]);
-            if (hh >= 0 && (int64_t)c * kMobaChunk + kMobaChunk > len) {
+            mbar_arrive(&s_free[0]);                 // this thread has read the scores
+            if ((int64_t)c * kMobaChunk + kMobaChunk > len) {
                 // the prompt ends inside this chunk: the value rows past its end hold whatever the cache's memory held;
                 // a weight of zero would not stop a NaN there, so those rows are cleared once they have landed
                 ok = mbar_wait(&full_v[hh % NST], (uint32_t)((hh / NST) & 1));
@@ -585,11 +655,9 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // ordinary stores, read by the tensor core
             }
-            if (hh >= 0) {
-                tmem_st_wait();                      // the weights are in tensor memory
-                tcgen05_before_sync();
-                mbar_arrive(&p_ready[hh & 1]);
-            }
+            tmem_st_wait();                          // the weights are in tensor memory
+            tcgen05_before_sync();
+            mbar_arrive(&p_ready[hh & 1]);
         }
         // the output once the last product is complete: each of a query's two threads writes half of the channels,
         // divided by the sum of the query's weights (the two threads' sums, exchanged through shared memory)
