@@ -33,7 +33,7 @@ namespace {
 
 constexpr int kMobaChunk = 64;                 // positions that pass through shared memory at a time
 constexpr int kMobaQueries = 16;               // queries (warps) of one attention CTA
-constexpr int kMobaRouteWarps = 8;             // queries (warps) of one routing CTA
+constexpr int kMobaRouteWarps = 16;            // queries (warps) of one routing CTA
 constexpr int kMobaMaxBlocks = 2048;           // blocks of a prompt at most
 constexpr unsigned FULLMASK = 0xffffffffu;
 
@@ -60,8 +60,41 @@ __global__ void moba_means_kernel(const T *kv, int64_t page_cap, int S, int D, i
     means[((int64_t)bh * nb + j) * D + c] = s / (float)(hi - lo);
 }
 
+// Ranking by counting for one warp: candidates are the blocks c_lo .. c_hi - 1 with scores sc[]; lane l owns the
+// candidates c_lo + l + 32 r, r < R.  Sets the mask bits of the candidates whose rank is below `want`.
+template <int R>
+__device__ __forceinline__ void moba_rank_take(const float *sc, uint32_t *mask, int c_lo, int c_hi, int want, int lane)
+{
+    float mv[R];
+    int rank[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int j = c_lo + lane + 32 * r;
+        mv[r] = j < c_hi ? sc[j] : 0.0f;
+        rank[r] = 0;
+    }
+    for (int i = c_lo; i < c_hi; ++i) {
+        const float ov = sc[i];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int j = c_lo + lane + 32 * r;
+            rank[r] += (ov > mv[r] || (ov == mv[r] && i < j)) ? 1 : 0;
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int j = c_lo + lane + 32 * r;
+        const unsigned take = __ballot_sync(0xffffffffu, j < c_hi && rank[r] < want);   // blocks c_lo + 32 r + bit
+        if (lane == 0 && take) {
+            const int p = c_lo + 32 * r;
+            mask[p >> 5] |= take << (p & 31);
+            if (p & 31) mask[(p >> 5) + 1] |= take >> (32 - (p & 31));
+        }
+    }
+}
+
 // ---------------------------------------------------------------- routing
-// Grid (ceil(T / 8), heads); a warp per query.  Shared memory per warp: the query (D floats), the
+// Grid (ceil(T / 16), heads); a warp per query.  Shared memory per warp: the query (D floats), the
 // scores of the candidate blocks (nb floats), the chosen blocks as a bit mask (nb / 32 words); and,
 // when they fit (STAGED), the head's representatives for the whole CTA, rows padded by four floats so
 // that the lanes of a quarter-warp, each reading its own row, hit different banks.
@@ -129,34 +162,12 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
     __syncwarp();
     if (c_hi - c_lo <= 4 * 32 && want >= 8) {
         // few candidates and more than a handful to take (a round per taken block is cheaper otherwise): a
-        // candidate's rank is the number of candidates that beat it (higher score, or the same
-        // score and a lower block); a lane ranks its own (at most four) against all of them, read as broadcasts
-        float mv[4];
-        int rank[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int j = c_lo + lane + 32 * r;
-            mv[r] = j < c_hi ? sc[j] : 0.0f;
-            rank[r] = 0;
-        }
-        for (int i = c_lo; i < c_hi; ++i) {
-            const float ov = sc[i];
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const int j = c_lo + lane + 32 * r;
-                rank[r] += (ov > mv[r] || (ov == mv[r] && i < j)) ? 1 : 0;
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int j = c_lo + lane + 32 * r;
-            const unsigned take = __ballot_sync(FULLMASK, j < c_hi && rank[r] < want);   // blocks c_lo + 32 r + bit
-            if (lane == 0 && take) {
-                const int p = c_lo + 32 * r;
-                mask[p >> 5] |= take << (p & 31);
-                if (p & 31) mask[(p >> 5) + 1] |= take >> (32 - (p & 31));
-            }
-        }
+        // candidate's rank is the number of candidates that beat it (higher score, or the same score and a lower
+        // block); a lane ranks its own (one, two or four) against all of them, read as broadcasts
+        const int ncand = c_hi - c_lo;
+        if (ncand <= 32) moba_rank_take<1>(sc, mask, c_lo, c_hi, want, lane);
+        else if (ncand <= 64) moba_rank_take<2>(sc, mask, c_lo, c_hi, want, lane);
+        else moba_rank_take<4>(sc, mask, c_lo, c_hi, want, lane);
         __syncwarp();
     } else {
     // the `want` best candidates, one per round: every lane's best of its blocks, then the warp's best;
