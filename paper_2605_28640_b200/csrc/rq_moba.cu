@@ -5,18 +5,21 @@
 // block (cut at the query's position) are always among them and count inside the budget.
 //
 //   moba_means_kernel    per (head, block): the mean of the block's stored keys, fp32
-//   moba_route_kernel    per (head, query), one warp: scores q . mean of the complete blocks before the
-//                        query's own (a lane per block), then the budget's best by repeated arg-max
-//                        (equal scores to the lower block), the list written ascending
-//   moba_attend_kernel   per (head, 16 consecutive queries), a warp per query: the blocks any of the 16
-//                        queries chose pass through shared memory once, 64 positions at a time
-//                        (cp.async, two buffers); a warp folds a chunk into its online softmax only if
-//                        its own query chose the block (the arithmetic is the decode path's tile
-//                        routine)
-//
-// This is the first correct form of the path: plain fp32 FMA work.  The attention is a dense
-// contraction per (query block, KV block) and belongs on the tensor cores like the SnapKV passes; the
-// routing on the query side makes that a larger kernel than this one.
+//   moba_route_kernel    per (head, 16 consecutive queries), a warp per query: scores q . mean of the
+//                        complete blocks before the query's own (a lane per block; the head's
+//                        representatives staged in shared memory once per CTA when they fit), then the
+//                        budget's best (equal scores to the lower block) by counting each candidate's
+//                        rank, or by repeated arg-max when the budget is small or the candidates many;
+//                        the list written ascending
+//   moba_mma_kernel      bf16 caches.  Per (head, 128 consecutive queries): both contractions on the
+//                        tensor cores (tcgen05.mma, accumulators and the weights in tensor memory),
+//                        the chunks of the blocks any of the 128 queries chose walked twice (row
+//                        maxima, then weights and O += P V); see the comment above the kernel
+//   moba_attend_kernel   fp32 caches.  Per (head, 16 consecutive queries), a warp per query: the blocks
+//                        any of the 16 queries chose pass through shared memory once, 64 positions at a
+//                        time (cp.async, two buffers); a warp folds a chunk into its online softmax
+//                        only if its own query chose the block (plain fp32 FMA work; the arithmetic is
+//                        the decode path's tile routine)
 #include <limits.h>
 #include <math_constants.h>
 
