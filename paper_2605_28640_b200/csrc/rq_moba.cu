@@ -59,30 +59,51 @@ __global__ void moba_means_kernel(const T *kv, int64_t page_cap, int S, int D, i
     const int j = blockIdx.x, bh = blockIdx.y, c = threadIdx.x;
     const int64_t lo = (int64_t)j * block, hi = min(lo + block, len);
     float s = 0.0f;
-    for (int64_t p = lo; p < hi; ++p) s += load1<T>(kv + ((((int64_t)bh * page_cap + p / S) * 2) * S + p % S) * D + c);
+    int64_t p = lo;
+    // sixteen loads in flight at a time (a page holds a multiple of 16 positions and lo is a multiple of 64, so
+    // a run of 16 stays inside one page); the additions keep the order of the positions
+    for (; p + 16 <= hi; p += 16) {
+        const T *src = kv + ((((int64_t)bh * page_cap + p / S) * 2) * S + p % S) * D + c;
+        float x[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = load1<T>(src + (int64_t)i * D);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) s += x[i];
+    }
+    for (; p < hi; ++p) s += load1<T>(kv + ((((int64_t)bh * page_cap + p / S) * 2) * S + p % S) * D + c);
     means[((int64_t)bh * nb + j) * D + c] = s / (float)(hi - lo);
 }
 
 // Ranking by counting for one warp: candidates are the blocks c_lo .. c_hi - 1 with scores sc[]; lane l owns the
-// candidates c_lo + l + 32 r, r < R.  Sets the mask bits of the candidates whose rank is below `want`.
+// candidates c_lo + l + 32 r, r < R.  Sets the mask bits of the candidates whose rank is below `want`.  A
+// candidate beats another with a higher score, or the same score and a lower block: one unsigned 64-bit
+// comparison of (order-preserving image of the score, complement of the block).  The scores are replaced by
+// their images in place.
 template <int R>
-__device__ __forceinline__ void moba_rank_take(const float *sc, uint32_t *mask, int c_lo, int c_hi, int want, int lane)
+__device__ __forceinline__ void moba_rank_take(float *sc, uint32_t *mask, int c_lo, int c_hi, int want, int lane)
 {
-    float mv[R];
+    uint32_t *key = reinterpret_cast<uint32_t *>(sc);
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+        const int j = c_lo + lane + 32 * r;
+        if (j < c_hi) {
+            const uint32_t b = __float_as_uint(sc[j] + 0.0f);          // -0 becomes +0
+            key[j] = b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
+        }
+    }
+    __syncwarp();
+    unsigned long long mine[R];
     int rank[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const int j = c_lo + lane + 32 * r;
-        mv[r] = j < c_hi ? sc[j] : 0.0f;
+        mine[r] = j < c_hi ? ((unsigned long long)key[j] << 32) | (uint32_t)~j : ~0ull;
         rank[r] = 0;
     }
     for (int i = c_lo; i < c_hi; ++i) {
-        const float ov = sc[i];
+        const unsigned long long other = ((unsigned long long)key[i] << 32) | (uint32_t)~i;
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int j = c_lo + lane + 32 * r;
-            rank[r] += (ov > mv[r] || (ov == mv[r] && i < j)) ? 1 : 0;
-        }
+        for (int r = 0; r < R; ++r) rank[r] += other > mine[r] ? 1 : 0;
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
@@ -149,17 +170,16 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
         const int j = j0 + lane;
         if (j < c_hi) {
             const float4 *row = reinterpret_cast<const float4 *>(mh + (int64_t)j * LDM);
-            float s = 0.0f;
+            // packed pairs: the even and the odd channels are summed apart and added at the end
+            float2 s2 = make_float2(0.0f, 0.0f);
 #pragma unroll 8
             for (int i = 0; i < D / 4; ++i) {
                 const float4 m4 = STAGED ? row[i] : __ldg(row + i);
                 const float4 q4 = *reinterpret_cast<const float4 *>(qs + 4 * i);
-                s = fmaf(q4.x, m4.x, s);
-                s = fmaf(q4.y, m4.y, s);
-                s = fmaf(q4.z, m4.z, s);
-                s = fmaf(q4.w, m4.w, s);
+                s2 = fma2(make_float2(q4.x, q4.y), make_float2(m4.x, m4.y), s2);
+                s2 = fma2(make_float2(q4.z, q4.w), make_float2(m4.z, m4.w), s2);
             }
-            sc[j] = s;
+            sc[j] = s2.x + s2.y;
         }
     }
     __syncwarp();
