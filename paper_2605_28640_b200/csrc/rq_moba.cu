@@ -392,6 +392,28 @@ __device__ __forceinline__ uint32_t pack2_bf16(float a, float b)
     return *reinterpret_cast<const uint32_t *>(&h);
 }
 
+// Walk over the 64-position chunks of the chosen blocks in ascending order: (block, chunk inside the block).
+// A block holds cpb chunks; the walk ends (returns n_chunks) after the last chosen block or at chunk n_chunks.
+struct MobaWalk {
+    int j = -1, r = 0;
+};
+__device__ __forceinline__ int moba_walk_next(MobaWalk &w, const uint32_t *chosen, int nb, int cpb, int n_chunks)
+{
+    if (w.j >= 0 && w.r + 1 < cpb && w.j * cpb + w.r + 1 < n_chunks) return w.j * cpb + ++w.r;
+    int jj = w.j + 1;
+    while (jj < nb) {
+        const uint32_t bits = chosen[jj >> 5] >> (jj & 31);
+        if (bits) {
+            jj += __ffs(bits) - 1;
+            break;
+        }
+        jj = (jj | 31) + 1;
+    }
+    w.j = jj;
+    w.r = 0;
+    return jj < nb ? min(jj * cpb, n_chunks) : n_chunks;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_constant__ CUtensorMap tmap, int64_t page_cap, int S,
                                                                   int64_t len, const bf16 *q, int H, int block, int nb, int K,
@@ -461,31 +483,31 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
     __syncthreads();
     tcgen05_after_sync();
     const uint32_t tb = tbase;
-    // number of chunks the CTA walks in one pass
+    // number of chunks the CTA walks in one pass: the chunks of the chosen blocks, below the CTA's last chunk
+    const int cpb = block / kMobaChunk;
+    const int ppc = kMobaChunk / S;                  // pages of a chunk (a page holds 16 or 64 positions)
     int n = 0;
-    for (int c = 0; c < n_chunks_all; ++c) {
-        const int j = (int)(((int64_t)c * kMobaChunk) / block);
-        n += (umask[j >> 5] >> (j & 31)) & 1u;
-    }
-    // the chunk after `c` that belongs to a chosen block (the walk of both roles)
-    auto next_chunk = [&](int c) {
-        for (++c; c < n_chunks_all; ++c) {
-            const int j = (int)(((int64_t)c * kMobaChunk) / block);
-            if ((umask[j >> 5] >> (j & 31)) & 1u) break;
+    for (int wd = 0; wd < words; ++wd) {
+        uint32_t bits = umask[wd];
+        while (bits) {
+            const int j = wd * 32 + __ffs(bits) - 1;
+            bits &= bits - 1;
+            n += max(0, min(cpb, n_chunks_all - j * cpb));
         }
-        return c;
-    };
+    }
+    // the next chunk of a walk (both roles walk the same chunks in the same order)
+    auto next_chunk = [&](MobaWalk &w) { return moba_walk_next(w, umask, nb, cpb, n_chunks_all); };
     bool ok = true;
 
     if (warp == kMobaMmaWarps) {
         if (lane == 0) {
             // ---- copies and products; hh counts the chunks of pass 2
-            int ck_issue = -1, cv_issue = -1;        // chunk walk of pass 2's key copies and value copies
+            MobaWalk wk, wv, w1;                     // chunk walks of pass 2's key copies and value copies, and of pass 1
             int gk_issued = 0, hv_issued = 0, gk_landed = 0, hv_landed = 0;
             auto issue_k = [&]() {                   // keys of the next chunk of the walk into stage gk_issued % NST
-                ck_issue = next_chunk(ck_issue);
+                const int ck_issue = next_chunk(wk);
                 const int st = gk_issued % NST;
-                const int page = (int)((int64_t)bh * page_cap + ((int64_t)ck_issue * kMobaChunk) / S);
+                const int page = (int)((int64_t)bh * page_cap + ck_issue * ppc);
                 mbar_arrive_expect_tx(&full_k[st], G::KC_BYTES);
 #pragma unroll
                 for (int hf = 0; hf < G::HALVES; ++hf)
@@ -493,9 +515,9 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
                 ++gk_issued;
             };
             auto issue_v = [&]() {
-                cv_issue = next_chunk(cv_issue);
+                const int cv_issue = next_chunk(wv);
                 const int st = hv_issued % NST;
-                const int page = (int)((int64_t)bh * page_cap + ((int64_t)cv_issue * kMobaChunk) / S);
+                const int page = (int)((int64_t)bh * page_cap + cv_issue * ppc);
                 mbar_arrive_expect_tx(&full_v[st], G::KC_BYTES);
 #pragma unroll
                 for (int hf = 0; hf < G::HALVES; ++hf)
@@ -520,14 +542,14 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             // are its two stages; two accumulators of 128 columns (the columns pass 2 uses for scores, output and weights)
             const uint32_t qa = smem_addr(qs);
             const int n1 = (n + 1) / 2;
-            int c1 = -1, issued1 = 0, landed1 = 0;
+            int issued1 = 0, landed1 = 0;
             auto issue1 = [&](int it) {
                 unsigned char *dst = (it & 1) ? vst : kst;
                 const int cnt = min(2, n - 2 * it);
                 mbar_arrive_expect_tx(&full1[it & 1], (uint32_t)cnt * G::KC_BYTES);
                 for (int u = 0; u < cnt; ++u) {
-                    c1 = next_chunk(c1);
-                    const int page = (int)((int64_t)bh * page_cap + ((int64_t)c1 * kMobaChunk) / S);
+                    const int c1 = next_chunk(w1);
+                    const int page = (int)((int64_t)bh * page_cap + c1 * ppc);
 #pragma unroll
                     for (int hf = 0; hf < G::HALVES; ++hf)
                         tma_load_4d(dst + hf * (128 * 128) + u * (kMobaChunk * 128), &tmap, hf * 64, 0, 0, page, &full1[it & 1]);
@@ -602,18 +624,18 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
         const uint32_t tl = tb + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t *mymask = qmask + lq * words;
         float m = -CUDART_INF_F, l = 0.0f, inv_l = 0.0f;
-        int c = -1;
+        MobaWalk wr;
         // ---- pass 1: the maximum of the scores this query attends.  A product covers two chunks; of a query's two
         // threads the first takes the first chunk, the second the other one.
         const int n1 = (n + 1) / 2;
 #pragma unroll 1
         for (int it = 0; it < n1; ++it) {
-            const int ca = next_chunk(c), cb2 = 2 * it + 1 < n ? next_chunk(ca) : -1;
-            c = cb2 >= 0 ? cb2 : ca;
+            const int ca = next_chunk(wr), ja = wr.j;
+            const int cb2 = 2 * it + 1 < n ? next_chunk(wr) : -1;
             const int cm = ch == 0 ? ca : cb2;       // this thread's chunk (none: -1)
             int nv = 0;
             if (cm >= 0 && tq < len) {
-                const int j = (int)(((int64_t)cm * kMobaChunk) / block);
+                const int j = ch == 0 ? ja : wr.j;
                 if ((mymask[j >> 5] >> (j & 31)) & 1u) nv = (int)max((int64_t)0, min((int64_t)kMobaChunk, tq - (int64_t)cm * kMobaChunk + 1));
             }
             ok = mbar_wait(&s1_ready[it & 1], (uint32_t)((it >> 1) & 1));
@@ -641,13 +663,12 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
             if (__all_sync(FULLMASK, ok)) m = fmaxf(m, stat[ch ^ 1][lq].x);
         }
         // ---- pass 2: the same chunks one by one; of a query's two threads each takes 32 of a chunk's positions
-        c = -1;
+        wr = MobaWalk();
 #pragma unroll 1
         for (int hh = 0; hh < n; ++hh) {
             if (!__all_sync(FULLMASK, ok)) break;
-            c = next_chunk(c);
+            const int c = next_chunk(wr), j = wr.j;
             const int64_t p0 = (int64_t)c * kMobaChunk + ch * 32;    // first of this thread's 32 positions
-            const int j = (int)(((int64_t)c * kMobaChunk) / block);
             // positions this query attends among them: none if it did not choose the block, else those up to its own
             int nv = 0;
             if (tq < len && ((mymask[j >> 5] >> (j & 31)) & 1u)) nv = (int)max((int64_t)0, min((int64_t)32, tq - p0 + 1));
