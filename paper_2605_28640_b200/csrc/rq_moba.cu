@@ -439,8 +439,10 @@ __global__ void __launch_bounds__(kMobaMmaThreads) moba_mma_kernel(const __grid_
     uint32_t *qmask = umask + words;                                     // [128][words] blocks chosen by each query
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
-    const int64_t t0 = (int64_t)blockIdx.x * kMobaMmaQueries;
+    // the work of a CTA grows with the position of its queries (the blocks before them): the CTAs of the last
+    // queries of every head start first, so that the short ones fill the end of the launch
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    const int64_t t0 = (int64_t)(gridDim.y - 1 - blockIdx.y) * kMobaMmaQueries;
     // chunks of 64 positions up to the CTA's last query; chunk c belongs to block c * 64 / block
     const int n_chunks_all = (int)((min(t0 + kMobaMmaQueries, len) + kMobaChunk - 1) / kMobaChunk);
 
@@ -801,7 +803,7 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
         alignas(64) CUtensorMap tmap;
         e = cache_tensor_map(&tmap, a.kv, D, a.S, (int64_t)BH * a.page_cap, kMobaChunk);
         if (e != cudaSuccess) return e;
-        moba_mma_kernel<D><<<dim3((unsigned)((a.len + kMobaMmaQueries - 1) / kMobaMmaQueries), (unsigned)BH), kMobaMmaThreads, ms, s>>>(
+        moba_mma_kernel<D><<<dim3((unsigned)BH, (unsigned)((a.len + kMobaMmaQueries - 1) / kMobaMmaQueries)), kMobaMmaThreads, ms, s>>>(
             tmap, a.page_cap, a.S, a.len, (const bf16 *)a.q, a.H, a.block, nb, a.K, a.sel, sl2, (bf16 *)a.o, a.status);
     } else {
         moba_attend_kernel<T, D><<<dim3((unsigned)((a.len + kMobaQueries - 1) / kMobaQueries), (unsigned)BH), kMobaQueries * 32, as, s>>>(
@@ -828,7 +830,8 @@ void moba_carve(void *scratch, int BH, int64_t len, int D, int block, float **me
 cudaError_t launch_moba(const MobaArgs &a, cudaStream_t s)
 {
     if (a.block < kMobaChunk || a.block % kMobaChunk != 0 || a.block % a.S != 0 || a.K < 2 || a.len < 1) return cudaErrorInvalidValue;
-    if ((a.len + a.block - 1) / a.block > kMobaMaxBlocks || a.B * a.H > 65535) return cudaErrorInvalidValue;
+    if ((a.len + a.block - 1) / a.block > kMobaMaxBlocks || a.B * a.H > 65535 || (a.len + kMobaMmaQueries - 1) / kMobaMmaQueries > 65535)
+        return cudaErrorInvalidValue;
     if (a.dtype == RQ_BF16) {
         if (a.D == 128) return moba_run<bf16, 128>(a, s);
         if (a.D == 64) return moba_run<bf16, 64>(a, s);
