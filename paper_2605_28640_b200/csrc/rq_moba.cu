@@ -8,8 +8,8 @@
 //   moba_route_kernel    per (head, 16 consecutive queries), a warp per query: scores q . mean of the
 //                        complete blocks before the query's own (a lane per block; the head's
 //                        representatives staged in shared memory once per CTA when they fit), then the
-//                        budget's best (equal scores to the lower block) by counting each candidate's
-//                        rank, or by repeated arg-max when the budget is small or the candidates many;
+//                        budget's best (equal scores to the lower block) by a bit-wise search for the
+//                        threshold score, or by repeated arg-max when the budget is small or the candidates many;
 //                        the list written ascending
 //   moba_mma_kernel      bf16 caches.  Per (head, 128 consecutive queries): both contractions on the
 //                        tensor cores (tcgen05.mma, accumulators and the weights in tensor memory),
@@ -74,41 +74,45 @@ __global__ void moba_means_kernel(const T *kv, int64_t page_cap, int S, int D, i
     means[((int64_t)bh * nb + j) * D + c] = s / (float)(hi - lo);
 }
 
-// Ranking by counting for one warp: candidates are the blocks c_lo .. c_hi - 1 with scores sc[]; lane l owns the
-// candidates c_lo + l + 32 r, r < R.  Sets the mask bits of the candidates whose rank is below `want`.  A
-// candidate beats another with a higher score, or the same score and a lower block: one unsigned 64-bit
-// comparison of (order-preserving image of the score, complement of the block).  The scores are replaced by
-// their images in place.
+// The `want` best of the candidate blocks c_lo .. c_hi - 1 with scores sc[], for one warp; lane l owns the
+// candidates c_lo + l + 32 r, r < R.  A candidate beats another with a higher score, or the same score and a lower
+// block.  The score of the want-th best is found bit by bit on the order-preserving integer image of the scores
+// (32 rounds of one comparison and one vote per owned candidate: far fewer operations than ranking every candidate
+// against every other); the candidates above it are taken, and of those equal to it the lowest blocks.  Sets their
+// mask bits.
 template <int R>
-__device__ __forceinline__ void moba_rank_take(float *sc, uint32_t *mask, int c_lo, int c_hi, int want, int lane)
+__device__ __forceinline__ void moba_rank_take(const float *sc, uint32_t *mask, int c_lo, int c_hi, int want, int lane)
 {
-    uint32_t *key = reinterpret_cast<uint32_t *>(sc);
+    uint32_t key[R];
+    bool valid[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const int j = c_lo + lane + 32 * r;
-        if (j < c_hi) {
-            const uint32_t b = __float_as_uint(sc[j] + 0.0f);          // -0 becomes +0
-            key[j] = b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
-        }
+        valid[r] = j < c_hi;
+        const uint32_t b = __float_as_uint((valid[r] ? sc[j] : 0.0f) + 0.0f);     // -0 becomes +0
+        key[r] = b ^ ((b >> 31) ? 0xffffffffu : 0x80000000u);
     }
-    __syncwarp();
-    unsigned long long mine[R];
-    int rank[R];
+    // the largest t with at least `want` keys >= t: the want-th largest key (want <= number of candidates)
+    uint32_t t = 0u;
+#pragma unroll 4
+    for (int bit = 31; bit >= 0; --bit) {
+        const uint32_t trial = t | (1u << bit);
+        int cnt = 0;
+#pragma unroll
+        for (int r = 0; r < R; ++r) cnt += __popc(__ballot_sync(0xffffffffu, valid[r] && key[r] >= trial));
+        if (cnt >= want) t = trial;
+    }
+    int above = 0;
+#pragma unroll
+    for (int r = 0; r < R; ++r) above += __popc(__ballot_sync(0xffffffffu, valid[r] && key[r] > t));
+    int need = want - above;                         // of the candidates equal to the threshold, in block order
+    const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-        const int j = c_lo + lane + 32 * r;
-        mine[r] = j < c_hi ? ((unsigned long long)key[j] << 32) | (uint32_t)~j : ~0ull;
-        rank[r] = 0;
-    }
-    for (int i = c_lo; i < c_hi; ++i) {
-        const unsigned long long other = ((unsigned long long)key[i] << 32) | (uint32_t)~i;
-#pragma unroll
-        for (int r = 0; r < R; ++r) rank[r] += other > mine[r] ? 1 : 0;
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        const int j = c_lo + lane + 32 * r;
-        const unsigned take = __ballot_sync(0xffffffffu, j < c_hi && rank[r] < want);   // blocks c_lo + 32 r + bit
+        const uint32_t eq = __ballot_sync(0xffffffffu, valid[r] && key[r] == t);
+        const bool mine = valid[r] && (key[r] > t || (key[r] == t && __popc(eq & lt) < need));
+        need = max(0, need - __popc(eq));
+        const unsigned take = __ballot_sync(0xffffffffu, mine);          // blocks c_lo + 32 r + bit
         if (lane == 0 && take) {
             const int p = c_lo + 32 * r;
             mask[p >> 5] |= take << (p & 31);
@@ -184,9 +188,8 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
     }
     __syncwarp();
     if (c_hi - c_lo <= 4 * 32 && want >= 8) {
-        // few candidates and more than a handful to take (a round per taken block is cheaper otherwise): a
-        // candidate's rank is the number of candidates that beat it (higher score, or the same score and a lower
-        // block); a lane ranks its own (one, two or four) against all of them, read as broadcasts
+        // few candidates and more than a handful to take (a round per taken block is cheaper otherwise): the
+        // threshold score by bit-wise search, a lane holding one, two or four candidates
         const int ncand = c_hi - c_lo;
         if (ncand <= 32) moba_rank_take<1>(sc, mask, c_lo, c_hi, want, lane);
         else if (ncand <= 64) moba_rank_take<2>(sc, mask, c_lo, c_hi, want, lane);
