@@ -223,6 +223,21 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
     __syncwarp();
     // ascending list from the mask
     int base = 0;
+    if (words <= 4) {
+        // few blocks: a lane looks at its own bit of every word; a chosen block's place in the list is the
+        // number of chosen blocks below it
+        const uint32_t lt = (1u << lane) - 1u;
+        for (int r = 0; r < words; ++r) {
+            const uint32_t w = mask[r];
+            if ((w >> lane) & 1u) {
+                const int pos = base + __popc(w & lt);
+                if (pos < K) out[pos] = r * 32 + lane;
+            }
+            base += __popc(w);
+        }
+        for (int i = base + lane; i < K; i += 32) out[i] = -1;
+        return;
+    }
     for (int w0 = 0; w0 < words; w0 += 32) {
         const uint32_t w = w0 + lane < words ? mask[w0 + lane] : 0u;
         const int cnt = __popc(w);
