@@ -36,7 +36,8 @@ namespace {
 
 constexpr int kMobaChunk = 64;                 // positions that pass through shared memory at a time
 constexpr int kMobaQueries = 16;               // queries (warps) of one attention CTA
-constexpr int kMobaRouteWarps = 16;            // queries (warps) of one routing CTA
+constexpr int kMobaRouteWarps = 16;            // warps of one routing CTA
+constexpr int kMobaRouteQ = 2;                 // consecutive queries of one routing warp when the representatives are staged (they share the reads)
 constexpr int kMobaMaxBlocks = 2048;           // blocks of a prompt at most
 constexpr unsigned FULLMASK = 0xffffffffu;
 
@@ -122,71 +123,19 @@ __device__ __forceinline__ void moba_rank_take(const float *sc, uint32_t *mask, 
 }
 
 // ---------------------------------------------------------------- routing
-// Grid (ceil(T / 16), heads); a warp per query.  Shared memory per warp: the query (D floats), the
-// scores of the candidate blocks (nb floats), the chosen blocks as a bit mask (nb / 32 words); and,
-// when they fit (STAGED), the head's representatives for the whole CTA, rows padded by four floats so
-// that the lanes of a quarter-warp, each reading its own row, hit different banks.
+// Grid (ceil(T / queries of a CTA), heads); a warp per query, or per two consecutive queries when the
+// representatives are staged (a lane reads a representative once for both).  Shared memory per query: the
+// query (D floats), the scores of the candidate blocks (nb floats), the chosen blocks as a bit mask
+// (nb / 32 words); and, when they fit (STAGED), the head's representatives for the whole CTA, rows padded
+// by four floats so that the lanes of a quarter-warp, each reading its own row, hit different banks.
 // q: [B][T][H][D].  sel: [BH][T][K], ascending, -1 beyond the chosen blocks.
 constexpr int kMobaStagedBlocks = 128;         // representatives of up to this many blocks are staged in shared memory
 
-template <typename T, int D, bool STAGED>
-__global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const T *q, const float *means, int64_t len, int H,
-                                                                         int block, int nb, int K, int32_t *sel)
+// The selection of one query once the scores of its candidate blocks c_lo .. c_hi - 1 are in sc[]: the `want` best
+// into the mask, the first block(s) and the own block(s) added, the chosen blocks written ascending.  One warp.
+__device__ __forceinline__ void moba_route_finish(const float *sc, uint32_t *mask, int32_t *out, int words, int K, int P, int ns,
+                                                  int nl, int c_lo, int c_hi, int want, int lane)
 {
-    extern __shared__ __align__(16) float rsm[];
-    constexpr int LDM = STAGED ? D + 4 : D;            // floats from one representative to the next
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int words = (nb + 31) / 32;
-    float *qs = rsm + (size_t)warp * moba_route_floats(D, nb);
-    float *sc = qs + D;
-    uint32_t *mask = reinterpret_cast<uint32_t *>(sc + nb);
-    const int bh = blockIdx.y;
-    const float *mh = means + (int64_t)bh * nb * D;
-    if (STAGED) {
-        // the representatives the CTA's queries can need: blocks before the last query's own
-        float *ms = rsm + (size_t)kMobaRouteWarps * moba_route_floats(D, nb);
-        const int64_t t_last = min((int64_t)blockIdx.x * kMobaRouteWarps + kMobaRouteWarps - 1, len - 1);
-        const int need = (int)(t_last / block);
-        for (int i = threadIdx.x; i < need * (D / 4); i += kMobaRouteWarps * 32) {
-            const int j = i / (D / 4), c = i % (D / 4);
-            *reinterpret_cast<float4 *>(ms + j * LDM + 4 * c) = __ldg(reinterpret_cast<const float4 *>(mh + (int64_t)j * D) + c);
-        }
-        __syncthreads();
-        mh = ms;
-    }
-    const int64_t t = (int64_t)blockIdx.x * kMobaRouteWarps + warp;
-    if (t >= len) return;                              // (no CTA-wide barrier below)
-    const int b = bh / H, h = bh % H;
-    int32_t *out = sel + ((int64_t)bh * len + t) * K;
-    const int bt = (int)(t / block), P = bt + 1;       // the query's own block; blocks it may attend
-    if (K >= P) {                                      // everything before the query
-        for (int i = lane; i < K; i += 32) out[i] = i < P ? i : -1;
-        return;
-    }
-    // the first block and the own block inside the budget (K >= 2), as the first and the newest page of a decode step
-    const int ns = min(1, K), nl = min(1, K - ns), want = K - ns - nl;
-    const int c_lo = ns, c_hi = P - nl;                // candidates: blocks c_lo .. c_hi - 1 (all complete)
-    for (int i = lane; i < D; i += 32) qs[i] = load1<T>(q + (((int64_t)b * len + t) * H + h) * D + i);
-    for (int i = lane; i < words; i += 32) mask[i] = 0u;
-    __syncwarp();
-    // scores: a lane per block, the block's representative read as 16-byte pieces
-    for (int j0 = c_lo; j0 < c_hi; j0 += 32) {
-        const int j = j0 + lane;
-        if (j < c_hi) {
-            const float4 *row = reinterpret_cast<const float4 *>(mh + (int64_t)j * LDM);
-            // packed pairs: the even and the odd channels are summed apart and added at the end
-            float2 s2 = make_float2(0.0f, 0.0f);
-#pragma unroll 8
-            for (int i = 0; i < D / 4; ++i) {
-                const float4 m4 = STAGED ? row[i] : __ldg(row + i);
-                const float4 q4 = *reinterpret_cast<const float4 *>(qs + 4 * i);
-                s2 = fma2(make_float2(q4.x, q4.y), make_float2(m4.x, m4.y), s2);
-                s2 = fma2(make_float2(q4.z, q4.w), make_float2(m4.z, m4.w), s2);
-            }
-            sc[j] = s2.x + s2.y;
-        }
-    }
-    __syncwarp();
     if (c_hi - c_lo <= 4 * 32 && want >= 8) {
         // few candidates and more than a handful to take (a round per taken block is cheaper otherwise): the
         // threshold score by bit-wise search, a lane holding one, two or four candidates
@@ -258,6 +207,96 @@ __global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const 
         base += __shfl_sync(FULLMASK, inc, 31);
     }
     for (int i = base + lane; i < K; i += 32) out[i] = -1;
+}
+
+template <typename T, int D, bool STAGED>
+__global__ void __launch_bounds__(kMobaRouteWarps * 32) moba_route_kernel(const T *q, const float *means, int64_t len, int H,
+                                                                         int block, int nb, int K, int32_t *sel)
+{
+    extern __shared__ __align__(16) float rsm[];
+    constexpr int LDM = STAGED ? D + 4 : D;            // floats from one representative to the next
+    constexpr int QW = STAGED ? kMobaRouteQ : 1, QC = kMobaRouteWarps * QW;   // queries of a warp, of the CTA
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int words = (nb + 31) / 32;
+    const int per = moba_route_floats(D, nb);
+    float *wsm = rsm + (size_t)warp * QW * per;        // this warp's queries, scores and masks
+    const int bh = blockIdx.y;
+    const float *mh = means + (int64_t)bh * nb * D;
+    if (STAGED) {
+        // the representatives the CTA's queries can need: blocks before the last query's own
+        float *ms = rsm + (size_t)kMobaRouteWarps * QW * per;
+        const int64_t t_last = min((int64_t)blockIdx.x * QC + QC - 1, len - 1);
+        const int need = (int)(t_last / block);
+        for (int i = threadIdx.x; i < need * (D / 4); i += kMobaRouteWarps * 32) {
+            const int j = i / (D / 4), c = i % (D / 4);
+            *reinterpret_cast<float4 *>(ms + j * LDM + 4 * c) = __ldg(reinterpret_cast<const float4 *>(mh + (int64_t)j * D) + c);
+        }
+        __syncthreads();
+        mh = ms;
+    }
+    const int b = bh / H, h = bh % H;
+    // the first block and the own block inside the budget (K >= 2), as the first and the newest page of a decode step
+    const int ns = min(1, K), nl = min(1, K - ns), want = K - ns - nl;
+    const int c_lo = ns;
+    int P[QW], c_hi[QW];                               // blocks a query may attend; its candidates end before c_hi
+    bool active[QW];
+    int c_hi_max = 0;
+#pragma unroll
+    for (int u = 0; u < QW; ++u) {
+        const int64_t t = (int64_t)blockIdx.x * QC + warp * QW + u;
+        active[u] = false;
+        P[u] = c_hi[u] = 0;
+        if (t >= len) continue;                        // (no CTA-wide barrier below)
+        int32_t *out = sel + ((int64_t)bh * len + t) * K;
+        P[u] = (int)(t / block) + 1;
+        if (K >= P[u]) {                               // everything before the query
+            for (int i = lane; i < K; i += 32) out[i] = i < P[u] ? i : -1;
+            continue;
+        }
+        active[u] = true;
+        c_hi[u] = P[u] - nl;                           // candidates: blocks c_lo .. c_hi - 1 (all complete)
+        c_hi_max = max(c_hi_max, c_hi[u]);
+        float *qs = wsm + u * per;
+        uint32_t *mask = reinterpret_cast<uint32_t *>(qs + D + nb);
+        for (int i = lane; i < D; i += 32) qs[i] = load1<T>(q + (((int64_t)b * len + t) * H + h) * D + i);
+        for (int i = lane; i < words; i += 32) mask[i] = 0u;
+    }
+    if (c_hi_max == 0) return;
+    __syncwarp();
+    // scores: a lane per block, the block's representative read as 16-byte pieces once for the warp's queries
+    for (int j0 = c_lo; j0 < c_hi_max; j0 += 32) {
+        const int j = j0 + lane;
+        if (j < c_hi_max) {
+            const float4 *row = reinterpret_cast<const float4 *>(mh + (int64_t)j * LDM);
+            // packed pairs: the even and the odd channels are summed apart and added at the end
+            float2 s2[QW];
+#pragma unroll
+            for (int u = 0; u < QW; ++u) s2[u] = make_float2(0.0f, 0.0f);
+#pragma unroll 8
+            for (int i = 0; i < D / 4; ++i) {
+                const float4 m4 = STAGED ? row[i] : __ldg(row + i);
+#pragma unroll
+                for (int u = 0; u < QW; ++u) {
+                    if (!active[u]) continue;          // (the same for the whole warp)
+                    const float4 q4 = *reinterpret_cast<const float4 *>(wsm + u * per + 4 * i);
+                    s2[u] = fma2(make_float2(q4.x, q4.y), make_float2(m4.x, m4.y), s2[u]);
+                    s2[u] = fma2(make_float2(q4.z, q4.w), make_float2(m4.z, m4.w), s2[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < QW; ++u)
+                if (active[u] && j < c_hi[u]) (wsm + u * per + D)[j] = s2[u].x + s2[u].y;
+        }
+    }
+    __syncwarp();
+#pragma unroll
+    for (int u = 0; u < QW; ++u) {
+        if (!active[u]) continue;
+        const int64_t t = (int64_t)blockIdx.x * QC + warp * QW + u;
+        float *sc = wsm + u * per + D;
+        moba_route_finish(sc, reinterpret_cast<uint32_t *>(sc + nb), sel + ((int64_t)bh * len + t) * K, words, K, P[u], ns, nl, c_lo,
+                          c_hi[u], want, lane);
+    }
 }
 
 // ---------------------------------------------------------------- attention
@@ -780,7 +819,8 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
     moba_means_kernel<T><<<dim3((unsigned)nb, (unsigned)BH), D, 0, s>>>((const T *)a.kv, a.page_cap, a.S, D, a.len, a.block,
                                                                       a.means, nb);
     const bool staged = nb <= kMobaStagedBlocks;
-    const size_t rs = (size_t)kMobaRouteWarps * moba_route_floats(D, nb) * sizeof(float) + (staged ? (size_t)nb * (D + 4) * sizeof(float) : 0);
+    const int rq = staged ? kMobaRouteQ : 1;         // queries of a routing warp
+    const size_t rs = (size_t)kMobaRouteWarps * rq * moba_route_floats(D, nb) * sizeof(float) + (staged ? (size_t)nb * (D + 4) * sizeof(float) : 0);
     constexpr int CHUNK_BYTES = 2 * kMobaChunk * D * (int)sizeof(T);
     const size_t as = 2 * (size_t)CHUNK_BYTES + (size_t)words * (kMobaQueries + 1) * sizeof(uint32_t);
     static bool ready[64];
@@ -793,7 +833,7 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
                                  (int)((size_t)kMobaRouteWarps * moba_route_floats(D, kMobaMaxBlocks) * sizeof(float)));
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(moba_route_kernel<T, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)((size_t)kMobaRouteWarps * moba_route_floats(D, kMobaStagedBlocks) * sizeof(float) +
+                                 (int)((size_t)kMobaRouteWarps * kMobaRouteQ * moba_route_floats(D, kMobaStagedBlocks) * sizeof(float) +
                                        (size_t)kMobaStagedBlocks * (D + 4) * sizeof(float)));
         if (e != cudaSuccess) return e;
         e = cudaFuncSetAttribute(moba_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -801,7 +841,7 @@ cudaError_t moba_run(const MobaArgs &a, cudaStream_t s)
         if (e != cudaSuccess) return e;
         ready[dev] = true;
     }
-    const dim3 rgrid((unsigned)((a.len + kMobaRouteWarps - 1) / kMobaRouteWarps), (unsigned)BH);
+    const dim3 rgrid((unsigned)((a.len + kMobaRouteWarps * rq - 1) / (kMobaRouteWarps * rq)), (unsigned)BH);
     if (staged)
         moba_route_kernel<T, D, true><<<rgrid, kMobaRouteWarps * 32, rs, s>>>((const T *)a.q, a.means, a.len, a.H, a.block, nb, a.K, a.sel);
     else
