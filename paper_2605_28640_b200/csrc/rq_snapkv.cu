@@ -178,7 +178,7 @@ constexpr int kMmaKeys = 128;                  // keys per tile
 constexpr int kMmaWarps = 4;                   // warps that read the accumulator: one thread per lane of it
 constexpr int kMmaThreads = (kMmaWarps + 1) * 32;   // and one warp that starts the copies and the products
 constexpr int kMmaStages = 2;                  // key tiles in shared memory: 97 KB with the queries, so that two CTAs share an SM
-constexpr int kMmaMaxTiles = 32;               // tiles per CTA at most
+constexpr int kMmaMaxTiles = 32;               // tiles per CTA: the search goes up to twice this
 
 template <int D>
 struct SnapMmaGeom {
@@ -633,9 +633,19 @@ cudaError_t snap_scores_mma(const SnapArgs &a, cudaStream_t s)
     e = cache_tensor_map(&tmap, a.kv, D, a.S, (int64_t)BH * a.page_cap, kMmaKeys);
     if (e != cudaSuccess) return e;
     const int ntiles = (int)((a.len + kMmaKeys - 1) / kMmaKeys);
-    // tiles per CTA: as many as leave a couple of CTAs for every SM
-    int tpc = kMmaMaxTiles;
-    while (tpc > 1 && (int64_t)BH * ((ntiles + tpc - 1) / tpc) < 2 * (int64_t)sm_count()) tpc >>= 1;
+    // tiles per CTA: two CTAs share an SM, so the launch runs in rounds of 2 * SMs CTAs; the choice with the fewest
+    // rounds * (tiles of a CTA + what a CTA costs before its first tile, about two tiles' time) ends soonest
+    const int64_t slots = 2 * (int64_t)sm_count();
+    int tpc = 1;
+    int64_t best = INT64_MAX;
+    for (int c = 1; c <= kMmaMaxTiles * 2 && c <= ntiles; ++c) {
+        const int64_t ctas = (int64_t)BH * ((ntiles + c - 1) / c);
+        const int64_t cost = ((ctas + slots - 1) / slots) * (c + 2);
+        if (cost <= best) {                            // equal cost: the longer runs (fewer partial statistics)
+            best = cost;
+            tpc = c;
+        }
+    }
     const int runs = (ntiles + tpc - 1) / tpc;
     const dim3 grid((unsigned)runs, (unsigned)BH);
     const float sl2 = a.scale * 1.4426950408889634f;
