@@ -178,6 +178,7 @@ constexpr int kMmaKeys = 128;                  // keys per tile
 constexpr int kMmaWarps = 4;                   // warps that read the accumulator: one thread per lane of it
 constexpr int kMmaThreads = (kMmaWarps + 1) * 32;   // and one warp that starts the copies and the products
 constexpr int kMmaStages = 2;                  // key tiles in shared memory: 97 KB with the queries, so that two CTAs share an SM
+constexpr int kMmaAhead = 3;                   // tiles between an L2 prefetch and the copy of the same keys
 constexpr int kMmaMaxTiles = 32;               // tiles per CTA: the search goes up to twice this
 
 template <int D>
@@ -258,6 +259,12 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
 #pragma unroll
         for (int hh = 0; hh < G::HALVES; ++hh) tma_load_4d(dst + hh * G::HALF_BYTES, &tmap, hh * 64, 0, 0, page, &full[stage]);
         n_issued = i + 1;
+        // two stages keep too few bytes on their way from DRAM for its latency: the keys of a later tile of this
+        // CTA are asked into L2 now, so that their copy is short when its turn comes
+        if (i + kMmaAhead < n) {
+#pragma unroll
+            for (int hh = 0; hh < G::HALVES; ++hh) tma_prefetch_4d(&tmap, hh * 64, 0, 0, page + kMmaAhead * ppt);
+        }
     };
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the queries, written with ordinary stores, are read by the tensor core
     tcgen05_before_sync();
@@ -272,6 +279,11 @@ __global__ void __launch_bounds__(kMmaThreads) snap_mma_kernel(const __grid_cons
         // ---- the producing warp: one thread starts the copies and the products; nobody else waits for it
         // except through the barriers
         if (lane == 0) {
+            for (int t = NST; t < kMmaAhead && t < n; ++t) {       // the tiles between the first copies and the first prefetch
+                const int page = (int)((int64_t)bh * page_cap + (int64_t)(t0 + t) * ppt);
+#pragma unroll
+                for (int hh = 0; hh < G::HALVES; ++hh) tma_prefetch_4d(&tmap, hh * 64, 0, 0, page);
+            }
             for (int s = 0; s < NST && s < n; ++s) issue(s);
             constexpr uint32_t idesc = PASS == 1 ? umma_idesc_bf16(128, kMmaKeys) : umma_idesc_bf16(kMmaKeys, kSnapRows);
             const uint32_t qa = smem_addr(qs);

@@ -56,6 +56,15 @@ __device__ __forceinline__ void tma_load_4d(void *dst_smem, const void *tmap, in
         : "memory");
 }
 
+// The same box brought into L2 only (no shared memory, no barrier): a hint issued a few tiles ahead of the copy
+// itself, so that the copy finds its bytes in L2.  One thread.
+__device__ __forceinline__ void tma_prefetch_4d(const void *tmap, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(tmap), "r"(c0), "r"(c1), "r"(c2),
+                 "r"(c3)
+                 : "memory");
+}
+
 // instruction descriptor of D[M x N] (fp32) = A[M x 16] (bf16, K-major) * B[N x 16]^T (bf16, K-major)
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N)
 {
